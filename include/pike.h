@@ -1,0 +1,178 @@
+/*
+ * pike.h — C ABI of the fused operator-chain library for NVIDIA B200 (sm_100a).
+ *
+ * The paper (arxiv 2511.16964, Section 5.3 "Task-wise Benchmark Analysis") names
+ * the optimisation pattern this library implements: fuse a heavy operator (a
+ * dense GEMM) with the pointwise and row-reduction operators that follow it into
+ * one kernel, so intermediates never round-trip through HBM and launch overhead
+ * disappears, and replace naive attention by a flash-attention kernel with
+ * on-the-fly causal masking (Appendix C, "VisionAttention", "MinGPT",
+ * "HunyuanVideo").  The paper gives no formulas for the operators; each entry
+ * point below states the textbook definition it computes.
+ *
+ * Conventions
+ *  - Plain C, no exceptions cross the boundary; every function returns
+ *    pike_status_t (PIKE_OK == 0).
+ *  - Every tensor is CALLER-OWNED DEVICE MEMORY on the handle's device, borrowed
+ *    until the enqueued work has finished.  Tensors are row-major with element
+ *    strides; the innermost stride must be 1 and the base address 16-byte
+ *    aligned.  The library never allocates per call: scratch comes from a caller
+ *    supplied workspace (device memory, 256-byte aligned) whose size the matching
+ *    *_workspace query returns.
+ *  - Calls enqueue on the caller's CUDA stream (a cudaStream_t passed as void*,
+ *    NULL = default stream) and return without synchronising.  The return value
+ *    reports host-detectable errors only.  Device-detected conditions (a bounded
+ *    wait inside a kernel that ran out) land in a status word that
+ *    pike_get_last_device_status reads after the caller has synchronised.
+ *  - There is no CPU or library fallback: a device that is not compute
+ *    capability 10.x yields PIKE_ERR_ARCH, an unsupported shape or combination
+ *    PIKE_ERR_UNSUPPORTED.
+ */
+#ifndef PIKE_H_
+#define PIKE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PIKE_OK = 0,
+    PIKE_ERR_NULL = 1,        /* a required pointer is NULL                              */
+    PIKE_ERR_SHAPE = 2,       /* ranks / extents do not fit together                     */
+    PIKE_ERR_DTYPE = 3,       /* dtype combination not accepted by this entry point      */
+    PIKE_ERR_ALIGNMENT = 4,   /* base pointer or row pitch not 16-byte aligned           */
+    PIKE_ERR_STRIDE = 5,      /* innermost stride != 1 or a non-dense layout             */
+    PIKE_ERR_UNSUPPORTED = 6, /* valid request outside the implemented envelope          */
+    PIKE_ERR_WORKSPACE = 7,   /* workspace NULL / misaligned / too small                 */
+    PIKE_ERR_ARCH = 8,        /* device is not sm_100                                    */
+    PIKE_ERR_CUDA = 9,        /* a CUDA runtime or driver call failed                    */
+    PIKE_ERR_TIMEOUT = 10     /* device status only: a bounded in-kernel wait ran out    */
+} pike_status_t;
+
+typedef enum { PIKE_F32 = 0, PIKE_BF16 = 1 } pike_dtype_t;
+
+/* A view of caller-owned device memory.  stride[] is in elements. */
+typedef struct {
+    void *data;
+    pike_dtype_t dtype;
+    int32_t ndim;             /* 1..4 */
+    int64_t shape[4];
+    int64_t stride[4];
+} pike_tensor_t;
+
+typedef enum { PIKE_ACT_NONE = 0, PIKE_ACT_GELU_ERF = 1, PIKE_ACT_GELU_TANH = 2, PIKE_ACT_SILU = 3 } pike_act_t;
+typedef enum { PIKE_REDUCE_NONE = 0, PIKE_REDUCE_LAYERNORM = 1, PIKE_REDUCE_SOFTMAX = 2 } pike_reduce_t;
+
+#define PIKE_FLAG_W_IS_NK 0x1u /* weight tensors are [N,K] ("out,in") instead of [K,N]   */
+#define PIKE_FLAG_CAUSAL  0x2u /* attention: key j takes part for query i only if j <= i */
+
+/* Epilogue descriptor: what follows the GEMM inside the same kernel. */
+typedef struct {
+    uint32_t struct_size;     /* sizeof(pike_epilogue_t), for forward compatibility      */
+    pike_act_t act;           /* activation applied to (acc + bias)                      */
+    float scale;              /* multiplies the activation (1.0f = off); attention: the  */
+                              /* factor applied to q.k before the softmax                */
+    pike_reduce_t reduce;     /* row reduction over N applied last                       */
+    float eps;                /* LayerNorm epsilon (inside the square root)              */
+    pike_dtype_t out_dtype;   /* must equal out->dtype                                   */
+    uint32_t flags;           /* PIKE_FLAG_*                                             */
+} pike_epilogue_t;
+
+typedef struct pike_handle_s *pike_handle_t;
+
+/* Create / destroy a handle for CUDA device `device`.  The handle caches device
+ * properties and owns a 16-byte device status word (its only allocation).  A
+ * handle is not thread-safe; use one per host thread.  PIKE_ERR_ARCH if the
+ * device is not compute capability 10.x. */
+pike_status_t pike_create(pike_handle_t *handle, int device);
+pike_status_t pike_destroy(pike_handle_t handle);
+
+/* Static, never-freed description of a status code. */
+const char *pike_status_string(pike_status_t status);
+
+/* Reads (and clears) the device status word.  Synchronises the device.
+ * *status is PIKE_OK or PIKE_ERR_TIMEOUT; *where identifies the wait that gave
+ * up (kernel id << 16 | barrier id). */
+pike_status_t pike_get_last_device_status(pike_handle_t handle, pike_status_t *status, uint32_t *where);
+
+/* Test hook: upper bound, in nanoseconds, for every in-kernel wait of kernels
+ * launched through this handle afterwards (default 2e9).  0 restores the default. */
+pike_status_t pike_set_wait_limit_ns(pike_handle_t handle, uint64_t ns);
+
+/*
+ * Linear + epilogue chain (the "operator fusion" pattern of Section 5.3):
+ *
+ *   v[m,n]   = scale * act( sum_k x[m,k] * w[k,n] + bias[n] ) + residual[m,n]
+ *   out[m,:] = v[m,:]                                   reduce == NONE
+ *            = (v - mean)/sqrt(var + eps) * gamma + beta reduce == LAYERNORM (biased var)
+ *            = exp(v - max v) / sum exp(v - max v)       reduce == SOFTMAX
+ *
+ * x [M,K]; w [K,N] (or [N,K] with PIKE_FLAG_W_IS_NK); bias, gamma, beta [N];
+ * residual, out [M,N].  bias, residual, gamma, beta may be NULL (0, 0, 1, 0).
+ *
+ * fp32 path (x, w, out all PIKE_F32; bias/residual/gamma/beta F32): true fp32
+ *   FMA on the CUDA cores; any M, K; N <= 1024; every reduce mode.
+ * bf16 path (x, w PIKE_BF16; bias/residual/gamma/beta BF16 or F32): tcgen05
+ *   tensor-core GEMM with fp32 accumulation; K and N multiples of 8; out BF16 or
+ *   F32 for reduce NONE; reduce SOFTMAX needs out F32 (rows are split across N
+ *   tiles, partial (max, sum) pairs go to the workspace and a second kernel
+ *   normalises in place); reduce LAYERNORM on this path is PIKE_ERR_UNSUPPORTED.
+ * out must not alias any input (PIKE_ERR_UNSUPPORTED if the ranges overlap).
+ *
+ * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless
+ * the bf16 softmax path is taken); it reads only shapes and dtypes.
+ */
+pike_status_t pike_linear_epilogue_workspace(pike_handle_t handle, const pike_tensor_t *x,
+                                             const pike_tensor_t *w, const pike_epilogue_t *epi,
+                                             size_t *bytes);
+pike_status_t pike_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
+                                   const pike_tensor_t *bias, const pike_tensor_t *residual,
+                                   const pike_tensor_t *gamma, const pike_tensor_t *beta,
+                                   const pike_epilogue_t *epi, pike_tensor_t *out, void *workspace,
+                                   size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Pre-LayerNorm transformer MLP block (sub-graph fusion, Section 5.3):
+ *
+ *   z   = LayerNorm(x; gamma, beta, eps)            over the last dimension D
+ *   h   = act( z @ w1 + b1 )                         [M,F]
+ *   out = x + h @ w2 + b2                            [M,D]   (residual = un-normalised x)
+ *
+ * All tensors PIKE_BF16 (gamma, beta, b1, b2 may be F32); x, out [M,D]; w1 [D,F];
+ * w2 [F,D] (or transposed with PIKE_FLAG_W_IS_NK); D, F multiples of 8, D <= 16384.
+ * epi->act selects the activation, epi->eps the LayerNorm epsilon; scale must be 1
+ * and reduce NONE.  z and h are rounded to bf16 and live in the workspace
+ * (M*D*2 + M*F*2 bytes, each part 256-byte aligned).  Three kernels are enqueued
+ * on the stream.
+ */
+pike_status_t pike_mlp_block_workspace(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w1,
+                                       const pike_epilogue_t *epi, size_t *bytes);
+pike_status_t pike_mlp_block(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *gamma,
+                             const pike_tensor_t *beta, const pike_tensor_t *w1, const pike_tensor_t *b1,
+                             const pike_tensor_t *w2, const pike_tensor_t *b2, const pike_epilogue_t *epi,
+                             pike_tensor_t *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Attention chain (flash attention with on-the-fly causal masking, Appendix C):
+ *
+ *   s[i,j]  = epi->scale * sum_d q[i,d] * k[j,d]
+ *   out[i,:] = sum_j softmax_j(s[i,.])[j] * v[j,:]   (j <= i only with PIKE_FLAG_CAUSAL)
+ *
+ * per (batch, head).  q, k, v, out are dense [B,H,S,D] PIKE_BF16, D == 128,
+ * S_q == S_k, any S >= 1.  The score matrix lives in tensor memory and registers
+ * only; probabilities are rounded to bf16 before the second GEMM.  Workspace: 0
+ * bytes (the query exists for symmetry).
+ */
+pike_status_t pike_attention_chain_workspace(pike_handle_t handle, const pike_tensor_t *q,
+                                             const pike_epilogue_t *epi, size_t *bytes);
+pike_status_t pike_attention_chain(pike_handle_t handle, const pike_tensor_t *q, const pike_tensor_t *k,
+                                   const pike_tensor_t *v, const pike_epilogue_t *epi, pike_tensor_t *out,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PIKE_H_ */

@@ -1,0 +1,242 @@
+"""ctypes binding of ``libpike.so``: argument marshalling only.
+
+Every function has the name of the C entry point it calls.  torch is used for
+device memory (outputs, workspaces) and the current CUDA stream; all arithmetic
+runs in the library's kernels.  There is no fallback: if the shared library is
+missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libpike.so")
+
+PIKE_F32, PIKE_BF16 = 0, 1
+ACT = {"none": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
+REDUCE = {"none": 0, "layernorm": 1, "softmax": 2}
+FLAG_W_IS_NK, FLAG_CAUSAL = 0x1, 0x2
+
+EXPORTS = (
+    "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
+    "pike_set_wait_limit_ns", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
+    "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
+    "pike_attention_chain",
+)
+
+
+class PikeError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: status {code} ({pike_status_string(code)})")
+        self.code = code
+
+
+class pike_tensor_t(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("dtype", ctypes.c_int), ("ndim", ctypes.c_int32),
+                ("shape", ctypes.c_int64 * 4), ("stride", ctypes.c_int64 * 4)]
+
+
+class pike_epilogue_t(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_uint32), ("act", ctypes.c_int), ("scale", ctypes.c_float),
+                ("reduce", ctypes.c_int), ("eps", ctypes.c_float), ("out_dtype", ctypes.c_int),
+                ("flags", ctypes.c_uint32)]
+
+
+_lib = None
+_lock = threading.Lock()
+_handles: dict[int, ctypes.c_void_p] = {}
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libpike.so and declare the prototypes.  Raises if it was not built."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(_LIB_PATH):
+                raise RuntimeError(
+                    f"{_LIB_PATH} is missing: build it with `python -m paper_2511_16964_b200.build` "
+                    "(there is no CPU or PyTorch fallback)")
+            lib = ctypes.CDLL(_LIB_PATH)
+            T, E = ctypes.POINTER(pike_tensor_t), ctypes.POINTER(pike_epilogue_t)
+            vp, sz = ctypes.c_void_p, ctypes.c_size_t
+            lib.pike_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+            lib.pike_destroy.argtypes = [vp]
+            lib.pike_status_string.argtypes = [ctypes.c_int]
+            lib.pike_status_string.restype = ctypes.c_char_p
+            lib.pike_get_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_uint32)]
+            lib.pike_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
+            lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
+            lib.pike_linear_epilogue.argtypes = [vp, T, T, T, T, T, T, E, T, vp, sz, vp]
+            lib.pike_mlp_block_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
+            lib.pike_mlp_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
+            lib.pike_attention_chain_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
+            lib.pike_attention_chain.argtypes = [vp, T, T, T, E, T, vp, sz, vp]
+            for name in EXPORTS:
+                if name != "pike_status_string":
+                    getattr(lib, name).restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def pike_status_string(code: int) -> str:
+    return load_library().pike_status_string(int(code)).decode()
+
+
+def _handle(device: torch.device) -> ctypes.c_void_p:
+    idx = device.index if device.index is not None else torch.cuda.current_device()
+    with _lock:
+        h = _handles.get(idx)
+    if h is None:
+        lib = load_library()
+        h = ctypes.c_void_p()
+        rc = lib.pike_create(ctypes.byref(h), idx)
+        if rc:
+            raise PikeError(rc, "pike_create")
+        with _lock:
+            _handles[idx] = h
+    return h
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return PIKE_F32
+    if t.dtype == torch.bfloat16:
+        return PIKE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _tensor(t):
+    """torch CUDA tensor -> pike_tensor_t (by reference); None -> NULL."""
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("tensors must live in CUDA device memory")
+    d = pike_tensor_t()
+    d.data = t.data_ptr()
+    d.dtype = _dtype_code(t)
+    d.ndim = t.dim()
+    for i in range(t.dim()):
+        d.shape[i] = t.shape[i]
+        d.stride[i] = t.stride(i)
+    return ctypes.byref(d)
+
+
+def _epilogue(act, scale, reduce, eps, out_dtype, flags) -> pike_epilogue_t:
+    e = pike_epilogue_t()
+    e.struct_size = ctypes.sizeof(pike_epilogue_t)
+    e.act = ACT[act]
+    e.scale = float(scale)
+    e.reduce = REDUCE[reduce]
+    e.eps = float(eps)
+    e.out_dtype = PIKE_F32 if out_dtype == torch.float32 else PIKE_BF16
+    e.flags = flags
+    return e
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _workspace(nbytes: int, device, workspace):
+    if workspace is None:
+        workspace = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    return workspace, ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def _check(rc: int, what: str):
+    if rc:
+        raise PikeError(rc, what)
+
+
+def pike_set_wait_limit_ns(ns: int, device=None) -> None:
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    _check(load_library().pike_set_wait_limit_ns(_handle(dev), int(ns)), "pike_set_wait_limit_ns")
+
+
+def pike_get_last_device_status(device=None) -> tuple[int, int]:
+    """(status, where) of the device status word; synchronises the device."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    st, where = ctypes.c_int(0), ctypes.c_uint32(0)
+    _check(load_library().pike_get_last_device_status(_handle(dev), ctypes.byref(st), ctypes.byref(where)),
+           "pike_get_last_device_status")
+    return st.value, where.value
+
+
+def pike_linear_epilogue_workspace(x, w, *, act="none", scale=1.0, reduce="none", eps=1e-5,
+                                   out_dtype=None, w_is_nk=False) -> int:
+    out_dtype = x.dtype if out_dtype is None else out_dtype
+    e = _epilogue(act, scale, reduce, eps, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
+    n = ctypes.c_size_t(0)
+    _check(load_library().pike_linear_epilogue_workspace(_handle(x.device), _tensor(x), _tensor(w),
+                                                         ctypes.byref(e), ctypes.byref(n)),
+           "pike_linear_epilogue_workspace")
+    return n.value
+
+
+def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, *, act="none", scale=1.0,
+                         reduce="none", eps=1e-5, out_dtype=None, w_is_nk=False, out=None, workspace=None,
+                         stream=None):
+    """out = reduce(scale*act(x @ w + bias) + residual); see include/pike.h."""
+    out_dtype = (out.dtype if out is not None else x.dtype) if out_dtype is None else out_dtype
+    N = w.shape[0] if w_is_nk else w.shape[1]
+    if out is None:
+        out = torch.empty((x.shape[0], N), dtype=out_dtype, device=x.device)
+    e = _epilogue(act, scale, reduce, eps, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
+    need = pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps,
+                                          out_dtype=out_dtype, w_is_nk=w_is_nk)
+    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    _check(load_library().pike_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
+                                               _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
+                                               _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
+           "pike_linear_epilogue")
+    return out
+
+
+def pike_mlp_block_workspace(x, w1, *, act="gelu_tanh", eps=1e-5, w_is_nk=False) -> int:
+    e = _epilogue(act, 1.0, "none", eps, torch.bfloat16, FLAG_W_IS_NK if w_is_nk else 0)
+    n = ctypes.c_size_t(0)
+    _check(load_library().pike_mlp_block_workspace(_handle(x.device), _tensor(x), _tensor(w1), ctypes.byref(e),
+                                                   ctypes.byref(n)), "pike_mlp_block_workspace")
+    return n.value
+
+
+def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5, w_is_nk=False, out=None,
+                   workspace=None, stream=None):
+    """out = x + act(LayerNorm(x) @ w1 + b1) @ w2 + b2; see include/pike.h."""
+    if out is None:
+        out = torch.empty_like(x)
+    e = _epilogue(act, 1.0, "none", eps, torch.bfloat16, FLAG_W_IS_NK if w_is_nk else 0)
+    need = pike_mlp_block_workspace(x, w1, act=act, eps=eps, w_is_nk=w_is_nk)
+    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    _check(load_library().pike_mlp_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta), _tensor(w1),
+                                         _tensor(b1), _tensor(w2), _tensor(b2), ctypes.byref(e), _tensor(out),
+                                         ws_ptr, ws_bytes, _stream(stream)), "pike_mlp_block")
+    return out
+
+
+def pike_attention_chain_workspace(q, *, scale, causal=True) -> int:
+    e = _epilogue("none", scale, "none", 0.0, torch.bfloat16, FLAG_CAUSAL if causal else 0)
+    n = ctypes.c_size_t(0)
+    _check(load_library().pike_attention_chain_workspace(_handle(q.device), _tensor(q), ctypes.byref(e),
+                                                         ctypes.byref(n)), "pike_attention_chain_workspace")
+    return n.value
+
+
+def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
+    """out = softmax(scale * q k^T [+ causal mask]) v per (batch, head); see include/pike.h."""
+    if out is None:
+        out = torch.empty_like(q)
+    e = _epilogue("none", scale, "none", 0.0, torch.bfloat16, FLAG_CAUSAL if causal else 0)
+    _check(load_library().pike_attention_chain(_handle(q.device), _tensor(q), _tensor(k), _tensor(v),
+                                               ctypes.byref(e), _tensor(out), None, 0, _stream(stream)),
+           "pike_attention_chain")
+    return out

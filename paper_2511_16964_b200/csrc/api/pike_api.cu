@@ -1,0 +1,480 @@
+// C ABI of the library: argument validation, TMA tensor-map encoding, kernel
+// selection and launch.  Host code only; every arithmetic step runs in the kernels.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../../include/pike.h"
+#include "../kernels/kernels.h"
+
+struct pike_handle_s {
+    int device;
+    int num_sms;
+    unsigned int *status;  // device, 4 words
+    unsigned long long limit_ns;
+    PFN_cuTensorMapEncodeTiled_v12000 encode;
+};
+
+namespace {
+
+constexpr unsigned long long DEFAULT_LIMIT_NS = 2000000000ull;
+
+size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+size_t elem_size(pike_dtype_t t) { return t == PIKE_F32 ? 4 : 2; }
+
+bool valid_dtype(pike_dtype_t t) { return t == PIKE_F32 || t == PIKE_BF16; }
+
+// a dense-enough 2-D view: innermost stride 1, row pitch >= columns, 16-byte aligned base and pitch
+pike_status_t check_matrix(const pike_tensor_t *t, int64_t rows, int64_t cols)
+{
+    if (t == nullptr || t->data == nullptr) return PIKE_ERR_NULL;
+    if (!valid_dtype(t->dtype)) return PIKE_ERR_DTYPE;
+    if (t->ndim != 2 || t->shape[0] != rows || t->shape[1] != cols) return PIKE_ERR_SHAPE;
+    if (t->stride[1] != 1 || t->stride[0] < cols) return PIKE_ERR_STRIDE;
+    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    if ((t->stride[0] * (int64_t)elem_size(t->dtype)) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    return PIKE_OK;
+}
+
+pike_status_t check_vector(const pike_tensor_t *t, int64_t n)
+{
+    if (t == nullptr) return PIKE_OK;  // optional
+    if (t->data == nullptr) return PIKE_ERR_NULL;
+    if (!valid_dtype(t->dtype)) return PIKE_ERR_DTYPE;
+    if (t->ndim != 1 || t->shape[0] != n) return PIKE_ERR_SHAPE;
+    if (t->stride[0] != 1) return PIKE_ERR_STRIDE;
+    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    return PIKE_OK;
+}
+
+void byte_range(const pike_tensor_t *t, uintptr_t &lo, uintptr_t &hi)
+{
+    int64_t last = 0;
+    for (int i = 0; i < t->ndim; ++i) last += (t->shape[i] - 1) * t->stride[i];
+    lo = reinterpret_cast<uintptr_t>(t->data);
+    hi = lo + (uintptr_t)(last + 1) * elem_size(t->dtype);
+}
+
+bool overlaps(const pike_tensor_t *a, const pike_tensor_t *b)
+{
+    if (a == nullptr || b == nullptr || a->data == nullptr || b->data == nullptr) return false;
+    uintptr_t alo, ahi, blo, bhi;
+    byte_range(a, alo, ahi);
+    byte_range(b, blo, bhi);
+    return alo < bhi && blo < ahi;
+}
+
+pike_status_t check_epilogue(const pike_epilogue_t *e)
+{
+    if (e == nullptr) return PIKE_ERR_NULL;
+    if (e->struct_size != sizeof(pike_epilogue_t)) return PIKE_ERR_UNSUPPORTED;
+    if ((int)e->act < 0 || (int)e->act > 3 || (int)e->reduce < 0 || (int)e->reduce > 2) return PIKE_ERR_UNSUPPORTED;
+    if (!valid_dtype(e->out_dtype)) return PIKE_ERR_DTYPE;
+    if (!isfinite(e->scale)) return PIKE_ERR_UNSUPPORTED;
+    return PIKE_OK;
+}
+
+// bf16 [rows, cols] row-major matrix -> tensor map with a (box_cols x box_rows) box, 128-byte swizzle
+pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
+                          uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {pitch_elems * 2};
+    const cuuint32_t box[2] = {box_cols, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+// bf16 [BH, S, D] dense tensor -> 3-D map with a (64 x 128 x 1) box
+pike_status_t make_map_bsd(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t BH, uint64_t S, uint64_t D)
+{
+    const cuuint64_t dims[3] = {D, S, BH};
+    const cuuint64_t strides[2] = {D * 2, S * D * 2};
+    const cuuint32_t box[3] = {64, 128, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+struct LinearShape {
+    int64_t M, K, N;
+    bool w_is_nk;
+    bool fp32_path;
+};
+
+pike_status_t linear_shape(const pike_tensor_t *x, const pike_tensor_t *w, const pike_epilogue_t *epi, LinearShape &s)
+{
+    if (x == nullptr || w == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = check_epilogue(epi)) return st;
+    if (x->ndim != 2 || w->ndim != 2) return PIKE_ERR_SHAPE;
+    if (!valid_dtype(x->dtype) || x->dtype != w->dtype) return PIKE_ERR_DTYPE;
+    s.w_is_nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
+    s.M = x->shape[0];
+    s.K = x->shape[1];
+    s.N = s.w_is_nk ? w->shape[0] : w->shape[1];
+    if ((s.w_is_nk ? w->shape[1] : w->shape[0]) != s.K) return PIKE_ERR_SHAPE;
+    if (s.M < 0 || s.K < 1 || s.N < 1) return PIKE_ERR_SHAPE;
+    if (s.M > 0x7fffffff || s.K > 0x7fffffff || s.N > 0x7fffffff) return PIKE_ERR_UNSUPPORTED;
+    s.fp32_path = x->dtype == PIKE_F32;
+    if (s.fp32_path) {
+        if (s.N > 1024) return PIKE_ERR_UNSUPPORTED;
+        if (epi->out_dtype != PIKE_F32) return PIKE_ERR_DTYPE;
+    } else {
+        if (s.K % 8 != 0 || s.N % 8 != 0) return PIKE_ERR_UNSUPPORTED;
+        if (epi->reduce == PIKE_REDUCE_LAYERNORM) return PIKE_ERR_UNSUPPORTED;
+        if (epi->reduce == PIKE_REDUCE_SOFTMAX && epi->out_dtype != PIKE_F32) return PIKE_ERR_UNSUPPORTED;
+    }
+    return PIKE_OK;
+}
+
+size_t softmax_partials_bytes(const LinearShape &s)
+{
+    const int64_t num_n = (s.N + pike::GEMM_BN - 1) / pike::GEMM_BN;
+    return align256((size_t)s.M * (size_t)num_n * sizeof(float2));
+}
+
+// Launch one bf16 GEMM + epilogue.  All tensors validated by the caller.
+pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pike_tensor_t *w, bool w_is_nk, int64_t M,
+                       int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
+                       void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
+                       cudaStream_t stream)
+{
+    CUtensorMap tmA, tmB;
+    if (pike_status_t st = make_map_2d(h, &tmA, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
+        return st;
+    if (w_is_nk) {
+        if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
+                                           pike::GEMM_BK, pike::GEMM_BN))
+            return st;
+    } else {
+        if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0], 64,
+                                           pike::GEMM_BK))
+            return st;
+    }
+    pike::GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = (int)M; g.N = (int)N; g.K = (int)K;
+    g.w_is_nk = w_is_nk ? 1 : 0;
+    g.bias = bias ? bias->data : nullptr;
+    g.bias_f32 = bias && bias->dtype == PIKE_F32;
+    g.residual = res_ptr; g.residual_f32 = res_f32 ? 1 : 0; g.ldr = ldr;
+    g.out = out_ptr; g.out_f32 = out_f32 ? 1 : 0; g.ldo = ldo;
+    g.act = act; g.scale = scale;
+    g.softmax_partials = partials != nullptr;
+    g.partials = partials;
+    g.status = h->status;
+    g.limit_ns = h->limit_ns;
+    return pike::launch_gemm_bf16(tmA, tmB, g, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *pike_status_string(pike_status_t s)
+{
+    switch (s) {
+    case PIKE_OK:              return "ok";
+    case PIKE_ERR_NULL:        return "a required pointer is NULL";
+    case PIKE_ERR_SHAPE:       return "tensor ranks or extents do not fit together";
+    case PIKE_ERR_DTYPE:       return "dtype combination not accepted";
+    case PIKE_ERR_ALIGNMENT:   return "base pointer or row pitch is not 16-byte aligned";
+    case PIKE_ERR_STRIDE:      return "innermost stride is not 1 or the layout is not dense enough";
+    case PIKE_ERR_UNSUPPORTED: return "request is outside the implemented envelope";
+    case PIKE_ERR_WORKSPACE:   return "workspace is NULL, misaligned or too small";
+    case PIKE_ERR_ARCH:        return "device is not compute capability 10.x (sm_100)";
+    case PIKE_ERR_CUDA:        return "a CUDA runtime or driver call failed";
+    case PIKE_ERR_TIMEOUT:     return "a bounded in-kernel wait ran out";
+    }
+    return "unknown status";
+}
+
+pike_status_t pike_create(pike_handle_t *handle, int device)
+{
+    if (handle == nullptr) return PIKE_ERR_NULL;
+    *handle = nullptr;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { cudaGetLastError(); return PIKE_ERR_CUDA; }
+    if (prop.major != 10) return PIKE_ERR_ARCH;
+    if (cudaSetDevice(device) != cudaSuccess) return PIKE_ERR_CUDA;
+    pike_handle_s *h = new (std::nothrow) pike_handle_s();
+    if (h == nullptr) return PIKE_ERR_CUDA;
+    h->device = device;
+    h->num_sms = prop.multiProcessorCount;
+    h->limit_ns = DEFAULT_LIMIT_NS;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        delete h;
+        return PIKE_ERR_CUDA;
+    }
+    h->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+    if (cudaMalloc(&h->status, 4 * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMemset(h->status, 0, 4 * sizeof(unsigned int)) != cudaSuccess) {
+        delete h;
+        return PIKE_ERR_CUDA;
+    }
+    *handle = h;
+    return PIKE_OK;
+}
+
+pike_status_t pike_destroy(pike_handle_t h)
+{
+    if (h == nullptr) return PIKE_ERR_NULL;
+    cudaFree(h->status);
+    delete h;
+    return PIKE_OK;
+}
+
+pike_status_t pike_get_last_device_status(pike_handle_t h, pike_status_t *status, uint32_t *where)
+{
+    if (h == nullptr || status == nullptr) return PIKE_ERR_NULL;
+    unsigned int host[4] = {0, 0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return PIKE_ERR_CUDA;
+    if (cudaMemcpy(host, h->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (host[0] != 0 && cudaMemset(h->status, 0, sizeof(host)) != cudaSuccess) return PIKE_ERR_CUDA;
+    *status = host[0] != 0 ? PIKE_ERR_TIMEOUT : PIKE_OK;
+    if (where != nullptr) *where = host[0];
+    return PIKE_OK;
+}
+
+pike_status_t pike_set_wait_limit_ns(pike_handle_t h, uint64_t ns)
+{
+    if (h == nullptr) return PIKE_ERR_NULL;
+    h->limit_ns = ns == 0 ? DEFAULT_LIMIT_NS : ns;
+    return PIKE_OK;
+}
+
+pike_status_t pike_linear_epilogue_workspace(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
+                                             const pike_epilogue_t *epi, size_t *bytes)
+{
+    if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
+    LinearShape s;
+    if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
+    *bytes = (!s.fp32_path && epi->reduce == PIKE_REDUCE_SOFTMAX) ? softmax_partials_bytes(s) : 0;
+    return PIKE_OK;
+}
+
+pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
+                                   const pike_tensor_t *bias, const pike_tensor_t *residual,
+                                   const pike_tensor_t *gamma, const pike_tensor_t *beta, const pike_epilogue_t *epi,
+                                   pike_tensor_t *out, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (h == nullptr || out == nullptr) return PIKE_ERR_NULL;
+    LinearShape s;
+    if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
+    if (pike_status_t st = check_matrix(x, s.M, s.K)) return st;
+    if (pike_status_t st = check_matrix(w, s.w_is_nk ? s.N : s.K, s.w_is_nk ? s.K : s.N)) return st;
+    if (pike_status_t st = check_matrix(out, s.M, s.N)) return st;
+    if (out->dtype != epi->out_dtype) return PIKE_ERR_DTYPE;
+    if (pike_status_t st = check_vector(bias, s.N)) return st;
+    if (pike_status_t st = check_vector(gamma, s.N)) return st;
+    if (pike_status_t st = check_vector(beta, s.N)) return st;
+    if (residual != nullptr)
+        if (pike_status_t st = check_matrix(residual, s.M, s.N)) return st;
+    const pike_tensor_t *ins[6] = {x, w, bias, residual, gamma, beta};
+    for (const pike_tensor_t *t : ins)
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (s.M == 0) return PIKE_OK;
+
+    if (s.fp32_path) {
+        for (const pike_tensor_t *t : {bias, residual, gamma, beta})
+            if (t != nullptr && t->dtype != PIKE_F32) return PIKE_ERR_DTYPE;
+        pike::Fp32ChainArgs a;
+        memset(&a, 0, sizeof(a));
+        a.x = static_cast<const float *>(x->data);
+        a.w = static_cast<const float *>(w->data);
+        a.bias = bias ? static_cast<const float *>(bias->data) : nullptr;
+        a.residual = residual ? static_cast<const float *>(residual->data) : nullptr;
+        a.gamma = gamma ? static_cast<const float *>(gamma->data) : nullptr;
+        a.beta = beta ? static_cast<const float *>(beta->data) : nullptr;
+        a.out = static_cast<float *>(out->data);
+        a.M = (int)s.M; a.K = (int)s.K; a.N = (int)s.N;
+        a.ldx = x->stride[0]; a.ldw = w->stride[0]; a.ldr = residual ? residual->stride[0] : 0; a.ldo = out->stride[0];
+        a.w_is_nk = s.w_is_nk;
+        a.act = (int)epi->act; a.reduce = (int)epi->reduce;
+        a.scale = epi->scale; a.eps = epi->eps;
+        return pike::launch_fp32_chain(a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+    }
+
+    float2 *partials = nullptr;
+    if (epi->reduce == PIKE_REDUCE_SOFTMAX) {
+        const size_t need = softmax_partials_bytes(s);
+        if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 || workspace_bytes < need)
+            return PIKE_ERR_WORKSPACE;
+        partials = static_cast<float2 *>(workspace);
+    }
+    if (pike_status_t st = run_gemm(h, x->data, x->stride[0], w, s.w_is_nk, s.M, s.K, s.N, bias,
+                                    residual ? residual->data : nullptr, residual && residual->dtype == PIKE_F32,
+                                    residual ? residual->stride[0] : 0, out->data, out->dtype == PIKE_F32,
+                                    out->stride[0], (int)epi->act, epi->scale, partials, stream))
+        return st;
+    if (partials != nullptr) {
+        const int num_n = (int)((s.N + pike::GEMM_BN - 1) / pike::GEMM_BN);
+        if (pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)s.M,
+                                        (int)s.N, stream) != cudaSuccess)
+            return PIKE_ERR_CUDA;
+    }
+    return PIKE_OK;
+}
+
+static pike_status_t mlp_shape(const pike_tensor_t *x, const pike_tensor_t *w1, const pike_epilogue_t *epi, int64_t &M,
+                               int64_t &D, int64_t &F, bool &nk)
+{
+    if (x == nullptr || w1 == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = check_epilogue(epi)) return st;
+    if (x->ndim != 2 || w1->ndim != 2) return PIKE_ERR_SHAPE;
+    if (x->dtype != PIKE_BF16 || w1->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (epi->reduce != PIKE_REDUCE_NONE || epi->scale != 1.0f) return PIKE_ERR_UNSUPPORTED;
+    nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
+    M = x->shape[0];
+    D = x->shape[1];
+    F = nk ? w1->shape[0] : w1->shape[1];
+    if ((nk ? w1->shape[1] : w1->shape[0]) != D) return PIKE_ERR_SHAPE;
+    if (M < 0 || D < 1 || F < 1) return PIKE_ERR_SHAPE;
+    if (D % 8 != 0 || F % 8 != 0 || D > 16384) return PIKE_ERR_UNSUPPORTED;
+    if (M > 0x7fffffff || F > 0x7fffffff) return PIKE_ERR_UNSUPPORTED;
+    return PIKE_OK;
+}
+
+pike_status_t pike_mlp_block_workspace(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w1,
+                                       const pike_epilogue_t *epi, size_t *bytes)
+{
+    if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
+    int64_t M, D, F;
+    bool nk;
+    if (pike_status_t st = mlp_shape(x, w1, epi, M, D, F, nk)) return st;
+    *bytes = align256((size_t)M * D * 2) + align256((size_t)M * F * 2);
+    return PIKE_OK;
+}
+
+pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *gamma,
+                             const pike_tensor_t *beta, const pike_tensor_t *w1, const pike_tensor_t *b1,
+                             const pike_tensor_t *w2, const pike_tensor_t *b2, const pike_epilogue_t *epi,
+                             pike_tensor_t *out, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (h == nullptr || out == nullptr || w2 == nullptr) return PIKE_ERR_NULL;
+    int64_t M, D, F;
+    bool nk;
+    if (pike_status_t st = mlp_shape(x, w1, epi, M, D, F, nk)) return st;
+    if (pike_status_t st = check_matrix(x, M, D)) return st;
+    if (pike_status_t st = check_matrix(w1, nk ? F : D, nk ? D : F)) return st;
+    if (pike_status_t st = check_matrix(w2, nk ? D : F, nk ? F : D)) return st;
+    if (pike_status_t st = check_matrix(out, M, D)) return st;
+    if (w2->dtype != PIKE_BF16 || out->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (pike_status_t st = check_vector(gamma, D)) return st;
+    if (pike_status_t st = check_vector(beta, D)) return st;
+    if (pike_status_t st = check_vector(b1, F)) return st;
+    if (pike_status_t st = check_vector(b2, D)) return st;
+    const pike_tensor_t *ins[7] = {x, gamma, beta, w1, b1, w2, b2};
+    for (const pike_tensor_t *t : ins)
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    const size_t z_bytes = align256((size_t)M * D * 2), h_bytes = align256((size_t)M * F * 2);
+    if (M > 0 && (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 ||
+                  workspace_bytes < z_bytes + h_bytes))
+        return PIKE_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (M == 0) return PIKE_OK;
+
+    void *z = workspace;
+    void *hbuf = static_cast<uint8_t *>(workspace) + z_bytes;
+    if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
+                                    gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
+                                    beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D, stream) != cudaSuccess)
+        return PIKE_ERR_CUDA;
+    // h = act(z @ w1 + b1), bf16
+    if (pike_status_t st = run_gemm(h, z, D, w1, nk, M, D, F, b1, nullptr, false, 0, hbuf, false, F, (int)epi->act,
+                                    1.0f, nullptr, stream))
+        return st;
+    // out = h @ w2 + b2 + x
+    return run_gemm(h, hbuf, F, w2, nk, M, F, D, b2, x->data, false, x->stride[0], out->data, false, out->stride[0],
+                    PIKE_ACT_NONE, 1.0f, nullptr, stream);
+}
+
+static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *epi)
+{
+    if (q == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = check_epilogue(epi)) return st;
+    if (q->ndim != 4) return PIKE_ERR_SHAPE;
+    if (q->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (q->shape[3] != 128) return PIKE_ERR_UNSUPPORTED;
+    if (q->shape[0] < 0 || q->shape[1] < 0 || q->shape[2] < 0) return PIKE_ERR_SHAPE;
+    if (q->shape[0] * q->shape[1] > 0x7fffff || q->shape[2] > 0x7fffff00) return PIKE_ERR_UNSUPPORTED;
+    if (!(epi->scale > 0.0f)) return PIKE_ERR_UNSUPPORTED;
+    if (epi->act != PIKE_ACT_NONE || epi->reduce != PIKE_REDUCE_NONE) return PIKE_ERR_UNSUPPORTED;
+    return PIKE_OK;
+}
+
+static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *like)
+{
+    if (t == nullptr || t->data == nullptr) return PIKE_ERR_NULL;
+    if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (t->ndim != 4) return PIKE_ERR_SHAPE;
+    for (int i = 0; i < 4; ++i)
+        if (t->shape[i] != like->shape[i]) return PIKE_ERR_SHAPE;
+    int64_t dense = 1;
+    for (int i = 3; i >= 0; --i) {
+        if (t->shape[i] > 1 && t->stride[i] != dense) return PIKE_ERR_STRIDE;
+        dense *= t->shape[i];
+    }
+    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    return PIKE_OK;
+}
+
+pike_status_t pike_attention_chain_workspace(pike_handle_t h, const pike_tensor_t *q, const pike_epilogue_t *epi,
+                                             size_t *bytes)
+{
+    if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = attn_shape(q, epi)) return st;
+    *bytes = 0;
+    return PIKE_OK;
+}
+
+pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, const pike_tensor_t *k,
+                                   const pike_tensor_t *v, const pike_epilogue_t *epi, pike_tensor_t *out,
+                                   void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    (void)workspace;
+    (void)workspace_bytes;
+    if (h == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = attn_shape(q, epi)) return st;
+    if (pike_status_t st = check_bhsd(q, q)) return st;
+    if (pike_status_t st = check_bhsd(k, q)) return st;
+    if (pike_status_t st = check_bhsd(v, q)) return st;
+    if (pike_status_t st = check_bhsd(out, q)) return st;
+    const pike_tensor_t *ins[3] = {q, k, v};
+    for (const pike_tensor_t *t : ins)
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    const int64_t BH = q->shape[0] * q->shape[1], S = q->shape[2];
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (BH == 0 || S == 0) return PIKE_OK;
+    CUtensorMap tmQ, tmK, tmV;
+    if (pike_status_t st = make_map_bsd(h, &tmQ, q->data, BH, S, 128)) return st;
+    if (pike_status_t st = make_map_bsd(h, &tmK, k->data, BH, S, 128)) return st;
+    if (pike_status_t st = make_map_bsd(h, &tmV, v->data, BH, S, 128)) return st;
+    pike::AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.BH = (int)BH; a.S = (int)S;
+    a.scale = epi->scale;
+    a.causal = (epi->flags & PIKE_FLAG_CAUSAL) != 0;
+    a.out = out->data;
+    a.status = h->status;
+    a.limit_ns = h->limit_ns;
+    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,301 @@
+// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores with the whole
+// pointwise epilogue applied in registers before one store.
+//
+//   out[m,n] = scale * act( sum_k A[m,k] * W[k,n] + bias[n] ) + residual[m,n]
+//
+// Persistent, warp-specialised CTAs (one per SM, 192 threads):
+//   warp 0      TMA producer: A tile 128x64 and W tile 256x64 (or 64x256 when W is
+//               [K,N]) into a 4-stage 128-byte-swizzled shared-memory ring
+//   warp 1      allocates 512 tensor-memory columns (two 128x256 fp32 accumulators)
+//               and issues tcgen05.mma (one thread), committing to mbarriers
+//   warps 2..5  epilogue: tcgen05.ld the finished accumulator (thread = row, 32
+//               columns at a time), bias/activation/scale/residual in registers,
+//               16-byte stores; optionally per-row (max, sum exp) partials for a
+//               softmax split across N tiles.  Runs under the next tile's K loop.
+// Every mbarrier wait is bounded (see mbar_wait).
+#include "../device/act.cuh"
+#include "../device/ptx.cuh"
+#include "kernels.h"
+
+namespace pike {
+namespace {
+
+constexpr int BM = GEMM_BM, BN = GEMM_BN, BK = GEMM_BK;
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;            // 16 KiB
+constexpr int B_BYTES = BN * BK * 2;            // 32 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 48 KiB
+constexpr int NUM_ACC = 2;
+constexpr int TMEM_COLS = NUM_ACC * BN;         // 512
+constexpr int THREADS = 192;
+constexpr int EPI_THREADS = 128;
+constexpr int GROUP_M = 8;                      // tile rasterisation: 8 row-blocks per column sweep
+
+struct __align__(8) Ctrl {
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
+    uint64_t tmem_full[NUM_ACC];
+    uint64_t tmem_empty[NUM_ACC];
+    uint32_t tmem_base;
+    uint32_t abort;
+    float bias[BN];
+};
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + sizeof(Ctrl);
+
+enum : uint32_t { BAR_EMPTY = 1, BAR_FULL = 2, BAR_TMEM_EMPTY = 3, BAR_TMEM_FULL = 4 };
+
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_blk, int &n_blk)
+{
+    const int per_group = GROUP_M * num_n;
+    const int g = t / per_group;
+    const int first_m = g * GROUP_M;
+    const int gsz = min(GROUP_M, num_m - first_m);
+    const int r = t - g * per_group;
+    m_blk = first_m + r % gsz;
+    n_blk = r / gsz;
+}
+
+template <int ACT>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(tiles + (size_t)STAGES * STAGE_BYTES);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_m = (p.M + BM - 1) / BM, num_n = (p.N + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], 1); }
+        for (int a = 0; a < NUM_ACC; ++a) { mbar_init(&ctrl->tmem_full[a], 1); mbar_init(&ctrl->tmem_empty[a], EPI_THREADS); }
+        ctrl->abort = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(&ctrl->tmem_base, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctrl->tmem_base;
+    const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+                int m_blk, n_blk;
+                tile_coords(t, num_m, num_n, m_blk, n_blk);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    mbar_wait(&ctrl->empty[s], ph ^ 1, ctx, BAR_EMPTY);
+                    uint8_t *a_s = tiles + (size_t)s * STAGE_BYTES;
+                    uint8_t *b_s = a_s + A_BYTES;
+                    mbar_arrive_expect_tx(&ctrl->full[s], STAGE_BYTES);
+                    tma_load_2d(a_s, &tmA, &ctrl->full[s], kb * BK, m_blk * BM);
+                    if (p.w_is_nk) {
+                        tma_load_2d(b_s, &tmB, &ctrl->full[s], kb * BK, n_blk * BN);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i)
+                            tma_load_2d(b_s + i * (64 * BK * 2), &tmB, &ctrl->full[s], n_blk * BN + i * 64, kb * BK);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc_bf16(BM, BN, false, !p.w_is_nk);
+            int s = 0;
+            uint32_t ph = 0;
+            int it = 0;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t aph = (it >> 1) & 1;
+                mbar_wait(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    mbar_wait(&ctrl->full[s], ph, ctx, BAR_FULL);
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * STAGE_BYTES);
+                    const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k) {
+                        const uint64_t adesc = make_smem_desc_sw128(a_addr + k * 32, 0, 1024);
+                        const uint64_t bdesc = p.w_is_nk ? make_smem_desc_sw128(b_addr + k * 32, 0, 1024)
+                                                         : make_smem_desc_sw128(b_addr + k * 2048, 64 * BK * 2, 1024);
+                        umma_ss(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&ctrl->empty[s]);
+                    if (++s == STAGES) { s = 0; ph ^= 1; }
+                }
+                umma_commit(&ctrl->tmem_full[acc]);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int et = threadIdx.x - 64;        // 0..127
+        int it = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            int m_blk, n_blk;
+            tile_coords(t, num_m, num_n, m_blk, n_blk);
+            const int acc = it & 1;
+            const uint32_t aph = (it >> 1) & 1;
+            const int n0 = n_blk * BN;
+            const int row = m_blk * BM + q * 32 + lane;
+            const bool row_ok = row < p.M;
+
+            // stage the tile's bias as fp32
+            named_bar_sync(1, EPI_THREADS);
+            for (int i = et; i < BN; i += EPI_THREADS) {
+                float b = 0.0f;
+                if (p.bias != nullptr && n0 + i < p.N)
+                    b = p.bias_f32 ? static_cast<const float *>(p.bias)[n0 + i]
+                                   : __bfloat162float(static_cast<const __nv_bfloat16 *>(p.bias)[n0 + i]);
+                ctrl->bias[i] = b;
+            }
+            named_bar_sync(1, EPI_THREADS);
+
+            mbar_wait(&ctrl->tmem_full[acc], aph, ctx, BAR_TMEM_FULL);
+            tc_fence_after();
+
+            float run_m = -INFINITY, run_l = 0.0f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int nc = n0 + c * 32;
+                if (nc >= p.N) break;
+                uint32_t r[32];
+                tmem_ld32(tmem_base + acc * BN + c * 32 + (static_cast<uint32_t>(q * 32) << 16), r);
+
+                // residual prefetch (thread = row, 32 consecutive columns)
+                uint4 res16[4];
+                float4 res32[8];
+                const bool has_res = p.residual != nullptr && row_ok;
+                if (has_res) {
+                    if (p.residual_f32) {
+                        const float *rp = static_cast<const float *>(p.residual) + (long long)row * p.ldr + nc;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            res32[g] = (nc + g * 4 < p.N) ? *reinterpret_cast<const float4 *>(rp + g * 4)
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+                    } else {
+                        const __nv_bfloat16 *rp =
+                            static_cast<const __nv_bfloat16 *>(p.residual) + (long long)row * p.ldr + nc;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            res16[g] = (nc + g * 8 < p.N) ? *reinterpret_cast<const uint4 *>(rp + g * 8)
+                                                          : make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                tmem_ld_wait();
+
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    v[j] = p.scale * act_fast<ACT>(__uint_as_float(r[j]) + ctrl->bias[c * 32 + j]);
+                if (has_res) {
+                    if (p.residual_f32) {
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            v[g * 4 + 0] += res32[g].x; v[g * 4 + 1] += res32[g].y;
+                            v[g * 4 + 2] += res32[g].z; v[g * 4 + 3] += res32[g].w;
+                        }
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const uint32_t w4[4] = {res16[g].x, res16[g].y, res16[g].z, res16[g].w};
+#pragma unroll
+                            for (int h = 0; h < 4; ++h) {
+                                v[g * 8 + 2 * h] += bf16_lo(w4[h]);
+                                v[g * 8 + 2 * h + 1] += bf16_hi(w4[h]);
+                            }
+                        }
+                    }
+                }
+
+                if (p.softmax_partials) {
+                    float cm = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nc + j < p.N) cm = fmaxf(cm, v[j]);
+                    const float nm = fmaxf(run_m, cm);
+                    float s = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nc + j < p.N) s += __expf(v[j] - nm);
+                    run_l = run_l * __expf(run_m - nm) + s;
+                    run_m = nm;
+                }
+
+                if (row_ok) {
+                    if (p.out_f32) {
+                        float *op = static_cast<float *>(p.out) + (long long)row * p.ldo + nc;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (nc + g * 4 < p.N)
+                                *reinterpret_cast<float4 *>(op + g * 4) =
+                                    make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+                    } else {
+                        __nv_bfloat16 *op = static_cast<__nv_bfloat16 *>(p.out) + (long long)row * p.ldo + nc;
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            if (nc + g * 8 < p.N)
+                                *reinterpret_cast<uint4 *>(op + g * 8) =
+                                    make_uint4(pack_bf16x2(v[g * 8 + 0], v[g * 8 + 1]), pack_bf16x2(v[g * 8 + 2], v[g * 8 + 3]),
+                                               pack_bf16x2(v[g * 8 + 4], v[g * 8 + 5]), pack_bf16x2(v[g * 8 + 6], v[g * 8 + 7]));
+                    }
+                }
+            }
+            // accumulator drained: hand the TMEM stage back to the MMA warp
+            tc_fence_before();
+            mbar_arrive(&ctrl->tmem_empty[acc]);
+
+            if (p.softmax_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (ctrl->abort) abort_drain();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
+                             cudaStream_t stream)
+{
+    const int num_m = (a.M + BM - 1) / BM, num_n = (a.N + BN - 1) / BN;
+    const int num_tiles = num_m * num_n;
+    if (num_tiles <= 0) return cudaSuccess;
+    const dim3 grid(num_tiles < num_sms ? num_tiles : num_sms), block(THREADS);
+    auto go = [&](auto kern) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, a);
+        return cudaGetLastError();
+    };
+    switch (a.act) {
+    case ACT_GELU_ERF:  return go(gemm_bf16_kernel<ACT_GELU_ERF>);
+    case ACT_GELU_TANH: return go(gemm_bf16_kernel<ACT_GELU_TANH>);
+    case ACT_SILU:      return go(gemm_bf16_kernel<ACT_SILU>);
+    default:            return go(gemm_bf16_kernel<ACT_NONE>);
+    }
+}
+
+}  // namespace pike

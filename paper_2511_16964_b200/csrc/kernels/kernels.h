@@ -1,0 +1,65 @@
+// Host-side launchers of the chain kernels (internal to the library).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pike {
+
+enum : uint32_t {
+    KID_GEMM = 1,
+    KID_ATTN = 2,
+};
+
+// ---- fp32 CUDA-core chain: out = reduce(scale*act(x@w+b)+res) ------------------
+struct Fp32ChainArgs {
+    const float *x, *w, *bias, *residual, *gamma, *beta;
+    float *out;
+    int M, K, N;
+    long long ldx, ldw, ldr, ldo;
+    int w_is_nk;
+    int act, reduce;
+    float scale, eps;
+};
+cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, cudaStream_t stream);
+
+// ---- bf16 tcgen05 GEMM + epilogue ------------------------------------------------
+struct GemmArgs {
+    int M, N, K;
+    int w_is_nk;
+    const void *bias;      int bias_f32;
+    const void *residual;  int residual_f32;  long long ldr;
+    void *out;             int out_f32;       long long ldo;
+    int act;
+    float scale;
+    int softmax_partials;  // 1: also write per-(row, n-tile) (max, sum exp) pairs
+    float2 *partials;
+    unsigned int *status;
+    unsigned long long limit_ns;
+};
+constexpr int GEMM_BM = 128, GEMM_BN = 256, GEMM_BK = 64;
+cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
+                             cudaStream_t stream);
+
+// ---- row kernels -------------------------------------------------------------------
+// z = LayerNorm(x) rows, bf16 in/out, fp32 statistics; gamma/beta bf16 or f32 or null.
+cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
+                                  int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D,
+                                  cudaStream_t stream);
+// p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
+cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
+                                  cudaStream_t stream);
+
+// ---- attention ---------------------------------------------------------------------
+struct AttnArgs {
+    int BH, S;
+    float scale;
+    int causal;
+    void *out;  // bf16 [BH, S, 128]
+    unsigned int *status;
+    unsigned long long limit_ns;
+};
+cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
+                                  const AttnArgs &a, cudaStream_t stream);
+
+}  // namespace pike

@@ -1,0 +1,77 @@
+"""GPU parity: GEMM -> online softmax -> GEMM attention chain (scores never leave the chip)."""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+import pike_inputs as G
+from oracle import pike_oracle as O
+from util import check_bf16, dev, host64
+
+pytestmark = pytest.mark.gpu
+BF16 = torch.bfloat16
+
+
+def _run(c, causal):
+    import paper_2511_16964_b200 as P
+    out = P.pike_attention_chain(dev(c["q"], BF16), dev(c["k"], BF16), dev(c["v"], BF16), scale=c["scale"],
+                                 causal=causal)
+    torch.cuda.synchronize()
+    st, where = P.pike_get_last_device_status()
+    assert st == 0, f"device status {st} at {where:#x}"
+    return host64(out)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("B,H,S", [(1, 1, 128), (1, 2, 256), (2, 3, 300), (1, 1, 1), (1, 2, 129), (1, 1, 640)])
+def test_small_and_ragged_sequences(B, H, S, causal):
+    c = G.config5(B=B, H=H, S=S, seed=9)
+    got = _run(c, causal)
+    want = O.attention(c["q"], c["k"], c["v"], scale=c["scale"], causal=causal)
+    check_bf16(got, want, what=f"attention B{B} H{H} S{S} causal={causal}")
+
+
+def test_structural_properties_on_the_gpu_output():
+    c = G.config5(B=1, H=2, S=384, seed=10)
+    got = _run(c, True)
+    # causal row 0 attends to key 0 only -> O[0] = V[0] exactly (bf16 values pass through)
+    assert np.array_equal(got[:, :, 0, :], c["v"][:, :, 0, :].astype(np.float64))
+    # V == 1 -> O == 1
+    c1 = dict(c, v=np.ones_like(c["v"]))
+    assert np.abs(_run(c1, True) - 1).max() <= 2 ** -7
+    # run-to-run bit reproducibility
+    assert np.array_equal(got, _run(c, True))
+
+
+@functools.lru_cache(maxsize=1)
+def _config5_full():
+    return G.config5()
+
+
+def test_config5_full_size_sampled_rows():
+    c = _config5_full()
+    got = _run(c, True)
+    rng = np.random.default_rng(11)
+    worst = 0.0
+    for b, h in [(0, 0), (3, 17), (7, 31), (5, 8)]:
+        rows = np.unique(np.concatenate([[0, 127, 128, 2047], rng.integers(0, 2048, 12)]))
+        want = O.attention_head(c["q"][b, h], c["k"][b, h], c["v"][b, h], scale=c["scale"], causal=True, rows=rows)
+        worst = max(worst, check_bf16(got[b, h][rows], want, what=f"config 5 head ({b},{h})"))
+    assert worst < 2e-2
+
+
+def test_rejections():
+    import paper_2511_16964_b200 as P
+    q = torch.zeros((1, 1, 16, 64), device="cuda", dtype=BF16)
+    with pytest.raises(P.PikeError) as e:                 # head dimension other than 128
+        P.pike_attention_chain(q, q.clone(), q.clone(), scale=1.0)
+    assert e.value.code == 6
+    q = torch.zeros((1, 1, 16, 128), device="cuda", dtype=BF16)
+    with pytest.raises(P.PikeError) as e:                 # k has another sequence length
+        P.pike_attention_chain(q, torch.zeros((1, 1, 32, 128), device="cuda", dtype=BF16), q.clone(), scale=1.0)
+    assert e.value.code == 2
+    with pytest.raises(P.PikeError) as e:                 # non-positive scale
+        P.pike_attention_chain(q, q.clone(), q.clone(), scale=0.0)
+    assert e.value.code == 6
+    assert P.pike_attention_chain_workspace(q, scale=1.0) == 0

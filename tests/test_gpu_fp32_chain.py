@@ -1,0 +1,73 @@
+"""GPU parity: fp32 Linear + bias + activation + scale + residual + reduction (CUDA-core path).
+Bar: max |gpu - oracle| <= 1e-4 (fp32 configs)."""
+import numpy as np
+import pytest
+import torch
+
+import pike_inputs as G
+from oracle import pike_oracle as O
+from util import check_f32, dev, host64
+
+pytestmark = pytest.mark.gpu
+F32 = torch.float32
+
+
+def _run(c, *, act, reduce, scale=1.0, residual=None, w_is_nk=False, gamma=None, beta=None, eps=1e-5):
+    import paper_2511_16964_b200 as P
+    w = c["w"].T.copy() if w_is_nk else c["w"]
+    out = P.pike_linear_epilogue(dev(c["x"], F32), dev(w, F32), dev(c.get("b"), F32), dev(residual, F32),
+                                 dev(gamma, F32), dev(beta, F32), act=act, scale=scale, reduce=reduce, eps=eps,
+                                 w_is_nk=w_is_nk)
+    torch.cuda.synchronize()
+    want = O.linear_epilogue(c["x"], c["w"], c.get("b"), residual, gamma, beta, act=act, scale=scale,
+                             reduce=reduce, eps=eps)
+    return host64(out), want
+
+
+def test_config1_full():
+    c = G.config1()
+    got, want = _run(c, act="gelu_erf", reduce="layernorm", gamma=c["gamma"], beta=c["beta"], eps=c["eps"])
+    check_f32(got, want, 1e-4, "config 1")
+    # LayerNorm invariants on the GPU output itself
+    assert np.abs(got.mean(axis=1)).max() < 1e-5
+
+
+@pytest.mark.parametrize("act", ["none", "gelu_erf", "gelu_tanh", "silu"])
+@pytest.mark.parametrize("reduce", ["none", "layernorm", "softmax"])
+def test_ragged_shapes_every_act_and_reduce(act, reduce):
+    c = G.config1(M=37, K=100, N=200, seed=3)
+    rng = np.random.default_rng(5)
+    res = rng.standard_normal((37, 200)).astype(np.float32)
+    gamma = rng.uniform(0.5, 1.5, 200).astype(np.float32)
+    beta = rng.uniform(-0.1, 0.1, 200).astype(np.float32)
+    got, want = _run(c, act=act, reduce=reduce, scale=0.5, residual=res, gamma=gamma, beta=beta)
+    check_f32(got, want, 1e-4, f"{act}/{reduce}")
+
+
+@pytest.mark.parametrize("M,K,N", [(1, 8, 8), (5, 1, 1024), (700, 300, 72), (3, 2500, 40)])
+def test_edge_shapes_and_weight_layout(M, K, N):
+    c = G.config1(M=M, K=K, N=N, seed=1)
+    for nk in (False, True):
+        got, want = _run(c, act="gelu_erf", reduce="layernorm", w_is_nk=nk)
+        check_f32(got, want, 1e-4, f"{M}x{K}x{N} nk={nk}")
+
+
+def test_empty_batch_and_rejections():
+    import paper_2511_16964_b200 as P
+    x = torch.zeros((0, 16), device="cuda")
+    w = torch.zeros((16, 8), device="cuda")
+    assert P.pike_linear_epilogue(x, w).shape == (0, 8)
+    with pytest.raises(P.PikeError) as e:            # N > 1024 on the fp32 path
+        P.pike_linear_epilogue(torch.zeros((4, 16), device="cuda"), torch.zeros((16, 1032), device="cuda"))
+    assert e.value.code == 6
+    with pytest.raises(P.PikeError) as e:            # K mismatch
+        P.pike_linear_epilogue(torch.zeros((4, 16), device="cuda"), torch.zeros((24, 8), device="cuda"))
+    assert e.value.code == 2
+    with pytest.raises(P.PikeError) as e:            # out aliases x
+        xx = torch.zeros((8, 8), device="cuda")
+        P.pike_linear_epilogue(xx, torch.zeros((8, 8), device="cuda"), out=xx)
+    assert e.value.code == 6
+    with pytest.raises(P.PikeError) as e:            # misaligned base pointer
+        buf = torch.zeros(4 * 16 + 1, device="cuda")
+        P.pike_linear_epilogue(buf[1:].view(4, 16), w)
+    assert e.value.code == 4
