@@ -103,6 +103,26 @@ pike_status_t pike_get_last_device_status(pike_handle_t handle, pike_status_t *s
 pike_status_t pike_set_wait_limit_ns(pike_handle_t handle, uint64_t ns);
 
 /*
+ * Per-kernel device timing, following the paper's timing protocol (Section 4.6:
+ * timed runs bracketed on the device, synchronisation inside the timed region).
+ * Between pike_profile_begin and pike_profile_end every kernel the handle launches
+ * is bracketed by two CUDA events on the caller's stream.  pike_profile_end
+ * synchronises the device and fills out[PIKE_KERNEL_COUNT] (caller-owned host
+ * memory) with the launch count and the summed device time of each kernel.
+ */
+typedef enum {
+    PIKE_KERNEL_FP32_CHAIN = 0,     /* fp32 linear + epilogue + row reduction          */
+    PIKE_KERNEL_GEMM_BF16 = 1,      /* tcgen05 GEMM + register epilogue                */
+    PIKE_KERNEL_LAYERNORM_BF16 = 2, /* MLP block prologue                              */
+    PIKE_KERNEL_SOFTMAX_FINISH = 3, /* combine split-row partials, normalise in place  */
+    PIKE_KERNEL_ATTENTION_BF16 = 4, /* GEMM -> online softmax -> GEMM                  */
+    PIKE_KERNEL_COUNT = 5
+} pike_kernel_t;
+typedef struct { uint64_t launches; double device_ms; } pike_kernel_profile_t;
+pike_status_t pike_profile_begin(pike_handle_t handle);
+pike_status_t pike_profile_end(pike_handle_t handle, pike_kernel_profile_t *out);
+
+/*
  * Linear + epilogue chain (the "operator fusion" pattern of Section 5.3):
  *
  *   v[m,n]   = scale * act( sum_k x[m,k] * w[k,n] + bias[n] ) + residual[m,n]

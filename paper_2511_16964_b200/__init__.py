@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     pike_linear_epilogue_workspace,
     pike_mlp_block,
     pike_mlp_block_workspace,
+    pike_profile_begin,
+    pike_profile_end,
     pike_set_wait_limit_ns,
     pike_status_string,
 )

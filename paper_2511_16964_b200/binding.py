@@ -23,7 +23,7 @@ FLAG_W_IS_NK, FLAG_CAUSAL = 0x1, 0x2
 
 EXPORTS = (
     "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
-    "pike_set_wait_limit_ns", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
+    "pike_set_wait_limit_ns", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
     "pike_attention_chain",
 )
@@ -45,6 +45,12 @@ class pike_epilogue_t(ctypes.Structure):
                 ("reduce", ctypes.c_int), ("eps", ctypes.c_float), ("out_dtype", ctypes.c_int),
                 ("flags", ctypes.c_uint32)]
 
+
+class pike_kernel_profile_t(ctypes.Structure):
+    _fields_ = [("launches", ctypes.c_uint64), ("device_ms", ctypes.c_double)]
+
+
+KERNELS = ("fp32_chain", "gemm_bf16", "layernorm_bf16", "softmax_finish", "attention_bf16")
 
 _lib = None
 _lock = threading.Lock()
@@ -73,6 +79,8 @@ def load_library() -> ctypes.CDLL:
             lib.pike_status_string.restype = ctypes.c_char_p
             lib.pike_get_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_uint32)]
             lib.pike_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
+            lib.pike_profile_begin.argtypes = [vp]
+            lib.pike_profile_end.argtypes = [vp, ctypes.POINTER(pike_kernel_profile_t)]
             lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
             lib.pike_linear_epilogue.argtypes = [vp, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_mlp_block_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
@@ -169,6 +177,19 @@ def pike_get_last_device_status(device=None) -> tuple[int, int]:
     _check(load_library().pike_get_last_device_status(_handle(dev), ctypes.byref(st), ctypes.byref(where)),
            "pike_get_last_device_status")
     return st.value, where.value
+
+
+def pike_profile_begin(device=None) -> None:
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    _check(load_library().pike_profile_begin(_handle(dev)), "pike_profile_begin")
+
+
+def pike_profile_end(device=None) -> dict:
+    """{kernel name: (launches, summed device ms)} since pike_profile_begin; synchronises."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    out = (pike_kernel_profile_t * len(KERNELS))()
+    _check(load_library().pike_profile_end(_handle(dev), out), "pike_profile_end")
+    return {name: (int(out[i].launches), float(out[i].device_ms)) for i, name in enumerate(KERNELS)}
 
 
 def pike_linear_epilogue_workspace(x, w, *, act="none", scale=1.0, reduce="none", eps=1e-5,

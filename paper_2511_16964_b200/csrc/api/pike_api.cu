@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "../../../include/pike.h"
 #include "../kernels/kernels.h"
@@ -17,11 +18,43 @@ struct pike_handle_s {
     unsigned int *status;  // device, 4 words
     unsigned long long limit_ns;
     PFN_cuTensorMapEncodeTiled_v12000 encode;
+    // per-kernel device timing (pike_profile_begin / pike_profile_end)
+    bool profiling;
+    std::vector<cudaEvent_t> ev_pool;                       // recycled events
+    std::vector<cudaEvent_t> ev_start[PIKE_KERNEL_COUNT];
+    std::vector<cudaEvent_t> ev_stop[PIKE_KERNEL_COUNT];
 };
 
 namespace {
 
 constexpr unsigned long long DEFAULT_LIMIT_NS = 2000000000ull;
+
+// Brackets one kernel launch with CUDA events on the caller's stream while profiling is on.
+struct TimedLaunch {
+    pike_handle_t h;
+    pike_kernel_t kid;
+    cudaStream_t stream;
+    static cudaEvent_t get(pike_handle_t h)
+    {
+        cudaEvent_t e = nullptr;
+        if (!h->ev_pool.empty()) { e = h->ev_pool.back(); h->ev_pool.pop_back(); }
+        else if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); e = nullptr; }
+        return e;
+    }
+    TimedLaunch(pike_handle_t h_, pike_kernel_t kid_, cudaStream_t s) : h(h_), kid(kid_), stream(s)
+    {
+        if (!h->profiling) return;
+        cudaEvent_t e = get(h);
+        if (e != nullptr) { cudaEventRecord(e, stream); h->ev_start[kid].push_back(e); }
+    }
+    ~TimedLaunch()
+    {
+        if (!h->profiling || h->ev_start[kid].size() == h->ev_stop[kid].size()) return;
+        cudaEvent_t e = get(h);
+        if (e != nullptr) { cudaEventRecord(e, stream); h->ev_stop[kid].push_back(e); }
+        else { h->ev_pool.push_back(h->ev_start[kid].back()); h->ev_start[kid].pop_back(); }
+    }
+};
 
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 size_t elem_size(pike_dtype_t t) { return t == PIKE_F32 ? 4 : 2; }
@@ -29,14 +62,16 @@ size_t elem_size(pike_dtype_t t) { return t == PIKE_F32 ? 4 : 2; }
 bool valid_dtype(pike_dtype_t t) { return t == PIKE_F32 || t == PIKE_BF16; }
 
 // a dense-enough 2-D view: innermost stride 1, row pitch >= columns, 16-byte aligned base and pitch
-pike_status_t check_matrix(const pike_tensor_t *t, int64_t rows, int64_t cols)
+pike_status_t check_matrix(const pike_tensor_t *t, int64_t rows, int64_t cols, bool pitch16 = true)
 {
-    if (t == nullptr || t->data == nullptr) return PIKE_ERR_NULL;
+    if (t == nullptr) return PIKE_ERR_NULL;
     if (!valid_dtype(t->dtype)) return PIKE_ERR_DTYPE;
     if (t->ndim != 2 || t->shape[0] != rows || t->shape[1] != cols) return PIKE_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return PIKE_OK;  // an empty tensor may have no storage
+    if (t->data == nullptr) return PIKE_ERR_NULL;
     if (t->stride[1] != 1 || t->stride[0] < cols) return PIKE_ERR_STRIDE;
     if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
-    if ((t->stride[0] * (int64_t)elem_size(t->dtype)) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    if (pitch16 && (t->stride[0] * (int64_t)elem_size(t->dtype)) % 16 != 0) return PIKE_ERR_ALIGNMENT;
     return PIKE_OK;
 }
 
@@ -173,6 +208,7 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.partials = partials;
     g.status = h->status;
     g.limit_ns = h->limit_ns;
+    TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
     return pike::launch_gemm_bf16(tmA, tmB, g, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
@@ -211,6 +247,7 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     h->device = device;
     h->num_sms = prop.multiProcessorCount;
     h->limit_ns = DEFAULT_LIMIT_NS;
+    h->profiling = false;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -232,8 +269,48 @@ pike_status_t pike_destroy(pike_handle_t h)
 {
     if (h == nullptr) return PIKE_ERR_NULL;
     cudaFree(h->status);
+    for (int k = 0; k < PIKE_KERNEL_COUNT; ++k) {
+        for (cudaEvent_t e : h->ev_start[k]) cudaEventDestroy(e);
+        for (cudaEvent_t e : h->ev_stop[k]) cudaEventDestroy(e);
+    }
+    for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
     delete h;
     return PIKE_OK;
+}
+
+pike_status_t pike_profile_begin(pike_handle_t h)
+{
+    if (h == nullptr) return PIKE_ERR_NULL;
+    for (int k = 0; k < PIKE_KERNEL_COUNT; ++k) {
+        for (cudaEvent_t e : h->ev_start[k]) h->ev_pool.push_back(e);
+        for (cudaEvent_t e : h->ev_stop[k]) h->ev_pool.push_back(e);
+        h->ev_start[k].clear();
+        h->ev_stop[k].clear();
+    }
+    h->profiling = true;
+    return PIKE_OK;
+}
+
+pike_status_t pike_profile_end(pike_handle_t h, pike_kernel_profile_t *out)
+{
+    if (h == nullptr || out == nullptr) return PIKE_ERR_NULL;
+    h->profiling = false;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PIKE_ERR_CUDA;
+    pike_status_t rc = PIKE_OK;
+    for (int k = 0; k < PIKE_KERNEL_COUNT; ++k) {
+        out[k].launches = h->ev_stop[k].size();
+        out[k].device_ms = 0.0;
+        for (size_t i = 0; i < h->ev_stop[k].size(); ++i) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, h->ev_start[k][i], h->ev_stop[k][i]) != cudaSuccess) rc = PIKE_ERR_CUDA;
+            out[k].device_ms += ms;
+        }
+        for (cudaEvent_t e : h->ev_start[k]) h->ev_pool.push_back(e);
+        for (cudaEvent_t e : h->ev_stop[k]) h->ev_pool.push_back(e);
+        h->ev_start[k].clear();
+        h->ev_stop[k].clear();
+    }
+    return rc;
 }
 
 pike_status_t pike_get_last_device_status(pike_handle_t h, pike_status_t *status, uint32_t *where)
@@ -273,15 +350,16 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
     if (h == nullptr || out == nullptr) return PIKE_ERR_NULL;
     LinearShape s;
     if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
-    if (pike_status_t st = check_matrix(x, s.M, s.K)) return st;
-    if (pike_status_t st = check_matrix(w, s.w_is_nk ? s.N : s.K, s.w_is_nk ? s.K : s.N)) return st;
-    if (pike_status_t st = check_matrix(out, s.M, s.N)) return st;
+    const bool p16 = !s.fp32_path;  // the fp32 kernel uses scalar accesses: any row pitch is fine
+    if (pike_status_t st = check_matrix(x, s.M, s.K, p16)) return st;
+    if (pike_status_t st = check_matrix(w, s.w_is_nk ? s.N : s.K, s.w_is_nk ? s.K : s.N, p16)) return st;
+    if (pike_status_t st = check_matrix(out, s.M, s.N, p16)) return st;
     if (out->dtype != epi->out_dtype) return PIKE_ERR_DTYPE;
     if (pike_status_t st = check_vector(bias, s.N)) return st;
     if (pike_status_t st = check_vector(gamma, s.N)) return st;
     if (pike_status_t st = check_vector(beta, s.N)) return st;
     if (residual != nullptr)
-        if (pike_status_t st = check_matrix(residual, s.M, s.N)) return st;
+        if (pike_status_t st = check_matrix(residual, s.M, s.N, p16)) return st;
     const pike_tensor_t *ins[6] = {x, w, bias, residual, gamma, beta};
     for (const pike_tensor_t *t : ins)
         if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
@@ -306,6 +384,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         a.w_is_nk = s.w_is_nk;
         a.act = (int)epi->act; a.reduce = (int)epi->reduce;
         a.scale = epi->scale; a.eps = epi->eps;
+        TimedLaunch timed(h, PIKE_KERNEL_FP32_CHAIN, stream);
         return pike::launch_fp32_chain(a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
 
@@ -323,6 +402,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         return st;
     if (partials != nullptr) {
         const int num_n = (int)((s.N + pike::GEMM_BN - 1) / pike::GEMM_BN);
+        TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
         if (pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)s.M,
                                         (int)s.N, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
@@ -391,10 +471,14 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
 
     void *z = workspace;
     void *hbuf = static_cast<uint8_t *>(workspace) + z_bytes;
-    if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
-                                    gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
-                                    beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D, stream) != cudaSuccess)
-        return PIKE_ERR_CUDA;
+    {
+        TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
+        if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
+                                        gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
+                                        beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D,
+                                        stream) != cudaSuccess)
+            return PIKE_ERR_CUDA;
+    }
     // h = act(z @ w1 + b1), bf16
     if (pike_status_t st = run_gemm(h, z, D, w1, nk, M, D, F, b1, nullptr, false, 0, hbuf, false, F, (int)epi->act,
                                     1.0f, nullptr, stream))
@@ -420,11 +504,13 @@ static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *e
 
 static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *like)
 {
-    if (t == nullptr || t->data == nullptr) return PIKE_ERR_NULL;
+    if (t == nullptr) return PIKE_ERR_NULL;
     if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
     if (t->ndim != 4) return PIKE_ERR_SHAPE;
     for (int i = 0; i < 4; ++i)
         if (t->shape[i] != like->shape[i]) return PIKE_ERR_SHAPE;
+    if (t->shape[0] * t->shape[1] * t->shape[2] == 0) return PIKE_OK;  // empty: no storage needed
+    if (t->data == nullptr) return PIKE_ERR_NULL;
     int64_t dense = 1;
     for (int i = 3; i >= 0; --i) {
         if (t->shape[i] > 1 && t->stride[i] != dense) return PIKE_ERR_STRIDE;
@@ -474,6 +560,7 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     a.out = out->data;
     a.status = h->status;
     a.limit_ns = h->limit_ns;
+    TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
     return pike::launch_attention_bf16(tmQ, tmK, tmV, a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
