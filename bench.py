@@ -146,6 +146,22 @@ def oracle_sample_text():
 ALL = ("C1", "C2", "C3", "C4", "C5")
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """The slowest rank's time: the whole job is only done when the last rank is."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tflops(step_flops: float, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank processes one full suite per step (weak scaling)."""
+    return world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+
 def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5}
@@ -295,13 +311,10 @@ def run_ours(args):
     total_ms = t_start.elapsed_time(t_stop)
     prof = P.pike_profile_end()
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, device)
     ms_per_step = total_ms / args.steps
     step_flops = sum(f.values())
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = job_tflops(step_flops, world, ms_per_step)
     per_cfg_ms = {n: float(np.mean([a.elapsed_time(b) for a, b in events[n]])) for n in names}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ---
@@ -325,11 +338,8 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * step_flops / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
+    e2e_value = job_tflops(step_flops, world, e2e_ms)
 
     if rank != 0:
         if world > 1:
