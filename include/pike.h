@@ -155,6 +155,37 @@ pike_status_t pike_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x,
                                    size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Logits + row softmax for callers that cannot allocate device memory.  (The paper has
+ * no counterpart to this entry point; it exists for how the library gets embedded.)
+ *
+ *   out[m,:] = softmax_n( scale * act( sum_k x[m,k] * w[k,n] + bias[n] ) )
+ *
+ * Same arithmetic, kernels and bf16 envelope as pike_linear_epilogue with
+ * reduce == PIKE_REDUCE_SOFTMAX (x, w PIKE_BF16, bias BF16/F32 or NULL, out PIKE_F32,
+ * K and N multiples of 8, M >= 1; epi->reduce must be PIKE_REDUCE_SOFTMAX and
+ * epi->out_dtype PIKE_F32), but it takes no workspace: some hosts of this library
+ * cannot produce one -- a server that gave the whole device heap to its own pool, a
+ * plugin running inside another framework's step, a latency-critical thread that may
+ * not enter cudaMalloc (it locks and can synchronise the device).  The per-(row,
+ * 256-column tile) partial (max, sum) pairs go to an array built into the library
+ * image instead.  The call itself performs no cudaMalloc/cudaFree and calls no
+ * allocating routine.  What follows from the built-in array:
+ *  - Capacity: M * ceil(N/256) <= PIKE_NOALLOC_MAX_PARTIALS (2 MiB of pairs, resident
+ *    on every GPU that loads the library until the process exits).  A larger problem
+ *    returns PIKE_ERR_WORKSPACE and enqueues nothing.
+ *  - The first call on a device looks up the array's device address
+ *    (cudaGetSymbolAddress); make that first call outside any stream capture.
+ *  - All calls on a device share the array.  Calls that can overlap on the GPU (issued
+ *    to different streams without an ordering between them) race on it and produce
+ *    wrong results; calls on one stream are safe.  The array keeps the previous call's
+ *    values, which is harmless: each call writes every pair before reading it.
+ */
+#define PIKE_NOALLOC_MAX_PARTIALS 262144
+pike_status_t pike_linear_softmax_noalloc(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
+                                          const pike_tensor_t *bias, const pike_epilogue_t *epi, pike_tensor_t *out,
+                                          void *cuda_stream);
+
+/*
  * Pre-LayerNorm transformer MLP block (sub-graph fusion, Section 5.3):
  *
  *   z   = LayerNorm(x; gamma, beta, eps)            over the last dimension D

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     pike_get_last_device_status,
     pike_linear_epilogue,
     pike_linear_epilogue_workspace,
+    pike_linear_softmax_noalloc,
     pike_mlp_block,
     pike_mlp_block_workspace,
     pike_profile_begin,

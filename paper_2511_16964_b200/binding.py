@@ -25,7 +25,7 @@ EXPORTS = (
     "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
     "pike_set_wait_limit_ns", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
-    "pike_attention_chain",
+    "pike_attention_chain", "pike_linear_softmax_noalloc",
 )
 
 
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
             lib.pike_profile_end.argtypes = [vp, ctypes.POINTER(pike_kernel_profile_t)]
             lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
             lib.pike_linear_epilogue.argtypes = [vp, T, T, T, T, T, T, E, T, vp, sz, vp]
+            lib.pike_linear_softmax_noalloc.argtypes = [vp, T, T, T, E, T, vp]
             lib.pike_mlp_block_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
             lib.pike_mlp_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_attention_chain_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
@@ -219,6 +220,23 @@ def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, 
                                                _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
                                                _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
            "pike_linear_epilogue")
+    return out
+
+
+NOALLOC_MAX_PARTIALS = 262144
+
+
+def pike_linear_softmax_noalloc(x, w, bias=None, *, out, act="none", scale=1.0, w_is_nk=False, stream=None):
+    """out = softmax(scale*act(x @ w + bias)) with the scratch inside the library.
+
+    For callers that cannot hand the library a workspace because they cannot allocate
+    device memory.  `out` (fp32, [M,N]) must be supplied: this wrapper allocates nothing
+    either.  M*ceil(N/256) is limited to NOALLOC_MAX_PARTIALS; calls on different
+    streams must not overlap (they share one scratch array).  See include/pike.h."""
+    e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
+    _check(load_library().pike_linear_softmax_noalloc(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
+                                                      ctypes.byref(e), _tensor(out), _stream(stream)),
+           "pike_linear_softmax_noalloc")
     return out
 
 

@@ -13,6 +13,7 @@ LIB = os.path.join(HERE, "libpike.so")
 
 SOURCES = [
     "api/pike_api.cu",
+    "api/pike_noalloc.cu",
     "kernels/fp32_chain.cu",
     "kernels/gemm_bf16.cu",
     "kernels/row_kernels.cu",

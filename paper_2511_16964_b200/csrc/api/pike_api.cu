@@ -12,18 +12,7 @@
 #include "../../../include/pike.h"
 #include "../kernels/kernels.h"
 
-struct pike_handle_s {
-    int device;
-    int num_sms;
-    unsigned int *status;  // device, 4 words
-    unsigned long long limit_ns;
-    PFN_cuTensorMapEncodeTiled_v12000 encode;
-    // per-kernel device timing (pike_profile_begin / pike_profile_end)
-    bool profiling;
-    std::vector<cudaEvent_t> ev_pool;                       // recycled events
-    std::vector<cudaEvent_t> ev_start[PIKE_KERNEL_COUNT];
-    std::vector<cudaEvent_t> ev_stop[PIKE_KERNEL_COUNT];
-};
+#include "handle.h"
 
 namespace {
 
