@@ -431,7 +431,7 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         "C4": lambda: torch.softmax(d["c4x"] @ d["c4w"], dim=-1, dtype=torch.float32),
         "C5": attn,
     }
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=d["c1x"].device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=next(iter(d.values())).device)
     res = {}
     for n in names:
         ops[n]()

@@ -1,19 +1,24 @@
 // GEMM -> online softmax -> GEMM attention chain on tcgen05 / tensor memory.
-// The score tile lives in tensor memory and registers only; nothing but Q, K, V
-// and O touches HBM.
+// Scores and probabilities live in tensor memory and registers only; nothing but
+// Q, K, V and O touches HBM.
 //
-// One CTA per (batch*head, 128-query tile), 192 threads:
-//   warp 0      TMA producer: Q once, then K_j / V_j tiles (128 keys x 128 d) into
-//               two-stage 128-byte-swizzled rings
-//   warp 1      MMA issuer: S_j = Q K_j^T (K-major operands) into TMEM columns
-//               [0,128); PV_j = P_j V_j (V is the MN-major B operand) into [128,256)
-//   warps 2..5  softmax: thread = query row.  Pass 1 reads S_j for the row maximum,
-//               pass 2 recomputes p = 2^(s*c - m), rounds to bf16 and writes P_j to
-//               shared memory in the K-major swizzled operand layout.  The running
-//               output O lives in registers: O = O*alpha + PV_j is folded in one tile
-//               late, so PV_j overlaps the next tile's S MMA and softmax.
-// Causal masking is computed from indices on the diagonal tile only; tiles above the
-// diagonal are never loaded.  CTAs are ordered longest-first.
+// One CTA per (batch*head, PAIR of 128-query tiles), 384 threads = 3 warpgroups:
+//   WG0  warp 0: TMA producer (both Q tiles once, then K_j / V_j tiles of 128 keys into
+//        two-stage 128-byte-swizzled rings); warp 1: MMA issuer (one thread)
+//   WG1  softmax for query tile 0        WG2  softmax for query tile 1   (thread = row)
+// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.
+//   S_t(j) = Q_t K_j^T      both operands K-major from shared memory
+//   P_t(j) = bf16 probabilities, written by the softmax threads over the first 64
+//            columns of S_t (two per 32-bit column) and read by the second MMA as its
+//            A operand straight from tensor memory
+//   O_t   += P_t(j) V_j     V is the MN-major B operand; accumulates in tensor memory
+// The MMA warp interleaves the two tiles (PV0, S0', PV1, S1', ...) so one tile's softmax
+// runs under the other tile's MMAs.  The running maximum is only raised when it grows by
+// more than 2^8 (probabilities stay bounded by 256 in between), so rescaling O in tensor
+// memory is rare; it is done by the softmax threads themselves between two PV MMAs.
+// Causal masking comes from indices on the diagonal tile only; tiles above the diagonal
+// are never loaded.  CTAs are ordered longest-first.  Register budgets are re-partitioned
+// with setmaxnreg (56 for WG0, 224 for the softmax warpgroups; 384 x 168 at launch).
 #include "../device/ptx.cuh"
 #include "kernels.h"
 
@@ -25,22 +30,25 @@ constexpr int BQ = 128, BKV = 128;
 constexpr int KV_STAGES = 2;
 constexpr int SUB_BYTES = 128 * 64 * 2;       // one 128-row x 64-element swizzled sub-tile: 16 KiB
 constexpr int TILE_BYTES = 2 * SUB_BYTES;     // 128 x 128 bf16: 32 KiB
-constexpr int THREADS = 192;
-constexpr int SOFTMAX_THREADS = 128;
-constexpr int TMEM_COLS = 256;
-constexpr uint32_t COL_S = 0, COL_PV = 128;
+constexpr int THREADS = 384;
+constexpr int SOFTMAX_THREADS = 128;          // per query tile
+constexpr int TMEM_COLS = 512;
+constexpr int REGS_AT_LAUNCH = 168, REGS_WG0 = 56, REGS_SOFTMAX = 224;
+static_assert(128 * REGS_WG0 + 256 * REGS_SOFTMAX <= THREADS * REGS_AT_LAUNCH, "setmaxnreg split exceeds the pool");
+constexpr float RESCALE_THRESHOLD = 8.0f;     // log2 domain
 
 struct __align__(8) Ctrl {
     uint64_t q_full;
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
-    uint64_t s_full, p_full, o_full;
+    uint64_t s_full[2], p_full[2];
+    uint64_t o_final;
     uint32_t tmem_base;
     uint32_t abort;
 };
-constexpr size_t SMEM_BYTES = 1024 + (size_t)TILE_BYTES * (1 + 2 * KV_STAGES + 1) + sizeof(Ctrl);
+constexpr size_t SMEM_BYTES = 1024 + (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + sizeof(Ctrl);
 
-enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FULL };
+enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FINAL };
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -55,17 +63,25 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t *q_s = base;
-    uint8_t *k_s = q_s + TILE_BYTES;                  // [KV_STAGES]
-    uint8_t *v_s = k_s + KV_STAGES * TILE_BYTES;      // [KV_STAGES]
-    uint8_t *p_s = v_s + KV_STAGES * TILE_BYTES;
-    Ctrl *ctrl = reinterpret_cast<Ctrl *>(p_s + TILE_BYTES);
+    uint8_t *q_s = base;                               // [2] query tiles
+    uint8_t *k_s = q_s + 2 * TILE_BYTES;               // [KV_STAGES]
+    uint8_t *v_s = k_s + KV_STAGES * TILE_BYTES;       // [KV_STAGES]
+    Ctrl *ctrl = reinterpret_cast<Ctrl *>(v_s + KV_STAGES * TILE_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_tiles = (p.S + BQ - 1) / BQ;
-    const int qt = num_q_tiles - 1 - (int)(blockIdx.x / (unsigned)p.BH);   // longest first
+    const int num_pairs = (num_q_tiles + 1) / 2;
+    const int pair = num_pairs - 1 - (int)(blockIdx.x / (unsigned)p.BH);    // longest first
     const int bh = (int)(blockIdx.x % (unsigned)p.BH);
-    const int num_kv = p.causal ? qt + 1 : (p.S + BKV - 1) / BKV;
+    const int num_kv_all = (p.S + BKV - 1) / BKV;
+    // KV tiles each query tile walks over (0 if the second tile of the pair does not exist)
+    int J[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        const int qt = 2 * pair + t;
+        J[t] = qt >= num_q_tiles ? 0 : (p.causal ? qt + 1 : num_kv_all);
+    }
+    const int Jmax = J[0] > J[1] ? J[0] : J[1];
 
     if (threadIdx.x == 0) {
         mbar_init(&ctrl->q_full, 1);
@@ -73,9 +89,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             mbar_init(&ctrl->k_full[s], 1); mbar_init(&ctrl->k_empty[s], 1);
             mbar_init(&ctrl->v_full[s], 1); mbar_init(&ctrl->v_empty[s], 1);
         }
-        mbar_init(&ctrl->s_full, 1);
-        mbar_init(&ctrl->p_full, SOFTMAX_THREADS);
-        mbar_init(&ctrl->o_full, 1);
+        for (int t = 0; t < 2; ++t) { mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], SOFTMAX_THREADS); }
+        mbar_init(&ctrl->o_final, 1);
         ctrl->abort = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -90,13 +105,17 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const uint32_t tmem_base = ctrl->tmem_base;
     const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_ATTN};
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            mbar_arrive_expect_tx(&ctrl->q_full, TILE_BYTES);
-            tma_load_3d(q_s, &tmQ, &ctrl->q_full, 0, qt * BQ, bh);
-            tma_load_3d(q_s + SUB_BYTES, &tmQ, &ctrl->q_full, 64, qt * BQ, bh);
-            for (int j = 0; j < num_kv; ++j) {
+    if (warp < 4) {
+        setmaxnreg_dec<REGS_WG0>();
+        if (warp == 0 && lane == 0) {
+            // -------------------------------------------------------- TMA producer
+            mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
+                tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
+            }
+            for (int j = 0; j < Jmax; ++j) {
                 const int s = j % KV_STAGES;
                 const uint32_t ph = (j / KV_STAGES) & 1;
                 mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
@@ -108,162 +127,169 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
                 tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
             }
-        }
-    } else if (warp == 1) {
-        // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        } else if (warp == 1 && lane == 0) {
+            // ---------------------------------------------------------- MMA issuer
             const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false);   // Q, K both K-major (d contiguous)
-            const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major, V MN-major (d contiguous)
-            const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
-            auto issue_s = [&](int j) {
-                const int s = j % KV_STAGES;
-                const uint32_t ph = (j / KV_STAGES) & 1;
-                mbar_wait(&ctrl->k_full[s], ph, ctx, BAR_K_FULL);
-                tc_fence_after();
-                const uint32_t k_addr = smem_u32(k_s + s * TILE_BYTES);
+            const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major (TMEM), V MN-major
+            // S_t(j) = Q_t K_j^T into columns [t*128, t*128+128)
+            auto issue_s = [&](int t, int j) {
+                const uint32_t q_addr = smem_u32(q_s + t * TILE_BYTES);
+                const uint32_t k_addr = smem_u32(k_s + (j % KV_STAGES) * TILE_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
-                    umma_ss(tmem_base + COL_S, make_smem_desc_sw128(q_addr + off, 0, 1024),
+                    umma_ss(tmem_base + t * 128, make_smem_desc_sw128(q_addr + off, 0, 1024),
                             make_smem_desc_sw128(k_addr + off, 0, 1024), idesc_s, ks != 0 ? 1u : 0u);
                 }
-                umma_commit(&ctrl->s_full);
-                umma_commit(&ctrl->k_empty[s]);
+                umma_commit(&ctrl->s_full[t]);
+            };
+            // O_t (+)= P_t(j) V_j : A = bf16 P in TMEM (8 columns per 16 keys), B = V_j
+            auto issue_pv = [&](int t, int j) {
+                const uint32_t v_addr = smem_u32(v_s + (j % KV_STAGES) * TILE_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < BKV / 16; ++ks)
+                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8,
+                            make_smem_desc_sw128(v_addr + ks * 2048, SUB_BYTES, 1024), idesc_o,
+                            (j | ks) != 0 ? 1u : 0u);
             };
             mbar_wait(&ctrl->q_full, 0, ctx, BAR_Q);
-            issue_s(0);
-            for (int j = 0; j < num_kv; ++j) {
-                const int s = j % KV_STAGES;
-                const uint32_t ph = (j / KV_STAGES) & 1;
-                mbar_wait(&ctrl->p_full, j & 1, ctx, BAR_P_FULL);   // P_j in smem, S_j and PV_{j-1} consumed
+            if (Jmax > 0) {
+                mbar_wait(&ctrl->k_full[0], 0, ctx, BAR_K_FULL);
                 tc_fence_after();
-                if (j + 1 < num_kv) issue_s(j + 1);
-                mbar_wait(&ctrl->v_full[s], ph, ctx, BAR_V_FULL);
-                tc_fence_after();
-                const uint32_t v_addr = smem_u32(v_s + s * TILE_BYTES);
-#pragma unroll
-                for (int ks = 0; ks < BKV / 16; ++ks) {
-                    const uint32_t a_off = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
-                    umma_ss(tmem_base + COL_PV, make_smem_desc_sw128(p_addr + a_off, 0, 1024),
-                            make_smem_desc_sw128(v_addr + ks * 2048, SUB_BYTES, 1024), idesc_o, ks != 0 ? 1u : 0u);
-                }
-                umma_commit(&ctrl->o_full);
-                umma_commit(&ctrl->v_empty[s]);
+                if (J[0] > 0) issue_s(0, 0);
+                if (J[1] > 0) issue_s(1, 0);
+                umma_commit(&ctrl->k_empty[0]);
             }
+            for (int j = 0; j < Jmax; ++j) {
+                const int sv = j % KV_STAGES;
+                const uint32_t phv = (j / KV_STAGES) & 1;
+                const int sk = (j + 1) % KV_STAGES;
+                const uint32_t phk = ((j + 1) / KV_STAGES) & 1;
+                const bool act0 = j < J[0], act1 = j < J[1];
+                const bool nxt0 = j + 1 < J[0], nxt1 = j + 1 < J[1];
+                mbar_wait(&ctrl->v_full[sv], phv, ctx, BAR_V_FULL);
+                if (nxt0 || nxt1) mbar_wait(&ctrl->k_full[sk], phk, ctx, BAR_K_FULL);
+                if (act0) {
+                    mbar_wait(&ctrl->p_full[0], j & 1, ctx, BAR_P_FULL);
+                    tc_fence_after();
+                    issue_pv(0, j);
+                }
+                if (nxt0) issue_s(0, j + 1);
+                if (act1) {
+                    mbar_wait(&ctrl->p_full[1], j & 1, ctx, BAR_P_FULL);
+                    tc_fence_after();
+                    issue_pv(1, j);
+                }
+                umma_commit(&ctrl->v_empty[sv]);
+                if (nxt1) issue_s(1, j + 1);
+                if (nxt0 || nxt1) umma_commit(&ctrl->k_empty[sk]);
+            }
+            umma_commit(&ctrl->o_final);
         }
     } else {
-        // ----------------------------------------------------------------- softmax
-        const int q = warp & 3;
-        const int r_in_tile = q * 32 + lane;
-        const int qidx = qt * BQ + r_in_tile;
-        const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-        const float c = p.scale * 1.4426950408889634f;   // scores are kept in the log2 domain
-        float o[D];
+        setmaxnreg_inc<REGS_SOFTMAX>();
+        // --------------------------------------------------------------- softmax
+        const int t = (warp >> 2) - 1;
+        const int Jt = J[t];
+        if (Jt > 0) {
+            const int q = warp & 3;
+            const int r_in_tile = q * 32 + lane;
+            const int qidx = (2 * pair + t) * BQ + r_in_tile;
+            const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+            const uint32_t s_addr = tmem_base + lane_addr + t * 128;
+            const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128;
+            const float c = p.scale * 1.4426950408889634f;   // scores are kept in the log2 domain
+            float m_used = -INFINITY, l_run = 0.0f;
+
+            for (int j = 0; j < Jt; ++j) {
+                const bool edge = (j == Jt - 1);
+                const int k0 = j * BKV;
+                mbar_wait(&ctrl->s_full[t], j & 1, ctx, BAR_S_FULL);
+                tc_fence_after();
+
+                uint32_t s[BKV];
 #pragma unroll
-        for (int i = 0; i < D; ++i) o[i] = 0.0f;
-        float m_run = -INFINITY, l_run = 0.0f, alpha_prev = 0.0f;
-
-        for (int j = 0; j < num_kv; ++j) {
-            const bool edge = (j == num_kv - 1);
-            const int k0 = j * BKV;
-            mbar_wait(&ctrl->s_full, j & 1, ctx, BAR_S_FULL);
-            tc_fence_after();
-
-            // pass 1: row maximum of the scaled, masked scores
-            float tmax = -INFINITY;
-#pragma unroll 1
-            for (int cc = 0; cc < BKV / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + lane_addr + COL_S + cc * 32, r);
+                for (int cc = 0; cc < BKV / 32; ++cc)
+                    tmem_ld32(s_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cc * 32]));
                 tmem_ld_wait();
+
+                float tmax = -INFINITY;
                 if (edge) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const int kidx = k0 + cc * 32 + i;
+                    for (int i = 0; i < BKV; ++i) {
+                        const int kidx = k0 + i;
                         const bool ok = kidx < p.S && (!p.causal || kidx <= qidx);
-                        if (ok) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+                        const float v = ok ? __uint_as_float(s[i]) : -INFINITY;
+                        s[i] = __float_as_uint(v);
+                        tmax = fmaxf(tmax, v);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(r[i]));
+                    for (int i = 0; i < BKV; ++i) tmax = fmaxf(tmax, __uint_as_float(s[i]));
                 }
-            }
-            // the scale is positive, so max(s)*c == max(s*c); rows past S keep -inf and are never stored
-            float m_new = fmaxf(m_run, tmax * c);
-            if (m_new == -INFINITY) m_new = 0.0f;
-            const float alpha = ex2(m_run - m_new);
-
-            // fold the previous tile's PV into the register accumulator
-            if (j > 0) {
-                mbar_wait(&ctrl->o_full, (j - 1) & 1, ctx, BAR_O_FULL);
-                tc_fence_after();
-#pragma unroll
-                for (int cc = 0; cc < D / 32; ++cc) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem_base + lane_addr + COL_PV + cc * 32, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) o[cc * 32 + i] = fmaf(o[cc * 32 + i], alpha_prev, __uint_as_float(r[i]));
+                // the scale is positive, so max(s)*c == max(s*c)
+                float m_new = tmax * c;
+                if (m_new == -INFINITY) m_new = 0.0f;          // rows past S: nothing valid, never stored
+                const bool grow = m_new > m_used + RESCALE_THRESHOLD;
+                float alpha = 1.0f;
+                if (grow) {
+                    alpha = ex2(m_used - m_new);                // 0 on the first tile
+                    m_used = m_new;
                 }
-            }
-
-            // pass 2: probabilities -> bf16 -> shared memory (K-major, 128-byte swizzle)
-            float lsum = 0.0f;
-            const float neg_m = -m_new;
+                l_run *= alpha;
+                // S_t(j) complete implies PV_t(j-1) complete: O_t is quiescent until we signal P_t(j)
+                if (j > 0 && __any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-            for (int cc = 0; cc < BKV / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + lane_addr + COL_S + cc * 32, r);
-                tmem_ld_wait();
-                float pr[32];
+                    for (int cc = 0; cc < D / 32; ++cc) {
+                        uint32_t o[32];
+                        tmem_ld32(o_addr + cc * 32, o);
+                        tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float e = ex2(fmaf(__uint_as_float(r[i]), c, neg_m));
-                    if (edge) {
-                        const int kidx = k0 + cc * 32 + i;
-                        const bool ok = kidx < p.S && (!p.causal || kidx <= qidx);
-                        e = ok ? e : 0.0f;
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(o_addr + cc * 32, o);
                     }
-                    pr[i] = e;
-                    lsum += e;
                 }
-                uint8_t *prow = p_s + (cc >> 1) * SUB_BYTES + r_in_tile * 128;
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int chunk = ((cc & 1) * 4 + g) ^ (r_in_tile & 7);
-                    *reinterpret_cast<uint4 *>(prow + chunk * 16) =
-                        make_uint4(pack_bf16x2(pr[g * 8 + 0], pr[g * 8 + 1]), pack_bf16x2(pr[g * 8 + 2], pr[g * 8 + 3]),
-                                   pack_bf16x2(pr[g * 8 + 4], pr[g * 8 + 5]), pack_bf16x2(pr[g * 8 + 6], pr[g * 8 + 7]));
-                }
-            }
-            l_run = fmaf(l_run, alpha, lsum);
-            m_run = m_new;
-            alpha_prev = alpha;
-            fence_proxy_async_smem();
-            tc_fence_before();
-            mbar_arrive(&ctrl->p_full);
-        }
 
-        // last PV, normalise, store
-        mbar_wait(&ctrl->o_full, (num_kv - 1) & 1, ctx, BAR_O_FULL);
-        tc_fence_after();
-        const float inv_l = 1.0f / l_run;
-        __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + ((long long)bh * p.S + qidx) * D;
+                const float neg_m = -m_used;
+                float lsum = 0.0f;
 #pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-            uint32_t r[32];
-            tmem_ld32(tmem_base + lane_addr + COL_PV + cc * 32, r);
-            tmem_ld_wait();
-            if (qidx < p.S) {
+                for (int cc = 0; cc < 2; ++cc) {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    float f[8];
+                    for (int i = 0; i < 32; ++i) {
+                        const float e0 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i]), c, neg_m));
+                        const float e1 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i + 1]), c, neg_m));
+                        lsum += e0 + e1;
+                        pk[i] = pack_bf16x2(e0, e1);
+                    }
+                    tmem_st32(s_addr + cc * 32, pk);
+                }
+                l_run += lsum;
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&ctrl->p_full[t]);
+            }
+
+            // all MMAs done: normalise and store
+            mbar_wait(&ctrl->o_final, 0, ctx, BAR_O_FINAL);
+            tc_fence_after();
+            const float inv_l = 1.0f / l_run;
+            __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + ((long long)bh * p.S + qidx) * D;
+#pragma unroll 1
+            for (int cc = 0; cc < D / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(o_addr + cc * 32, r);
+                tmem_ld_wait();
+                if (qidx < p.S) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        f[i] = fmaf(o[cc * 32 + g * 8 + i], alpha_prev, __uint_as_float(r[g * 8 + i])) * inv_l;
-                    *reinterpret_cast<uint4 *>(orow + cc * 32 + g * 8) =
-                        make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
-                                   pack_bf16x2(f[6], f[7]));
+                    for (int g = 0; g < 4; ++g) {
+                        float f[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[g * 8 + i]) * inv_l;
+                        *reinterpret_cast<uint4 *>(orow + cc * 32 + g * 8) =
+                            make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
+                                       pack_bf16x2(f[6], f[7]));
+                    }
                 }
             }
         }
@@ -284,11 +310,22 @@ cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK
                                   const AttnArgs &a, cudaStream_t stream)
 {
     if (a.BH <= 0 || a.S <= 0) return cudaSuccess;
+    // The in-kernel setmaxnreg split draws on threads x registers-at-launch; refuse to launch
+    // (rather than wait forever inside the kernel) if the compiled kernel was given fewer.
+    static int regs_ok = -1;
+    if (regs_ok < 0) {
+        cudaFuncAttributes attr;
+        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel);
+        if (e != cudaSuccess) return e;
+        regs_ok = (attr.numRegs * THREADS >= 128 * REGS_WG0 + 256 * REGS_SOFTMAX) ? 1 : 0;
+    }
+    if (!regs_ok) return cudaErrorLaunchOutOfResources;
     const int num_q_tiles = (a.S + BQ - 1) / BQ;
+    const int num_pairs = (num_q_tiles + 1) / 2;
     cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attention_bf16_kernel<<<dim3((unsigned)num_q_tiles * (unsigned)a.BH), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
+    attention_bf16_kernel<<<dim3((unsigned)num_pairs * (unsigned)a.BH), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError();
 }
 
