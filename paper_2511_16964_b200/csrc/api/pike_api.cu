@@ -177,7 +177,7 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
         return st;
     if (w_is_nk) {
         if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
-                                           pike::GEMM_BK, pike::GEMM_BN))
+                                           pike::GEMM_BK, pike::GEMM_BN / 2))
             return st;
     } else {
         if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0], 64,

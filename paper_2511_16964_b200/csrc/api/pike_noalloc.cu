@@ -129,7 +129,7 @@ extern "C" pike_status_t pike_linear_softmax_noalloc(pike_handle_t h, const pike
                                      pike::GEMM_BM))
         return st;
     if (pike_status_t st = nk ? encode_2d(h, &tmB, w->data, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
-                                          pike::GEMM_BK, pike::GEMM_BN)
+                                          pike::GEMM_BK, pike::GEMM_BN / 2)
                               : encode_2d(h, &tmB, w->data, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0], 64,
                                           pike::GEMM_BK))
         return st;

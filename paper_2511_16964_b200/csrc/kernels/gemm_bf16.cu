@@ -3,15 +3,20 @@
 //
 //   out[m,n] = scale * act( sum_k A[m,k] * W[k,n] + bias[n] ) + residual[m,n]
 //
-// Persistent, warp-specialised CTAs (one per SM, 192 threads):
-//   warp 0      TMA producer: A tile 128x64 and W tile 256x64 (or 64x256 when W is
-//               [K,N]) into a 4-stage 128-byte-swizzled shared-memory ring
-//   warp 1      allocates 512 tensor-memory columns (two 128x256 fp32 accumulators)
-//               and issues tcgen05.mma (one thread), committing to mbarriers
-//   warps 2..5  epilogue: tcgen05.ld the finished accumulator (thread = row, 32
-//               columns at a time), bias/activation/scale/residual in registers,
-//               16-byte stores; optionally per-row (max, sum exp) partials for a
-//               softmax split across N tiles.  Runs under the next tile's K loop.
+// Persistent clusters of two CTAs (cta_group::2), one cluster per SM pair, each cluster
+// walking over 256 x 256 output tiles.  Per CTA (192 threads):
+//   warp 0      TMA producer: this CTA's 128 rows of A and its 128 of the tile's 256 W
+//               columns, 64 k at a time, into a 6-stage 128-byte-swizzled ring (32 KiB per
+//               stage).  Both CTAs' loads complete on the LEADER's "full" barrier.
+//   warp 1      allocates 512 tensor-memory columns (two 128x256 fp32 accumulator stages
+//               per CTA); in the leader CTA one thread issues tcgen05.mma.cta_group::2
+//               (256x256x16) for the pair and commits to mbarriers in both CTAs
+//   warps 2..5  epilogue: tcgen05.ld this CTA's accumulator rows (thread = row, 32
+//               columns at a time), bias/activation/scale/residual in registers, 16-byte
+//               stores; optionally per-row (max, sum exp) partials for a softmax split
+//               across N tiles.  Runs under the next tile's K loop.
+// The pair halves the W traffic each SM's shared memory sees compared with a 128x256
+// single-CTA tile, which was shared-memory-bandwidth bound.  No TMA multicast is used.
 // Every mbarrier wait is bounded (see mbar_wait).
 #include "../device/act.cuh"
 #include "../device/ptx.cuh"
@@ -20,22 +25,25 @@
 namespace pike {
 namespace {
 
-constexpr int BM = GEMM_BM, BN = GEMM_BN, BK = GEMM_BK;
-constexpr int STAGES = 4;
+constexpr int BM = GEMM_BM;                     // rows per CTA (the pair covers 2*BM)
+constexpr int BN = GEMM_BN, BK = GEMM_BK;
+constexpr int BN_HALF = BN / 2;                 // W columns staged by each CTA
+constexpr int STAGES = 6;
 constexpr int A_BYTES = BM * BK * 2;            // 16 KiB
-constexpr int B_BYTES = BN * BK * 2;            // 32 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 48 KiB
+constexpr int B_BYTES = BN_HALF * BK * 2;       // 16 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 32 KiB per CTA
 constexpr int NUM_ACC = 2;
 constexpr int TMEM_COLS = NUM_ACC * BN;         // 512
 constexpr int THREADS = 192;
 constexpr int EPI_THREADS = 128;
-constexpr int GROUP_M = 8;                      // tile rasterisation: 8 row-blocks per column sweep
+constexpr int EPI_WARPS = 4;
+constexpr int GROUP_M = 4;                      // rasterisation: 4 pair-row-blocks (1024 rows) per column sweep
 
 struct __align__(8) Ctrl {
-    uint64_t full[STAGES];
-    uint64_t empty[STAGES];
-    uint64_t tmem_full[NUM_ACC];
-    uint64_t tmem_empty[NUM_ACC];
+    uint64_t full[STAGES];        // used in the leader: both CTAs' TMA bytes land here
+    uint64_t empty[STAGES];       // in each CTA: stage consumed (multicast commit)
+    uint64_t tmem_full[NUM_ACC];  // in each CTA: accumulator ready (multicast commit)
+    uint64_t tmem_empty[NUM_ACC]; // used in the leader: 4 epilogue warps x 2 CTAs drained it
     uint32_t tmem_base;
     uint32_t abort;
     float bias[BN];
@@ -56,7 +64,7 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_
 }
 
 template <int ACT>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -64,24 +72,27 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(tiles + (size_t)STAGES * STAGE_BYTES);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_m = (p.M + BM - 1) / BM, num_n = (p.N + BN - 1) / BN;
+    const uint32_t rank = cluster_ctarank();           // 0 = leader
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    const int num_m = (p.M + 2 * BM - 1) / (2 * BM), num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], 1); }
-        for (int a = 0; a < NUM_ACC; ++a) { mbar_init(&ctrl->tmem_full[a], 1); mbar_init(&ctrl->tmem_empty[a], EPI_THREADS); }
+        for (int a = 0; a < NUM_ACC; ++a) { mbar_init(&ctrl->tmem_full[a], 1); mbar_init(&ctrl->tmem_empty[a], 2 * EPI_WARPS); }
         ctrl->abort = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
     }
     if (warp == 1) {
-        tmem_alloc(&ctrl->tmem_base, TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc_pair(&ctrl->tmem_base, TMEM_COLS);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();          // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = ctrl->tmem_base;
     const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
@@ -91,41 +102,44 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane == 0) {
             int s = 0;
             uint32_t ph = 0;
-            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+            for (int t = cluster_id; t < num_tiles; t += num_clusters) {
                 int m_blk, n_blk;
                 tile_coords(t, num_m, num_n, m_blk, n_blk);
+                const int row0 = m_blk * 2 * BM + (int)rank * BM;
+                const int col0 = n_blk * BN + (int)rank * BN_HALF;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     mbar_wait(&ctrl->empty[s], ph ^ 1, ctx, BAR_EMPTY);
                     uint8_t *a_s = tiles + (size_t)s * STAGE_BYTES;
                     uint8_t *b_s = a_s + A_BYTES;
-                    mbar_arrive_expect_tx(&ctrl->full[s], STAGE_BYTES);
-                    tma_load_2d(a_s, &tmA, &ctrl->full[s], kb * BK, m_blk * BM);
+                    const uint32_t full_leader = mapa_shared(smem_u32(&ctrl->full[s]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&ctrl->full[s], 2 * STAGE_BYTES);
+                    tma_load_2d_pair(a_s, &tmA, full_leader, kb * BK, row0);
                     if (p.w_is_nk) {
-                        tma_load_2d(b_s, &tmB, &ctrl->full[s], kb * BK, n_blk * BN);
+                        tma_load_2d_pair(b_s, &tmB, full_leader, kb * BK, col0);
                     } else {
 #pragma unroll
-                        for (int i = 0; i < BN / 64; ++i)
-                            tma_load_2d(b_s + i * (64 * BK * 2), &tmB, &ctrl->full[s], n_blk * BN + i * 64, kb * BK);
+                        for (int i = 0; i < BN_HALF / 64; ++i)
+                            tma_load_2d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK);
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
-        // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc_bf16(BM, BN, false, !p.w_is_nk);
+        // ------------------------------------------------- MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk);
             int s = 0;
             uint32_t ph = 0;
             int it = 0;
-            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+            for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
                 const int acc = it & 1;
                 const uint32_t aph = (it >> 1) & 1;
-                mbar_wait(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
+                mbar_wait_cluster(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
-                    mbar_wait(&ctrl->full[s], ph, ctx, BAR_FULL);
+                    mbar_wait_cluster(&ctrl->full[s], ph, ctx, BAR_FULL);
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(tiles + (size_t)s * STAGE_BYTES);
                     const uint32_t b_addr = a_addr + A_BYTES;
@@ -134,12 +148,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         const uint64_t adesc = make_smem_desc_sw128(a_addr + k * 32, 0, 1024);
                         const uint64_t bdesc = p.w_is_nk ? make_smem_desc_sw128(b_addr + k * 32, 0, 1024)
                                                          : make_smem_desc_sw128(b_addr + k * 2048, 64 * BK * 2, 1024);
-                        umma_ss(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(&ctrl->empty[s]);
+                    umma_commit_pair(&ctrl->empty[s], 0x3);
                     if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
-                umma_commit(&ctrl->tmem_full[acc]);
+                umma_commit_pair(&ctrl->tmem_full[acc], 0x3);
             }
         }
     } else {
@@ -147,13 +161,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int et = threadIdx.x - 64;        // 0..127
         int it = 0;
-        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+        for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
             int m_blk, n_blk;
             tile_coords(t, num_m, num_n, m_blk, n_blk);
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int n0 = n_blk * BN;
-            const int row = m_blk * BM + q * 32 + lane;
+            const int row = m_blk * 2 * BM + (int)rank * BM + q * 32 + lane;
             const bool row_ok = row < p.M;
 
             // stage the tile's bias as fp32
@@ -257,9 +271,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
-            // accumulator drained: hand the TMEM stage back to the MMA warp
+            // accumulator drained: one arrival per epilogue warp on the LEADER's barrier
             tc_fence_before();
-            mbar_arrive(&ctrl->tmem_empty[acc]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctrl->tmem_empty[acc]), 0));
 
             if (p.softmax_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
         }
@@ -269,9 +284,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (ctrl->abort) abort_drain();
+    cluster_sync_all();          // neither CTA frees tensor memory while the pair may still use it
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
     }
 }
 
@@ -280,14 +296,33 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
                              cudaStream_t stream)
 {
-    const int num_m = (a.M + BM - 1) / BM, num_n = (a.N + BN - 1) / BN;
+    const int num_m = (a.M + 2 * BM - 1) / (2 * BM), num_n = (a.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     if (num_tiles <= 0) return cudaSuccess;
-    const dim3 grid(num_tiles < num_sms ? num_tiles : num_sms), block(THREADS);
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        kern<<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, a);
+        // how many CTA pairs the device can hold at once (one CTA per SM at this shared-memory size)
+        static int max_clusters = 0;
+        if (max_clusters == 0) {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * (num_sms / 2));
+            cfg.blockDim = dim3(THREADS);
+            cfg.dynamicSmemBytes = SMEM_BYTES;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+                cudaGetLastError();
+                n = num_sms / 2;
+            }
+            max_clusters = n < num_sms / 2 ? n : num_sms / 2;
+        }
+        const int clusters = num_tiles < max_clusters ? num_tiles : max_clusters;
+        kern<<<dim3(2 * clusters), dim3(THREADS), SMEM_BYTES, stream>>>(tmA, tmB, a);
         return cudaGetLastError();
     };
     switch (a.act) {

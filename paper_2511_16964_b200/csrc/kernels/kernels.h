@@ -37,6 +37,9 @@ struct GemmArgs {
     unsigned int *status;
     unsigned long long limit_ns;
 };
+// A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
+// the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
+// W as [K,N] {64, GEMM_BK}.
 constexpr int GEMM_BM = 128, GEMM_BN = 256, GEMM_BK = 64;
 cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
                              cudaStream_t stream);
