@@ -68,14 +68,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // releases tensor memory and returns; the host sees PIKE_ERR_TIMEOUT.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const WaitCtx &ctx, uint32_t barrier_id)
 {
+    // Fast path: poll.  The clock (a slow system register) and the abort word are only looked at
+    // every 1024 failed polls, so an ordinary hand-off never pays for them.
     if (mbar_try_wait(bar, parity)) return true;
-    if (*ctx.abort) return false;
-    const unsigned long long t0 = globaltimer_ns();
     uint32_t spins = 0;
+    unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0xFF) == 0) {
+        if ((++spins & 0x3FF) == 0) {
             if (*ctx.abort) return false;
-            if (globaltimer_ns() - t0 > ctx.limit_ns) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > ctx.limit_ns) {
                 *ctx.abort = 1;
                 if (ctx.status != nullptr) {
                     if (atomicCAS(ctx.status, 0u, (ctx.kernel_id << 16) | barrier_id) == 0u)
@@ -299,13 +303,15 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mas
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, const WaitCtx &ctx, uint32_t barrier_id)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
-    if (*ctx.abort) return false;
-    const unsigned long long t0 = globaltimer_ns();
     uint32_t spins = 0;
+    unsigned long long t0 = 0;
     while (!mbar_try_wait_cluster(bar, parity)) {
-        if ((++spins & 0xFF) == 0) {
+        if ((++spins & 0x3FF) == 0) {
             if (*ctx.abort) return false;
-            if (globaltimer_ns() - t0 > ctx.limit_ns) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > ctx.limit_ns) {
                 *ctx.abort = 1;
                 if (ctx.status != nullptr) {
                     if (atomicCAS(ctx.status, 0u, (ctx.kernel_id << 16) | barrier_id) == 0u)

@@ -17,7 +17,7 @@
 // more than 2^8 (probabilities stay bounded by 256 in between), so rescaling O in tensor
 // memory is rare; it is done by the softmax threads themselves between two PV MMAs.
 // Causal masking comes from indices on the diagonal tile only; tiles above the diagonal
-// are never loaded.  CTAs are ordered longest-first.  Register budgets are re-partitioned
+// are never loaded.  CTAs are ordered head by head, longest first within a head.  Register budgets are re-partitioned
 // with setmaxnreg (56 for WG0, 224 for the softmax warpgroups; 384 x 168 at launch).
 #include "../device/ptx.cuh"
 #include "kernels.h"
@@ -71,8 +71,10 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_tiles = (p.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
-    const int pair = num_pairs - 1 - (int)(blockIdx.x / (unsigned)p.BH);    // longest first
-    const int bh = (int)(blockIdx.x % (unsigned)p.BH);
+    // head-major order: the CTAs of one head are neighbours (longest first within the head), so the
+    // head's K/V tiles are shared through L2 by the CTAs walking over them at the same time
+    const int bh = (int)(blockIdx.x / (unsigned)num_pairs);
+    const int pair = num_pairs - 1 - (int)(blockIdx.x % (unsigned)num_pairs);
     const int num_kv_all = (p.S + BKV - 1) / BKV;
     // KV tiles each query tile walks over (0 if the second tile of the pair does not exist)
     int J[2];
@@ -213,7 +215,10 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     tmem_ld32(s_addr + cc * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[cc * 32]));
                 tmem_ld_wait();
 
-                float tmax = -INFINITY;
+                // eight independent partial maxima keep the dependency chains short
+                float pm[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pm[i] = -INFINITY;
                 if (edge) {
 #pragma unroll
                     for (int i = 0; i < BKV; ++i) {
@@ -221,12 +226,14 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                         const bool ok = kidx < p.S && (!p.causal || kidx <= qidx);
                         const float v = ok ? __uint_as_float(s[i]) : -INFINITY;
                         s[i] = __float_as_uint(v);
-                        tmax = fmaxf(tmax, v);
+                        pm[i & 7] = fmaxf(pm[i & 7], v);
                     }
                 } else {
 #pragma unroll
-                    for (int i = 0; i < BKV; ++i) tmax = fmaxf(tmax, __uint_as_float(s[i]));
+                    for (int i = 0; i < BKV; ++i) pm[i & 7] = fmaxf(pm[i & 7], __uint_as_float(s[i]));
                 }
+                const float tmax = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])),
+                                         fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
                 // the scale is positive, so max(s)*c == max(s*c)
                 float m_new = tmax * c;
                 if (m_new == -INFINITY) m_new = 0.0f;          // rows past S: nothing valid, never stored
@@ -251,7 +258,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 }
 
                 const float neg_m = -m_used;
-                float lsum = 0.0f;
+                float ls[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
                     uint32_t pk[32];
@@ -259,12 +266,12 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     for (int i = 0; i < 32; ++i) {
                         const float e0 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i]), c, neg_m));
                         const float e1 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i + 1]), c, neg_m));
-                        lsum += e0 + e1;
+                        ls[i & 3] += e0 + e1;
                         pk[i] = pack_bf16x2(e0, e1);
                     }
                     tmem_st32(s_addr + cc * 32, pk);
                 }
-                l_run += lsum;
+                l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(&ctrl->p_full[t]);
