@@ -91,6 +91,99 @@ layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_b
     }
 }
 
+// One WARP per row for rows of at most 4096 elements: the row sits in 16 x 16-byte registers per
+// lane, both reductions are pure shuffles (no block barrier), and eight independent rows per CTA keep
+// many loads in flight.
+constexpr int LNW_WARPS = 8;
+constexpr int LNW_MAX_CHUNKS = 16;  // D <= 32 * 16 * 8 = 4096
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// eight consecutive parameters starting at element e (e % 8 == 0) as fp32; KIND 0 = absent, 1 = bf16, 2 = f32
+template <int KIND>
+__device__ __forceinline__ void load_param8(const void *p, int e, float dflt, float (&out)[8])
+{
+    if constexpr (KIND == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i] = dflt;
+    } else if constexpr (KIND == 2) {
+        const float4 a = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(p) + e));
+        const float4 b = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(p) + e + 4));
+        out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+        out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+    } else {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p) + e));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) { out[2 * h] = bf16_lo(w[h]); out[2 * h + 1] = bf16_hi(w[h]); }
+    }
+}
+
+template <int GK, int BK>
+__global__ void __launch_bounds__(LNW_WARPS * 32, 2)
+layernorm_bf16_warp_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_bfloat16 *__restrict__ z,
+                           long long ldz, const void *gamma, const void *beta, float eps, int M, int D)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * LNW_WARPS + (threadIdx.x >> 5);
+    if (row >= M) return;
+    const uint4 *xr = reinterpret_cast<const uint4 *>(x + row * ldx);
+    const int nchunks = D / 8;
+
+    uint4 c[LNW_MAX_CHUNKS];
+#pragma unroll
+    for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
+        const int ci = lane + i * 32;
+        c[i] = ci < nchunks ? __ldg(xr + ci) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    float sum = 0.0f;
+#pragma unroll
+    for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
+        const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+        for (int h = 0; h < 4; ++h) sum += bf16_lo(w[h]) + bf16_hi(w[h]);   // padding chunks are zero
+    }
+    const float mean = warp_sum(sum) / (float)D;
+    float ss = 0.0f;
+#pragma unroll
+    for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
+        if (lane + i * 32 < nchunks) {
+            const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const float a = bf16_lo(w[h]) - mean, b = bf16_hi(w[h]) - mean;
+                ss += a * a + b * b;
+            }
+        }
+    }
+    const float rstd = rsqrtf(warp_sum(ss) / (float)D + eps);
+    uint4 *zr = reinterpret_cast<uint4 *>(z + row * ldz);
+#pragma unroll
+    for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
+        const int ci = lane + i * 32;
+        if (ci < nchunks) {
+            const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
+            float g[8], be[8];
+            load_param8<GK>(gamma, ci * 8, 1.0f, g);
+            load_param8<BK>(beta, ci * 8, 0.0f, be);
+            uint32_t o[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const float a = (bf16_lo(w[h]) - mean) * rstd * g[2 * h] + be[2 * h];
+                const float b = (bf16_hi(w[h]) - mean) * rstd * g[2 * h + 1] + be[2 * h + 1];
+                o[h] = pack_bf16x2(a, b);
+            }
+            zr[ci] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+        asm volatile("" ::: "memory");   // keep the parameter loads of later chunks from being hoisted (registers)
+    }
+}
+
 constexpr int SM_THREADS = 256;
 
 // One CTA per row: combine the per-tile (max, sum exp) pairs
@@ -149,6 +242,18 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
 {
     if (M <= 0) return cudaSuccess;
     if (D % 8 != 0 || D > LN_THREADS * LN_MAX_CHUNKS * 8) return cudaErrorInvalidValue;
+    if (D <= 32 * LNW_MAX_CHUNKS * 8) {
+        const int gk = gamma == nullptr ? 0 : (gamma_f32 ? 2 : 1), bk = beta == nullptr ? 0 : (beta_f32 ? 2 : 1);
+        const dim3 grid((M + LNW_WARPS - 1) / LNW_WARPS), block(LNW_WARPS * 32);
+        const __nv_bfloat16 *xp = static_cast<const __nv_bfloat16 *>(x);
+        __nv_bfloat16 *zp = static_cast<__nv_bfloat16 *>(z);
+#define PIKE_LN_CASE(G, B) \
+    if (gk == G && bk == B) layernorm_bf16_warp_kernel<G, B><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D);
+        PIKE_LN_CASE(0, 0) PIKE_LN_CASE(0, 1) PIKE_LN_CASE(0, 2) PIKE_LN_CASE(1, 0) PIKE_LN_CASE(1, 1)
+        PIKE_LN_CASE(1, 2) PIKE_LN_CASE(2, 0) PIKE_LN_CASE(2, 1) PIKE_LN_CASE(2, 2)
+#undef PIKE_LN_CASE
+        return cudaGetLastError();
+    }
     layernorm_bf16_kernel<<<M, LN_THREADS, 0, stream>>>(static_cast<const __nv_bfloat16 *>(x), ldx,
                                                          static_cast<__nv_bfloat16 *>(z), ldz, gamma, gamma_f32, beta,
                                                          beta_f32, eps, D);
