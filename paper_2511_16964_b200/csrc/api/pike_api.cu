@@ -550,7 +550,7 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     a.status = h->status;
     a.limit_ns = h->limit_ns;
     TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
-    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -2,7 +2,10 @@
 // Scores and probabilities live in tensor memory and registers only; nothing but
 // Q, K, V and O touches HBM.
 //
-// One CTA per (batch*head, PAIR of 128-query tiles), 384 threads = 3 warpgroups:
+// Persistent CTAs (one per SM) walk over work items = (batch*head, PAIR of 128-query tiles), longest
+// items first, round-robin; barriers, rings and tensor memory carry over from item to item, so the next
+// item's Q/K/V loads and first MMAs overlap the previous item's last softmax and output store.
+// 384 threads = 3 warpgroups:
 //   WG0  warp 0: TMA producer (both Q tiles once, then K_j / V_j tiles of 128 keys into
 //        two-stage 128-byte-swizzled rings); warp 1: MMA issuer (one thread)
 //   WG1  softmax for query tile 0        WG2  softmax for query tile 1   (thread = row)
@@ -17,8 +20,8 @@
 // more than 2^8 (probabilities stay bounded by 256 in between), so rescaling O in tensor
 // memory is rare; it is done by the softmax threads themselves between two PV MMAs.
 // Causal masking comes from indices on the diagonal tile only; tiles above the diagonal
-// are never loaded.  CTAs are ordered head by head, longest first within a head.  Register budgets are re-partitioned
-// with setmaxnreg (56 for WG0, 224 for the softmax warpgroups; 384 x 168 at launch).
+// are never loaded.  Register budgets are re-partitioned
+// with setmaxnreg (104 for WG0, 200 for the softmax warpgroups; 384 x 168 at launch).
 #include "../device/ptx.cuh"
 #include "kernels.h"
 
@@ -33,7 +36,7 @@ constexpr int TILE_BYTES = 2 * SUB_BYTES;     // 128 x 128 bf16: 32 KiB
 constexpr int THREADS = 384;
 constexpr int SOFTMAX_THREADS = 128;          // per query tile
 constexpr int TMEM_COLS = 512;
-constexpr int REGS_AT_LAUNCH = 168, REGS_WG0 = 56, REGS_SOFTMAX = 224;
+constexpr int REGS_AT_LAUNCH = 168, REGS_WG0 = 104, REGS_SOFTMAX = 200;
 static_assert(128 * REGS_WG0 + 256 * REGS_SOFTMAX <= THREADS * REGS_AT_LAUNCH, "setmaxnreg split exceeds the pool");
 constexpr float RESCALE_THRESHOLD = 8.0f;     // log2 domain
 
@@ -41,14 +44,15 @@ struct __align__(8) Ctrl {
     uint64_t q_full;
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
+    uint64_t q_empty;
     uint64_t s_full[2], p_full[2];
-    uint64_t o_final;
+    uint64_t o_final[2], o_free[2];
     uint32_t tmem_base;
     uint32_t abort;
 };
 constexpr size_t SMEM_BYTES = 1024 + (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + sizeof(Ctrl);
 
-enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FINAL };
+enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FINAL, BAR_Q_EMPTY, BAR_O_FREE };
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -71,19 +75,31 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_tiles = (p.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
-    // head-major order: the CTAs of one head are neighbours (longest first within the head), so the
-    // head's K/V tiles are shared through L2 by the CTAs walking over them at the same time
-    const int bh = (int)(blockIdx.x / (unsigned)num_pairs);
-    const int pair = num_pairs - 1 - (int)(blockIdx.x % (unsigned)num_pairs);
     const int num_kv_all = (p.S + BKV - 1) / BKV;
-    // KV tiles each query tile walks over (0 if the second tile of the pair does not exist)
-    int J[2];
+    // Work order.  A "slot" is one head's longest remaining pair of query tiles together with its shortest
+    // (under the causal mask pair u costs 4u+3 tile-MMAs, so every slot of a head costs the same); slots
+    // are dealt round-robin to the persistent CTAs.  All CTAs get equal work, CTAs running at the same
+    // time sit on neighbouring heads (their K/V tiles are shared through L2), and a CTA's second item
+    // re-reads the K/V tiles its first item just used.  i counts this CTA's items: 2 per slot.
+    const int slots_per_head = (num_pairs + 1) / 2;
+    const int num_slots = slots_per_head * p.BH;
+    // returns 0 = past the end, 1 = nothing to do for this i, 2 = item decoded; J[t] = KV tiles query
+    // tile t walks over (0 if the second tile of the pair does not exist)
+    auto decode = [&](int i, int &pair, int &bh, int (&J)[2]) -> int {
+        const int v = (int)blockIdx.x + (i >> 1) * (int)gridDim.x;
+        if (v >= num_slots) return 0;
+        bh = v / slots_per_head;
+        const int combo = v % slots_per_head;
+        const int hi = num_pairs - 1 - combo, lo = combo;
+        if ((i & 1) && lo >= hi) return 1;     // odd pair count: the middle pair is a slot by itself
+        pair = (i & 1) ? lo : hi;
 #pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        const int qt = 2 * pair + t;
-        J[t] = qt >= num_q_tiles ? 0 : (p.causal ? qt + 1 : num_kv_all);
-    }
-    const int Jmax = J[0] > J[1] ? J[0] : J[1];
+        for (int t = 0; t < 2; ++t) {
+            const int qt = 2 * pair + t;
+            J[t] = qt >= num_q_tiles ? 0 : (p.causal ? qt + 1 : num_kv_all);
+        }
+        return 2;
+    };
 
     if (threadIdx.x == 0) {
         mbar_init(&ctrl->q_full, 1);
@@ -91,8 +107,11 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             mbar_init(&ctrl->k_full[s], 1); mbar_init(&ctrl->k_empty[s], 1);
             mbar_init(&ctrl->v_full[s], 1); mbar_init(&ctrl->v_empty[s], 1);
         }
-        for (int t = 0; t < 2; ++t) { mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], SOFTMAX_THREADS); }
-        mbar_init(&ctrl->o_final, 1);
+        mbar_init(&ctrl->q_empty, 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], SOFTMAX_THREADS);
+            mbar_init(&ctrl->o_final[t], 1); mbar_init(&ctrl->o_free[t], SOFTMAX_THREADS);
+        }
         ctrl->abort = 0;
         fence_barrier_init();
         tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -111,102 +130,131 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         setmaxnreg_dec<REGS_WG0>();
         if (warp == 0 && lane == 0) {
             // -------------------------------------------------------- TMA producer
-            mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
+            int g = 0, it = 0;      // KV tiles and items issued so far
+            for (int i = 0;; ++i) {
+                int pair, bh, J[2];
+                const int st = decode(i, pair, bh, J);
+                if (st == 0) break;
+                if (st == 1) continue;
+                const int Jmax = J[0] > J[1] ? J[0] : J[1];
+                mbar_wait(&ctrl->q_empty, (it & 1) ^ 1, ctx, BAR_Q_EMPTY);   // the previous item's S MMAs are done
+                mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
 #pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
-                tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
-            }
-            for (int j = 0; j < Jmax; ++j) {
-                const int s = j % KV_STAGES;
-                const uint32_t ph = (j / KV_STAGES) & 1;
-                mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
-                mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
-                tma_load_3d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh);
-                tma_load_3d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh);
-                mbar_wait(&ctrl->v_empty[s], ph ^ 1, ctx, BAR_V_EMPTY);
-                mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
-                tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
-                tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
+                for (int t = 0; t < 2; ++t) {
+                    tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
+                    tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
+                }
+                for (int j = 0; j < Jmax; ++j, ++g) {
+                    const int s = g % KV_STAGES;
+                    const uint32_t ph = (g / KV_STAGES) & 1;
+                    mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
+                    mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
+                    tma_load_3d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh);
+                    tma_load_3d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh);
+                    mbar_wait(&ctrl->v_empty[s], ph ^ 1, ctx, BAR_V_EMPTY);
+                    mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
+                    tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
+                    tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
+                }
+                ++it;
             }
         } else if (warp == 1 && lane == 0) {
             // ---------------------------------------------------------- MMA issuer
             const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false);   // Q, K both K-major (d contiguous)
             const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major (TMEM), V MN-major
-            // S_t(j) = Q_t K_j^T into columns [t*128, t*128+128)
-            auto issue_s = [&](int t, int j) {
+            // S_t = Q_t K^T (K tile in ring stage ks) into columns [t*128, t*128+128)
+            auto issue_s = [&](int t, int ks) {
                 const uint32_t q_addr = smem_u32(q_s + t * TILE_BYTES);
-                const uint32_t k_addr = smem_u32(k_s + (j % KV_STAGES) * TILE_BYTES);
+                const uint32_t k_addr = smem_u32(k_s + ks * TILE_BYTES);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * SUB_BYTES + (kk & 3) * 32;
                     umma_ss(tmem_base + t * 128, make_smem_desc_sw128(q_addr + off, 0, 1024),
-                            make_smem_desc_sw128(k_addr + off, 0, 1024), idesc_s, ks != 0 ? 1u : 0u);
+                            make_smem_desc_sw128(k_addr + off, 0, 1024), idesc_s, kk != 0 ? 1u : 0u);
                 }
                 umma_commit(&ctrl->s_full[t]);
             };
-            // O_t (+)= P_t(j) V_j : A = bf16 P in TMEM (8 columns per 16 keys), B = V_j
-            auto issue_pv = [&](int t, int j) {
-                const uint32_t v_addr = smem_u32(v_s + (j % KV_STAGES) * TILE_BYTES);
+            // O_t (+)= P_t V (V tile in ring stage vs): A = bf16 P in TMEM (8 columns per 16 keys)
+            auto issue_pv = [&](int t, int vs, bool first) {
+                const uint32_t v_addr = smem_u32(v_s + vs * TILE_BYTES);
 #pragma unroll
-                for (int ks = 0; ks < BKV / 16; ++ks)
-                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + ks * 8,
-                            make_smem_desc_sw128(v_addr + ks * 2048, SUB_BYTES, 1024), idesc_o,
-                            (j | ks) != 0 ? 1u : 0u);
+                for (int kk = 0; kk < BKV / 16; ++kk)
+                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8,
+                            make_smem_desc_sw128(v_addr + kk * 2048, SUB_BYTES, 1024), idesc_o,
+                            (first && kk == 0) ? 0u : 1u);
             };
-            mbar_wait(&ctrl->q_full, 0, ctx, BAR_Q);
-            if (Jmax > 0) {
-                mbar_wait(&ctrl->k_full[0], 0, ctx, BAR_K_FULL);
+            int g = 0, it = 0;                 // KV tiles / items consumed so far
+            uint32_t n_s[2] = {0, 0};          // softmax hand-offs per query tile so far
+            uint32_t n_o[2] = {0, 0};          // items finished per query tile so far
+            for (int i = 0;; ++i) {
+                int pair, bh, J[2];
+                const int st = decode(i, pair, bh, J);
+                if (st == 0) break;
+                if (st == 1) continue;
+                const int Jmax = J[0] > J[1] ? J[0] : J[1];
+                mbar_wait(&ctrl->q_full, it & 1, ctx, BAR_Q);
+                mbar_wait(&ctrl->k_full[g % KV_STAGES], (g / KV_STAGES) & 1, ctx, BAR_K_FULL);
                 tc_fence_after();
-                if (J[0] > 0) issue_s(0, 0);
-                if (J[1] > 0) issue_s(1, 0);
-                umma_commit(&ctrl->k_empty[0]);
-            }
-            for (int j = 0; j < Jmax; ++j) {
-                const int sv = j % KV_STAGES;
-                const uint32_t phv = (j / KV_STAGES) & 1;
-                const int sk = (j + 1) % KV_STAGES;
-                const uint32_t phk = ((j + 1) / KV_STAGES) & 1;
-                const bool act0 = j < J[0], act1 = j < J[1];
-                const bool nxt0 = j + 1 < J[0], nxt1 = j + 1 < J[1];
-                mbar_wait(&ctrl->v_full[sv], phv, ctx, BAR_V_FULL);
-                if (nxt0 || nxt1) mbar_wait(&ctrl->k_full[sk], phk, ctx, BAR_K_FULL);
-                if (act0) {
-                    mbar_wait(&ctrl->p_full[0], j & 1, ctx, BAR_P_FULL);
-                    tc_fence_after();
-                    issue_pv(0, j);
+                if (J[0] > 0) issue_s(0, g % KV_STAGES);
+                if (J[1] > 0) issue_s(1, g % KV_STAGES);
+                umma_commit(&ctrl->k_empty[g % KV_STAGES]);
+                if (Jmax == 1) umma_commit(&ctrl->q_empty);
+                for (int j = 0; j < Jmax; ++j) {
+                    const int gv = g + j, gk = g + j + 1;
+                    const int sv = gv % KV_STAGES, sk = gk % KV_STAGES;
+                    const bool nxt0 = j + 1 < J[0], nxt1 = j + 1 < J[1];
+                    mbar_wait(&ctrl->v_full[sv], (gv / KV_STAGES) & 1, ctx, BAR_V_FULL);
+                    if (nxt0 || nxt1) mbar_wait(&ctrl->k_full[sk], (gk / KV_STAGES) & 1, ctx, BAR_K_FULL);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (j < J[t]) {
+                            // the first PV of an item overwrites O_t: the previous item's O_t must have been read out
+                            if (j == 0 && n_o[t] > 0) mbar_wait(&ctrl->o_free[t], (n_o[t] - 1) & 1, ctx, BAR_O_FREE);
+                            mbar_wait(&ctrl->p_full[t], n_s[t] & 1, ctx, BAR_P_FULL);
+                            ++n_s[t];
+                            tc_fence_after();
+                            issue_pv(t, sv, j == 0);
+                            if (j == J[t] - 1) umma_commit(&ctrl->o_final[t]);
+                        }
+                        if (t == 1) umma_commit(&ctrl->v_empty[sv]);
+                        if (j + 1 < J[t]) issue_s(t, sk);
+                    }
+                    if (nxt0 || nxt1) {
+                        umma_commit(&ctrl->k_empty[sk]);
+                        if (j + 1 == Jmax - 1) umma_commit(&ctrl->q_empty);   // the item's last S MMAs are issued
+                    }
                 }
-                if (nxt0) issue_s(0, j + 1);
-                if (act1) {
-                    mbar_wait(&ctrl->p_full[1], j & 1, ctx, BAR_P_FULL);
-                    tc_fence_after();
-                    issue_pv(1, j);
-                }
-                umma_commit(&ctrl->v_empty[sv]);
-                if (nxt1) issue_s(1, j + 1);
-                if (nxt0 || nxt1) umma_commit(&ctrl->k_empty[sk]);
+                g += Jmax;
+                n_o[0] += J[0] > 0;
+                n_o[1] += J[1] > 0;
+                ++it;
             }
-            umma_commit(&ctrl->o_final);
         }
     } else {
         setmaxnreg_inc<REGS_SOFTMAX>();
         // --------------------------------------------------------------- softmax
         const int t = (warp >> 2) - 1;
-        const int Jt = J[t];
-        if (Jt > 0) {
-            const int q = warp & 3;
-            const int r_in_tile = q * 32 + lane;
+        const int q = warp & 3;
+        const int r_in_tile = q * 32 + lane;
+        const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+        const uint32_t s_addr = tmem_base + lane_addr + t * 128;
+        const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128;
+        const float c = p.scale * 1.4426950408889634f;   // scores are kept in the log2 domain
+        uint32_t n_s = 0, n_o = 0;                       // hand-offs / items done by this query tile so far
+        for (int i = 0;; ++i) {
+            int pair, bh, J[2];
+            const int st = decode(i, pair, bh, J);
+            if (st == 0) break;
+            if (st == 1) continue;
+            const int Jt = J[t];
+            if (Jt == 0) continue;
             const int qidx = (2 * pair + t) * BQ + r_in_tile;
-            const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
-            const uint32_t s_addr = tmem_base + lane_addr + t * 128;
-            const uint32_t o_addr = tmem_base + lane_addr + 256 + t * 128;
-            const float c = p.scale * 1.4426950408889634f;   // scores are kept in the log2 domain
             float m_used = -INFINITY, l_run = 0.0f;
 
-            for (int j = 0; j < Jt; ++j) {
+            for (int j = 0; j < Jt; ++j, ++n_s) {
                 const bool edge = (j == Jt - 1);
                 const int k0 = j * BKV;
-                mbar_wait(&ctrl->s_full[t], j & 1, ctx, BAR_S_FULL);
+                mbar_wait(&ctrl->s_full[t], n_s & 1, ctx, BAR_S_FULL);
                 tc_fence_after();
 
                 uint32_t s[BKV];
@@ -277,8 +325,9 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 mbar_arrive(&ctrl->p_full[t]);
             }
 
-            // all MMAs done: normalise and store
-            mbar_wait(&ctrl->o_final, 0, ctx, BAR_O_FINAL);
+            // this tile's last PV is done: normalise and store, then hand O_t back to the MMA warp
+            mbar_wait(&ctrl->o_final[t], n_o & 1, ctx, BAR_O_FINAL);
+            ++n_o;
             tc_fence_after();
             const float inv_l = 1.0f / l_run;
             __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + ((long long)bh * p.S + qidx) * D;
@@ -299,6 +348,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     }
                 }
             }
+            tc_fence_before();
+            mbar_arrive(&ctrl->o_free[t]);
         }
     }
 
@@ -314,7 +365,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 }  // namespace
 
 cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
-                                  const AttnArgs &a, cudaStream_t stream)
+                                  const AttnArgs &a, int num_sms, cudaStream_t stream)
 {
     if (a.BH <= 0 || a.S <= 0) return cudaSuccess;
     // The in-kernel setmaxnreg split draws on threads x registers-at-launch; refuse to launch
@@ -329,10 +380,12 @@ cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK
     if (!regs_ok) return cudaErrorLaunchOutOfResources;
     const int num_q_tiles = (a.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
+    const long long num_items = (long long)((num_pairs + 1) / 2) * a.BH;   // slots: two items each
     cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attention_bf16_kernel<<<dim3((unsigned)num_pairs * (unsigned)a.BH), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
+    const unsigned grid = (unsigned)(num_items < num_sms ? num_items : num_sms);   // persistent: one CTA per SM
+    attention_bf16_kernel<<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError();
 }
 

@@ -63,6 +63,6 @@ struct AttnArgs {
     unsigned long long limit_ns;
 };
 cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
-                                  const AttnArgs &a, cudaStream_t stream);
+                                  const AttnArgs &a, int num_sms, cudaStream_t stream);
 
 }  // namespace pike
