@@ -345,6 +345,14 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_
     return d;
 }
 
+// Advancing a descriptor's start address by `bytes` (a multiple of 16 that stays inside the 256 KiB
+// window, so the 14-bit address field cannot carry into its neighbours) is one 64-bit add.  The MMA
+// issue loop runs on ONE thread, so descriptors are built once and only advanced per instruction.
+__device__ __forceinline__ constexpr uint64_t desc_advance(uint64_t desc, uint32_t bytes)
+{
+    return desc + static_cast<uint64_t>(bytes >> 4);
+}
+
 // Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulator:
 //   [4,6) D format (1 = f32)  [7,10) A format (1 = bf16)  [10,13) B format (1 = bf16)
 //   bit 15 A is MN-major   bit 16 B is MN-major   [17,23) N >> 3   [24,29) M >> 4

@@ -162,26 +162,34 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             // ---------------------------------------------------------- MMA issuer
             const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false);   // Q, K both K-major (d contiguous)
             const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major (TMEM), V MN-major
+            // Descriptors are built once; the issue loops only add constants to them (this single thread's
+            // instruction stream is on the critical path of every hand-off).
+            const uint64_t q_desc0 = make_smem_desc_sw128(smem_u32(q_s), 0, 1024);
+            const uint64_t q_desc1 = make_smem_desc_sw128(smem_u32(q_s + TILE_BYTES), 0, 1024);
+            const uint64_t k_desc0 = make_smem_desc_sw128(smem_u32(k_s), 0, 1024);
+            const uint64_t k_desc1 = make_smem_desc_sw128(smem_u32(k_s + TILE_BYTES), 0, 1024);
+            const uint64_t v_desc0 = make_smem_desc_sw128(smem_u32(v_s), SUB_BYTES, 1024);
+            const uint64_t v_desc1 = make_smem_desc_sw128(smem_u32(v_s + TILE_BYTES), SUB_BYTES, 1024);
+            static_assert(KV_STAGES == 2, "descriptor selection below assumes two K/V stages");
             // S_t = Q_t K^T (K tile in ring stage ks) into columns [t*128, t*128+128)
             auto issue_s = [&](int t, int ks) {
-                const uint32_t q_addr = smem_u32(q_s + t * TILE_BYTES);
-                const uint32_t k_addr = smem_u32(k_s + ks * TILE_BYTES);
+                const uint64_t qd = t ? q_desc1 : q_desc0;
+                const uint64_t kd = ks ? k_desc1 : k_desc0;
+                const uint32_t d_tmem = tmem_base + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * SUB_BYTES + (kk & 3) * 32;
-                    umma_ss(tmem_base + t * 128, make_smem_desc_sw128(q_addr + off, 0, 1024),
-                            make_smem_desc_sw128(k_addr + off, 0, 1024), idesc_s, kk != 0 ? 1u : 0u);
+                    umma_ss(d_tmem, desc_advance(qd, off), desc_advance(kd, off), idesc_s, kk != 0 ? 1u : 0u);
                 }
                 umma_commit(&ctrl->s_full[t]);
             };
             // O_t (+)= P_t V (V tile in ring stage vs): A = bf16 P in TMEM (8 columns per 16 keys)
             auto issue_pv = [&](int t, int vs, bool first) {
-                const uint32_t v_addr = smem_u32(v_s + vs * TILE_BYTES);
+                const uint64_t vd = vs ? v_desc1 : v_desc0;
+                const uint32_t d_tmem = tmem_base + 256 + t * 128, a_tmem = tmem_base + t * 128;
 #pragma unroll
                 for (int kk = 0; kk < BKV / 16; ++kk)
-                    umma_ts(tmem_base + 256 + t * 128, tmem_base + t * 128 + kk * 8,
-                            make_smem_desc_sw128(v_addr + kk * 2048, SUB_BYTES, 1024), idesc_o,
-                            (first && kk == 0) ? 0u : 1u);
+                    umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o, (first && kk == 0) ? 0u : 1u);
             };
             int g = 0, it = 0;                 // KV tiles / items consumed so far
             uint32_t n_s[2] = {0, 0};          // softmax hand-offs per query tile so far

@@ -129,6 +129,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ------------------------------------------------- MMA issuer (leader only)
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk);
+            const uint32_t a_addr0 = smem_u32(tiles), b_addr0 = a_addr0 + A_BYTES;
+            const uint64_t adesc0 = make_smem_desc_sw128(a_addr0, 0, 1024);
+            const uint64_t bdesc0 = p.w_is_nk ? make_smem_desc_sw128(b_addr0, 0, 1024)
+                                              : make_smem_desc_sw128(b_addr0, 64 * BK * 2, 1024);
+            const uint32_t b_kstep = p.w_is_nk ? 32u : 2048u;     // bytes per 16-k step inside a stage
             int s = 0;
             uint32_t ph = 0;
             int it = 0;
@@ -141,15 +146,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int kb = 0; kb < num_kb; ++kb) {
                     mbar_wait_cluster(&ctrl->full[s], ph, ctx, BAR_FULL);
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(tiles + (size_t)s * STAGE_BYTES);
-                    const uint32_t b_addr = a_addr + A_BYTES;
+                    // stage 0's descriptors were built once; a stage is a constant number of bytes further
+                    const uint64_t adesc = desc_advance(adesc0, (uint32_t)s * STAGE_BYTES);
+                    const uint64_t bdesc = desc_advance(bdesc0, (uint32_t)s * STAGE_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {
-                        const uint64_t adesc = make_smem_desc_sw128(a_addr + k * 32, 0, 1024);
-                        const uint64_t bdesc = p.w_is_nk ? make_smem_desc_sw128(b_addr + k * 32, 0, 1024)
-                                                         : make_smem_desc_sw128(b_addr + k * 2048, 64 * BK * 2, 1024);
-                        umma_ss_pair(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
-                    }
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_ss_pair(d_tmem, desc_advance(adesc, k * 32), desc_advance(bdesc, k * b_kstep), idesc,
+                                     (kb | k) != 0 ? 1u : 0u);
                     umma_commit_pair(&ctrl->empty[s], 0x3);
                     if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
