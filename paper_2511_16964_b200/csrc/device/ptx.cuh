@@ -363,6 +363,20 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_m
 }
 
 // ------------------------------------------------------------------ misc ----
+// One lane of a fully active warp.  Role loops are run by the WHOLE warp (so addresses, descriptors
+// and loop state stay warp-uniform and live in uniform registers) and only the single-thread
+// instructions (TMA issue, tcgen05.mma, tcgen05.commit) are predicated on this.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ void named_bar_sync(int id, int nthreads)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

@@ -158,8 +158,11 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 }
                 ++it;
             }
-        } else if (warp == 1 && lane == 0) {
+        } else if (warp == 1) {
             // ---------------------------------------------------------- MMA issuer
+            // The whole warp runs this loop (uniform control flow keeps descriptors and counters in
+            // uniform registers); one elected lane issues the MMAs and commits.
+            const bool leader = elect_one();
             const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false);   // Q, K both K-major (d contiguous)
             const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major (TMEM), V MN-major
             // Descriptors are built once; the issue loops only add constants to them (this single thread's
@@ -176,20 +179,31 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 const uint64_t qd = t ? q_desc1 : q_desc0;
                 const uint64_t kd = ks ? k_desc1 : k_desc0;
                 const uint32_t d_tmem = tmem_base + t * 128;
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * SUB_BYTES + (kk & 3) * 32;
-                    umma_ss(d_tmem, desc_advance(qd, off), desc_advance(kd, off), idesc_s, kk != 0 ? 1u : 0u);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * SUB_BYTES + (kk & 3) * 32;
+                        umma_ss(d_tmem, desc_advance(qd, off), desc_advance(kd, off), idesc_s, kk != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&ctrl->s_full[t]);
                 }
-                umma_commit(&ctrl->s_full[t]);
+                __syncwarp();
             };
             // O_t (+)= P_t V (V tile in ring stage vs): A = bf16 P in TMEM (8 columns per 16 keys)
             auto issue_pv = [&](int t, int vs, bool first) {
                 const uint64_t vd = vs ? v_desc1 : v_desc0;
                 const uint32_t d_tmem = tmem_base + 256 + t * 128, a_tmem = tmem_base + t * 128;
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < BKV / 16; ++kk)
-                    umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o, (first && kk == 0) ? 0u : 1u);
+                    for (int kk = 0; kk < BKV / 16; ++kk)
+                        umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o,
+                                (first && kk == 0) ? 0u : 1u);
+                }
+                __syncwarp();
+            };
+            auto commit = [&](uint64_t *bar) {
+                if (leader) umma_commit(bar);
+                __syncwarp();
             };
             int g = 0, it = 0;                 // KV tiles / items consumed so far
             uint32_t n_s[2] = {0, 0};          // softmax hand-offs per query tile so far
@@ -205,8 +219,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 tc_fence_after();
                 if (J[0] > 0) issue_s(0, g % KV_STAGES);
                 if (J[1] > 0) issue_s(1, g % KV_STAGES);
-                umma_commit(&ctrl->k_empty[g % KV_STAGES]);
-                if (Jmax == 1) umma_commit(&ctrl->q_empty);
+                commit(&ctrl->k_empty[g % KV_STAGES]);
+                if (Jmax == 1) commit(&ctrl->q_empty);
                 for (int j = 0; j < Jmax; ++j) {
                     const int gv = g + j, gk = g + j + 1;
                     const int sv = gv % KV_STAGES, sk = gk % KV_STAGES;
@@ -222,14 +236,14 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                             ++n_s[t];
                             tc_fence_after();
                             issue_pv(t, sv, j == 0);
-                            if (j == J[t] - 1) umma_commit(&ctrl->o_final[t]);
+                            if (j == J[t] - 1) commit(&ctrl->o_final[t]);
                         }
-                        if (t == 1) umma_commit(&ctrl->v_empty[sv]);
+                        if (t == 1) commit(&ctrl->v_empty[sv]);
                         if (j + 1 < J[t]) issue_s(t, sk);
                     }
                     if (nxt0 || nxt1) {
-                        umma_commit(&ctrl->k_empty[sk]);
-                        if (j + 1 == Jmax - 1) umma_commit(&ctrl->q_empty);   // the item's last S MMAs are issued
+                        commit(&ctrl->k_empty[sk]);
+                        if (j + 1 == Jmax - 1) commit(&ctrl->q_empty);   // the item's last S MMAs are issued
                     }
                 }
                 g += Jmax;
