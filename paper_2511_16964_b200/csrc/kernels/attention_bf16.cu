@@ -128,8 +128,9 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 
     if (warp < 4) {
         setmaxnreg_dec<REGS_WG0>();
-        if (warp == 0 && lane == 0) {
-            // -------------------------------------------------------- TMA producer
+        if (warp == 0) {
+            // -------------------------------------------------------- TMA producer (warp-uniform loop, one elected lane issues)
+            const bool leader = elect_one();
             int g = 0, it = 0;      // KV tiles and items issued so far
             for (int i = 0;; ++i) {
                 int pair, bh, J[2];
@@ -138,23 +139,32 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 if (st == 1) continue;
                 const int Jmax = J[0] > J[1] ? J[0] : J[1];
                 mbar_wait(&ctrl->q_empty, (it & 1) ^ 1, ctx, BAR_Q_EMPTY);   // the previous item's S MMAs are done
-                mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
+                if (leader) {
+                    mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
-                    tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
+                    for (int t = 0; t < 2; ++t) {
+                        tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
+                        tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
+                    }
                 }
+                __syncwarp();
                 for (int j = 0; j < Jmax; ++j, ++g) {
                     const int s = g % KV_STAGES;
                     const uint32_t ph = (g / KV_STAGES) & 1;
                     mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
-                    mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
-                    tma_load_3d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh);
-                    tma_load_3d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh);
+                    if (leader) {
+                        mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
+                        tma_load_3d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh);
+                        tma_load_3d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh);
+                    }
+                    __syncwarp();
                     mbar_wait(&ctrl->v_empty[s], ph ^ 1, ctx, BAR_V_EMPTY);
-                    mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
-                    tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
-                    tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
+                    if (leader) {
+                        mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
+                        tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
+                        tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
+                    }
+                    __syncwarp();
                 }
                 ++it;
             }

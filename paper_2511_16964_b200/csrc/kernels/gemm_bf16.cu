@@ -98,8 +98,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // -------------------- TMA producer (warp-uniform loop, one elected lane issues)
+        {
+            const bool leader = elect_one();
             int s = 0;
             uint32_t ph = 0;
             for (int t = cluster_id; t < num_tiles; t += num_clusters) {
@@ -112,22 +113,26 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     uint8_t *a_s = tiles + (size_t)s * STAGE_BYTES;
                     uint8_t *b_s = a_s + A_BYTES;
                     const uint32_t full_leader = mapa_shared(smem_u32(&ctrl->full[s]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(&ctrl->full[s], 2 * STAGE_BYTES);
-                    tma_load_2d_pair(a_s, &tmA, full_leader, kb * BK, row0);
-                    if (p.w_is_nk) {
-                        tma_load_2d_pair(b_s, &tmB, full_leader, kb * BK, col0);
-                    } else {
+                    if (leader) {
+                        if (rank == 0) mbar_arrive_expect_tx(&ctrl->full[s], 2 * STAGE_BYTES);
+                        tma_load_2d_pair(a_s, &tmA, full_leader, kb * BK, row0);
+                        if (p.w_is_nk) {
+                            tma_load_2d_pair(b_s, &tmB, full_leader, kb * BK, col0);
+                        } else {
 #pragma unroll
-                        for (int i = 0; i < BN_HALF / 64; ++i)
-                            tma_load_2d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK);
+                            for (int i = 0; i < BN_HALF / 64; ++i)
+                                tma_load_2d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK);
+                        }
                     }
+                    __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------- MMA issuer (leader only)
-        if (lane == 0 && rank == 0) {
+        // ---------- MMA issuer (leader CTA only; warp-uniform loop, one elected lane issues)
+        if (rank == 0) {
+            const bool leader = elect_one();
             const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk);
             const uint32_t a_addr0 = smem_u32(tiles), b_addr0 = a_addr0 + A_BYTES;
             const uint64_t adesc0 = make_smem_desc_sw128(a_addr0, 0, 1024);
@@ -149,14 +154,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     // stage 0's descriptors were built once; a stage is a constant number of bytes further
                     const uint64_t adesc = desc_advance(adesc0, (uint32_t)s * STAGE_BYTES);
                     const uint64_t bdesc = desc_advance(bdesc0, (uint32_t)s * STAGE_BYTES);
+                    if (leader) {
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        umma_ss_pair(d_tmem, desc_advance(adesc, k * 32), desc_advance(bdesc, k * b_kstep), idesc,
-                                     (kb | k) != 0 ? 1u : 0u);
-                    umma_commit_pair(&ctrl->empty[s], 0x3);
+                        for (int k = 0; k < BK / 16; ++k)
+                            umma_ss_pair(d_tmem, desc_advance(adesc, k * 32), desc_advance(bdesc, k * b_kstep), idesc,
+                                         (kb | k) != 0 ? 1u : 0u);
+                        umma_commit_pair(&ctrl->empty[s], 0x3);
+                    }
+                    __syncwarp();
                     if (++s == STAGES) { s = 0; ph ^= 1; }
                 }
-                umma_commit_pair(&ctrl->tmem_full[acc], 0x3);
+                if (leader) umma_commit_pair(&ctrl->tmem_full[acc], 0x3);
+                __syncwarp();
             }
         }
     } else {
