@@ -102,6 +102,13 @@ pike_status_t pike_get_last_device_status(pike_handle_t handle, pike_status_t *s
  * launched through this handle afterwards (default 2e9).  0 restores the default. */
 pike_status_t pike_set_wait_limit_ns(pike_handle_t handle, uint64_t ns);
 
+/* Test hook for the failure-detection path (no counterpart in the paper): the NEXT bf16 GEMM launched
+ * through this handle issues no operand loads, so its first wait for data runs out after the wait limit,
+ * the kernel records where, skips its remaining waits, runs to its end (the output is garbage) and
+ * pike_get_last_device_status reports PIKE_ERR_TIMEOUT.  Nothing faults, traps or hangs; the context and
+ * the handle stay usable.  Use with a small pike_set_wait_limit_ns. */
+pike_status_t pike_test_withhold_loads(pike_handle_t handle);
+
 /*
  * Per-kernel device timing, following the paper's timing protocol (Section 4.6:
  * timed runs bracketed on the device, synchronisation inside the timed region).

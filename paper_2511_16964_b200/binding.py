@@ -23,7 +23,7 @@ FLAG_W_IS_NK, FLAG_CAUSAL = 0x1, 0x2
 
 EXPORTS = (
     "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
-    "pike_set_wait_limit_ns", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
+    "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
     "pike_attention_chain", "pike_linear_softmax_noalloc",
 )
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
             lib.pike_status_string.restype = ctypes.c_char_p
             lib.pike_get_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_uint32)]
             lib.pike_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
+            lib.pike_test_withhold_loads.argtypes = [vp]
             lib.pike_profile_begin.argtypes = [vp]
             lib.pike_profile_end.argtypes = [vp, ctypes.POINTER(pike_kernel_profile_t)]
             lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
@@ -169,6 +170,12 @@ def _check(rc: int, what: str):
 def pike_set_wait_limit_ns(ns: int, device=None) -> None:
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
     _check(load_library().pike_set_wait_limit_ns(_handle(dev), int(ns)), "pike_set_wait_limit_ns")
+
+
+def pike_test_withhold_loads(device=None) -> None:
+    """Test hook: the next bf16 GEMM issues no loads, so a bounded wait runs out (see include/pike.h)."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    _check(load_library().pike_test_withhold_loads(_handle(dev)), "pike_test_withhold_loads")
 
 
 def pike_get_last_device_status(device=None) -> tuple[int, int]:

@@ -14,6 +14,7 @@ struct pike_handle_s {
     int num_sms;
     unsigned int *status;  // device, 4 words
     unsigned long long limit_ns;
+    bool withhold_next;    // pike_test_withhold_loads: applies to the next bf16 GEMM launch only
     PFN_cuTensorMapEncodeTiled_v12000 encode;
     // per-kernel device timing (pike_profile_begin / pike_profile_end)
     bool profiling;

@@ -197,6 +197,8 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.partials = partials;
     g.status = h->status;
     g.limit_ns = h->limit_ns;
+    g.test_withhold_loads = h->withhold_next ? 1 : 0;
+    h->withhold_next = false;
     TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
     return pike::launch_gemm_bf16(tmA, tmB, g, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
@@ -237,6 +239,7 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     h->num_sms = prop.multiProcessorCount;
     h->limit_ns = DEFAULT_LIMIT_NS;
     h->profiling = false;
+    h->withhold_next = false;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -318,6 +321,13 @@ pike_status_t pike_set_wait_limit_ns(pike_handle_t h, uint64_t ns)
 {
     if (h == nullptr) return PIKE_ERR_NULL;
     h->limit_ns = ns == 0 ? DEFAULT_LIMIT_NS : ns;
+    return PIKE_OK;
+}
+
+pike_status_t pike_test_withhold_loads(pike_handle_t h)
+{
+    if (h == nullptr) return PIKE_ERR_NULL;
+    h->withhold_next = true;
     return PIKE_OK;
 }
 

@@ -68,14 +68,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // releases tensor memory and returns; the host sees PIKE_ERR_TIMEOUT.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const WaitCtx &ctx, uint32_t barrier_id)
 {
-    // Fast path: poll.  The clock (a slow system register) and the abort word are only looked at
-    // every 1024 failed polls, so an ordinary hand-off never pays for them.
+    // Fast path: poll.  The abort word is looked at every 32 failed polls and the clock (a slow system
+    // register) every 1024, so an ordinary hand-off never pays for them.
     if (mbar_try_wait(bar, parity)) return true;
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3FF) == 0) {
-            if (*ctx.abort) return false;
+        if ((++spins & 0x1F) == 0 && *ctx.abort) return false;   // another thread of the CTA gave up
+        if ((spins & 0x3FF) == 0) {
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) {
                 t0 = now;
@@ -306,8 +306,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait_cluster(bar, parity)) {
-        if ((++spins & 0x3FF) == 0) {
-            if (*ctx.abort) return false;
+        if ((++spins & 0x1F) == 0 && *ctx.abort) return false;   // another thread of the CTA gave up
+        if ((spins & 0x3FF) == 0) {
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) {
                 t0 = now;

@@ -103,7 +103,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool leader = elect_one();
             int s = 0;
             uint32_t ph = 0;
-            for (int t = cluster_id; t < num_tiles; t += num_clusters) {
+            for (int t = cluster_id; t < num_tiles && !p.test_withhold_loads; t += num_clusters) {
                 int m_blk, n_blk;
                 tile_coords(t, num_m, num_n, m_blk, n_blk);
                 const int row0 = m_blk * 2 * BM + (int)rank * BM;

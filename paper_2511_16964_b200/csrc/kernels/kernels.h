@@ -36,6 +36,7 @@ struct GemmArgs {
     float2 *partials;
     unsigned int *status;
     unsigned long long limit_ns;
+    int test_withhold_loads;  // test hook: the producers issue no loads, so the first "full" wait runs out
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
 // the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
