@@ -116,14 +116,16 @@ pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, const void *ptr, ui
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
-// bf16 [BH, S, D] dense tensor -> 3-D map with a (64 x 128 x 1) box
-pike_status_t make_map_bsd(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t BH, uint64_t S, uint64_t D)
+// bf16 attention operand, element (b, h, s, d) at ptr + b*sb + h*sh + s*ss + d (strides in elements, multiples
+// of 8) -> 4-D map {128, S, H, B} with a (64 x 128 x 1 x 1) box
+pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t B, uint64_t H, uint64_t S,
+                            uint64_t sb, uint64_t sh, uint64_t ss)
 {
-    const cuuint64_t dims[3] = {D, S, BH};
-    const cuuint64_t strides[2] = {D * 2, S * D * 2};
-    const cuuint32_t box[3] = {64, 128, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+    const cuuint64_t dims[4] = {128, S, H, B};
+    const cuuint64_t strides[3] = {ss * 2, sh * 2, sb * 2};
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
@@ -510,13 +512,37 @@ static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *lik
         if (t->shape[i] != like->shape[i]) return PIKE_ERR_SHAPE;
     if (t->shape[0] * t->shape[1] * t->shape[2] == 0) return PIKE_OK;  // empty: no storage needed
     if (t->data == nullptr) return PIKE_ERR_NULL;
-    int64_t dense = 1;
-    for (int i = 3; i >= 0; --i) {
-        if (t->shape[i] > 1 && t->stride[i] != dense) return PIKE_ERR_STRIDE;
-        dense *= t->shape[i];
-    }
+    // any [B,H,S,D] view whose rows are contiguous and whose other strides keep 16-byte alignment
+    // (dense [B,H,S,D], [B,S,H,D] seen as [B,H,S,D], a slice of a packed qkv buffer, ...)
+    if (t->stride[3] != 1) return PIKE_ERR_STRIDE;
+    for (int i = 0; i < 3; ++i)
+        if (t->shape[i] > 1 && (t->stride[i] < 128 || t->stride[i] % 8 != 0)) return PIKE_ERR_STRIDE;
     if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
     return PIKE_OK;
+}
+
+// stride of dimension i, or a harmless multiple of 16 bytes when the extent is 1
+static uint64_t eff_stride(const pike_tensor_t *t, int i) { return t->shape[i] > 1 ? (uint64_t)t->stride[i] : 128u; }
+
+static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, const pike_tensor_t *k, const pike_tensor_t *v,
+                                   const pike_tensor_t *out, float scale, bool causal, cudaStream_t stream)
+{
+    const uint64_t B = q->shape[0], H = q->shape[1], S = q->shape[2];
+    CUtensorMap tmQ, tmK, tmV;
+    if (pike_status_t st = make_map_bhsd(h, &tmQ, q->data, B, H, S, eff_stride(q, 0), eff_stride(q, 1), eff_stride(q, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmK, k->data, B, H, S, eff_stride(k, 0), eff_stride(k, 1), eff_stride(k, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmV, v->data, B, H, S, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
+    pike::AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.BH = (int)(B * H); a.H = (int)H; a.S = (int)S;
+    a.scale = scale;
+    a.causal = causal ? 1 : 0;
+    a.out = out->data;
+    a.out_b = (long long)eff_stride(out, 0); a.out_h = (long long)eff_stride(out, 1); a.out_s = (long long)eff_stride(out, 2);
+    a.status = h->status;
+    a.limit_ns = h->limit_ns;
+    TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
+    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 pike_status_t pike_attention_chain_workspace(pike_handle_t h, const pike_tensor_t *q, const pike_epilogue_t *epi,
@@ -547,20 +573,7 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (BH == 0 || S == 0) return PIKE_OK;
-    CUtensorMap tmQ, tmK, tmV;
-    if (pike_status_t st = make_map_bsd(h, &tmQ, q->data, BH, S, 128)) return st;
-    if (pike_status_t st = make_map_bsd(h, &tmK, k->data, BH, S, 128)) return st;
-    if (pike_status_t st = make_map_bsd(h, &tmV, v->data, BH, S, 128)) return st;
-    pike::AttnArgs a;
-    memset(&a, 0, sizeof(a));
-    a.BH = (int)BH; a.S = (int)S;
-    a.scale = epi->scale;
-    a.causal = (epi->flags & PIKE_FLAG_CAUSAL) != 0;
-    a.out = out->data;
-    a.status = h->status;
-    a.limit_ns = h->limit_ns;
-    TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
-    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+    return run_attention(h, q, k, v, out, epi->scale, (epi->flags & PIKE_FLAG_CAUSAL) != 0, stream);
 }
 
 }  // extern "C"

@@ -143,8 +143,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
-                        tma_load_3d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh);
-                        tma_load_3d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh);
+                        tma_load_4d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh % p.H, bh / p.H);
+                        tma_load_4d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh % p.H, bh / p.H);
                     }
                 }
                 __syncwarp();
@@ -154,15 +154,15 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
                     if (leader) {
                         mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
-                        tma_load_3d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh);
-                        tma_load_3d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh);
+                        tma_load_4d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh % p.H, bh / p.H);
+                        tma_load_4d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh % p.H, bh / p.H);
                     }
                     __syncwarp();
                     mbar_wait(&ctrl->v_empty[s], ph ^ 1, ctx, BAR_V_EMPTY);
                     if (leader) {
                         mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
-                        tma_load_3d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh);
-                        tma_load_3d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh);
+                        tma_load_4d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh % p.H, bh / p.H);
+                        tma_load_4d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh % p.H, bh / p.H);
                     }
                     __syncwarp();
                 }
@@ -362,7 +362,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             ++n_o;
             tc_fence_after();
             const float inv_l = 1.0f / l_run;
-            __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + ((long long)bh * p.S + qidx) * D;
+            __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + (long long)(bh / p.H) * p.out_b +
+                                  (long long)(bh % p.H) * p.out_h + (long long)qidx * p.out_s;
 #pragma unroll 1
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t r[32];

@@ -56,10 +56,11 @@ cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partial
 
 // ---- attention ---------------------------------------------------------------------
 struct AttnArgs {
-    int BH, S;
+    int BH, H, S;   // BH = batch * H; tensor maps are 4-D {128, S, H, batch}
     float scale;
     int causal;
-    void *out;  // bf16 [BH, S, 128]
+    void *out;      // bf16; element (b, h, s, d) at out + b*out_b + h*out_h + s*out_s + d
+    long long out_b, out_h, out_s;
     unsigned int *status;
     unsigned long long limit_ns;
 };

@@ -44,6 +44,23 @@ def test_structural_properties_on_the_gpu_output():
     assert np.array_equal(got, _run(c, True))
 
 
+def test_strided_views_of_a_packed_projection_buffer():
+    """q, k, v as slices of one [B,S,3,H,D] buffer and the output written as [B,S,H,D]: no copies."""
+    import paper_2511_16964_b200 as P
+    B, H, S = 2, 3, 200
+    c = G.config5(B=B, H=H, S=S, seed=12)
+    packed = torch.empty((B, S, 3, H, 128), dtype=BF16, device="cuda")
+    for i, name in enumerate("qkv"):
+        packed[:, :, i] = dev(c[name], BF16).permute(0, 2, 1, 3)
+    q, k, v = (packed[:, :, i].permute(0, 2, 1, 3) for i in range(3))      # [B,H,S,D] views, row pitch 3*H*128
+    out_bshd = torch.zeros((B, S, H, 128), dtype=BF16, device="cuda")
+    P.pike_attention_chain(q, k, v, scale=c["scale"], causal=True, out=out_bshd.permute(0, 2, 1, 3))
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    want = O.attention(c["q"], c["k"], c["v"], scale=c["scale"], causal=True)
+    check_bf16(host64(out_bshd.permute(0, 2, 1, 3)), want, what="strided attention")
+
+
 @functools.lru_cache(maxsize=1)
 def _config5_full():
     return G.config5()
