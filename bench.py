@@ -45,6 +45,8 @@ def flops_per_config():
         "C3": 2.0 * 2 * 8192 * 4096 * 16384,
         "C4": 2.0 * 2048 * 4096 * 32000,
         "C5": 4.0 * 8 * 32 * 128 * (2048 * 2049 / 2),
+        # X1 (not part of the default step): attention block with fused projections, B8 S2048 E4096 (32 heads)
+        "X1": 2.0 * 16384 * 4096 * (3 * 4096) + 4.0 * 8 * 32 * 128 * (2048 * 2049 / 2) + 2.0 * 16384 * 4096 * 4096,
     }
 
 
@@ -143,7 +145,8 @@ def oracle_sample_text():
             f"C4 first {n['C4']} of 2048 rows; C5 first {n['C5_heads']} of 256 heads (rows and heads are independent)")
 
 
-ALL = ("C1", "C2", "C3", "C4", "C5")
+ALL = ("C1", "C2", "C3", "C4", "C5")          # the step
+EXTRA = ("X1",)                                 # further workloads, only with --only
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -164,7 +167,8 @@ def job_tflops(step_flops: float, world: int, ms_per_step: float) -> float:
 
 def make_inputs(only=ALL):
     import pike_inputs as G
-    gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5}
+    gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
+           "X1": lambda: G.attention_block(B=8, S=2048, E=4096)}
     return {k: gen[k]() for k in only}
 
 
@@ -245,14 +249,22 @@ def run_ours(args):
         wts.update(c4w=pin(c4["w"], BF16))
     if c5:
         host_act.update(c5q=pin(c5["q"], BF16), c5k=pin(c5["k"], BF16), c5v=pin(c5["v"], BF16))
+    x1 = inputs.get("X1")
+    if x1:
+        host_act.update(x1x=pin(x1["x"], BF16))
+        wts.update(x1wq=pin(x1["w_qkv"], BF16), x1bq=pin(x1["b_qkv"], BF16), x1wo=pin(x1["w_o"], BF16),
+                   x1bo=pin(x1["b_o"], BF16), x1g=pin(x1["gamma"], BF16), x1be=pin(x1["beta"], BF16))
     d = {k: v.to(device) for k, v in host_act.items()}
     d.update({k: v.to(device) for k, v in wts.items()})
     shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
-              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16)}
+              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16)}
     out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in only}
     host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
     ws0 = torch.empty(256, dtype=torch.uint8, device=device)
-    ws3 = ws4 = ws0
+    ws3 = ws4 = wsx = ws0
+    if x1:
+        wsx = torch.empty(P.pike_attention_block_workspace(d["x1x"], scale=float(x1["scale"])), dtype=torch.uint8,
+                          device=device)
     if c3:
         ws3 = torch.empty(P.pike_mlp_block_workspace(d["c3x"], d["c3w1"]), dtype=torch.uint8, device=device)
     if c4:
@@ -270,6 +282,9 @@ def run_ours(args):
                                              workspace=ws4),
         "C5": lambda: P.pike_attention_chain(d["c5q"], d["c5k"], d["c5v"], scale=float(c5["scale"]), causal=True,
                                              out=out["C5"]),
+        "X1": lambda: P.pike_attention_block(d["x1x"], d["x1g"], d["x1be"], d["x1wq"], d["x1bq"], d["x1wo"], d["x1bo"],
+                                             scale=float(x1["scale"]), causal=True, eps=x1["eps"], out=out["X1"],
+                                             workspace=wsx),
     }
     names = [n for n in chains if n in only]
 
@@ -351,6 +366,8 @@ def run_ours(args):
     peaks = load_peaks()
     gemm_launches, gemm_ms = prof["gemm_bf16"]
     gemm_flops = sum(f.get(k, 0.0) for k in ("C2", "C3", "C4"))      # the launches of the bf16 GEMM kernel
+    if "X1" in f:
+        gemm_flops += 2.0 * 16384 * 4096 * (4 * 4096)
     gemm_tflops = gemm_flops * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     # a long timed region runs under the power cap: compare with the sustained library figure
     sustained = total_ms > 500.0 or "sw_power_cap" in (clocks or {}).get("reasons", [])
@@ -362,9 +379,9 @@ def run_ours(args):
         "launches": gemm_launches, "traffic": None,
     }
 
-    eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5, names)
+    eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5 or x1, names)
     library_gemm = None if args.no_eager else library_gemm_context(torch, device, sampler.__class__(local_rank))
-    if len(only) < len(ALL):
+    if tuple(only) != ALL:
         args.no_parity = args.no_cpu_baseline = True                 # partial suites are profiling runs
     per_config = {}
     for n in names:
@@ -388,7 +405,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": ("" if len(only) == len(ALL) else "SUBSET " + ",".join(only) + " of the ") +
+        "config": {"workload": ("" if tuple(only) == ALL else "SUBSET " + ",".join(only) + " of the ") +
                                "C1-C5 chain suite (fp32 linear+GELU+LN 128x256x256; bf16 linear+SiLU+scale+residual "
                                "4096^3; bf16 MLP block 8192x4096x16384; bf16 logits+softmax 2048x4096x32000; bf16 "
                                "causal attention B8 H32 S2048 D128)",
@@ -432,7 +449,20 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
                                         + d["c3b1"], approximate="tanh") @ d["c3w2"] + d["c3b2"],
         "C4": lambda: torch.softmax(d["c4x"] @ d["c4w"], dim=-1, dtype=torch.float32),
         "C5": attn,
+        "X1": lambda: x1_eager(),
     }
+
+    def x1_eager():
+        x = d["x1x"]
+        B, S, E = x.shape
+        H = E // 128
+        z = F.layer_norm(x, (E,), d["x1g"], d["x1be"], 1e-5)
+        qkv = (z @ d["x1wq"] + d["x1bq"]).view(B, S, 3, H, 128)
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3) for i in range(3))
+        sc = (q @ k.transpose(-1, -2)) * scale
+        mask = torch.ones((S, S), dtype=torch.bool, device=x.device).tril()
+        a = (torch.softmax(sc.masked_fill(~mask, float("-inf")), dim=-1) @ v).permute(0, 2, 1, 3).reshape(B, S, E)
+        return x + a @ d["x1wo"] + d["x1bo"]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=next(iter(d.values())).device)
     res = {}
     for n in names:
@@ -519,8 +549,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--only", type=lambda v: tuple(x for x in ALL if x in v.split(",")), default=ALL,
-                    help="comma-separated subset of C1..C5 (profiling runs; the default is the whole suite)")
+    ap.add_argument("--only", type=lambda v: tuple(x for x in ALL + EXTRA if x in v.split(",")), default=ALL,
+                    help="comma-separated subset of C1..C5 and X1 (profiling runs; the default is the whole suite C1..C5)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-eager", action="store_true")
     ap.add_argument("--no-parity", action="store_true")

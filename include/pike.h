@@ -232,6 +232,30 @@ pike_status_t pike_attention_chain(pike_handle_t handle, const pike_tensor_t *q,
                                    const pike_tensor_t *v, const pike_epilogue_t *epi, pike_tensor_t *out,
                                    void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/*
+ * Pre-LayerNorm attention block with fused input and output projections (Appendix C, "VisionAttention":
+ * the largest win reported is flash attention plus fused projection kernels; "MinGPT": causal blocks):
+ *
+ *   z   = LayerNorm(x; gamma, beta, eps)                     over the last dimension E
+ *   qkv = z @ w_qkv + b_qkv                                  [B,S,3E], columns ordered q | k | v, each H heads of 128
+ *   a   = softmax(scale * q k^T [+ causal mask]) v           per (batch, head), written as [B,S,H,128]
+ *   out = x + a @ w_o + b_o                                  [B,S,E]
+ *
+ * x, out dense [B,S,E] PIKE_BF16 with E = H*128 <= 4096; w_qkv [E,3E], w_o [E,E] PIKE_BF16 (or transposed
+ * with PIKE_FLAG_W_IS_NK); gamma, beta [E], b_qkv [3E], b_o [E] BF16 or F32, each may be NULL.  epi->eps is
+ * the LayerNorm epsilon, epi->scale (> 0) the factor on q.k, PIKE_FLAG_CAUSAL the mask; act must be NONE and
+ * reduce NONE.  The attention kernel reads q, k, v as strided views of the projection output and writes its
+ * result in the layout the output projection reads, so no transpose or copy kernel runs: four kernels are
+ * enqueued (LayerNorm, GEMM+bias, attention, GEMM+bias+residual).  z, qkv and a are bf16 in the workspace
+ * (2*B*S*E*2 + B*S*3E*2 bytes, each part 256-byte aligned).
+ */
+pike_status_t pike_attention_block_workspace(pike_handle_t handle, const pike_tensor_t *x, const pike_epilogue_t *epi,
+                                             size_t *bytes);
+pike_status_t pike_attention_block(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *gamma,
+                                   const pike_tensor_t *beta, const pike_tensor_t *w_qkv, const pike_tensor_t *b_qkv,
+                                   const pike_tensor_t *w_o, const pike_tensor_t *b_o, const pike_epilogue_t *epi,
+                                   pike_tensor_t *out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

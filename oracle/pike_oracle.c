@@ -180,3 +180,47 @@ int oracle_attention_rows(const double *q_rows, const long *q_pos, long R,
     }
     return fail;
 }
+
+/* Chain: pre-LN attention block with input and output projections, for one batch element.
+ *   z   = LN(x)                       x [S,E]
+ *   qkv = z @ w_qkv + b_qkv           [S,3E], columns q | k | v, each H heads of Dh (E = H*Dh)
+ *   a[:, h*Dh:(h+1)*Dh] = attention(q_h, k_h, v_h)      per head
+ *   out = x + a @ w_o + b_o
+ * Nothing is rounded between the stages. */
+int oracle_attention_block(const double *x, const double *gamma, const double *beta, double eps,
+                           const double *w_qkv, const double *b_qkv, const double *w_o, const double *b_o,
+                           double scale, int causal, double *out, long S, long E, long H)
+{
+    const long Dh = E / H;
+    double *z = (double *)malloc(sizeof(double) * (size_t)S * (size_t)E);
+    double *qkv = (double *)malloc(sizeof(double) * (size_t)S * (size_t)E * 3);
+    double *a = (double *)malloc(sizeof(double) * (size_t)S * (size_t)E);
+    double *qh = (double *)malloc(sizeof(double) * (size_t)S * (size_t)Dh * 4);
+    long *pos = (long *)malloc(sizeof(long) * (size_t)S);
+    int rc = 1;
+    if (z && qkv && a && qh && pos) {
+        double *kh = qh + S * Dh, *vh = kh + S * Dh, *oh = vh + S * Dh;
+        memcpy(z, x, sizeof(double) * (size_t)S * (size_t)E);
+        oracle_layernorm_rows(z, S, E, gamma, beta, eps);
+        oracle_linear(z, w_qkv, b_qkv, qkv, S, E, 3 * E);
+        for (long i = 0; i < S; ++i) pos[i] = i;
+        rc = 0;
+        for (long h = 0; h < H && !rc; ++h) {
+            for (long i = 0; i < S; ++i)
+                for (long d = 0; d < Dh; ++d) {
+                    qh[i * Dh + d] = qkv[i * 3 * E + 0 * E + h * Dh + d];
+                    kh[i * Dh + d] = qkv[i * 3 * E + 1 * E + h * Dh + d];
+                    vh[i * Dh + d] = qkv[i * 3 * E + 2 * E + h * Dh + d];
+                }
+            rc = oracle_attention_rows(qh, pos, S, kh, vh, S, Dh, scale, causal, oh);
+            for (long i = 0; i < S; ++i)
+                for (long d = 0; d < Dh; ++d) a[i * E + h * Dh + d] = oh[i * Dh + d];
+        }
+        if (!rc) {
+            oracle_linear(a, w_o, b_o, out, S, E, E);
+            for (long i = 0; i < S * E; ++i) out[i] += x[i];
+        }
+    }
+    free(z); free(qkv); free(a); free(qh); free(pos);
+    return rc;
+}

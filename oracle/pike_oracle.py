@@ -59,6 +59,8 @@ def _load():
             lib.oracle_linear_epilogue.argtypes = [dp, dp, dp, dp, dp, dp, I, d, I, d, dp, L, L, L]
             lib.oracle_mlp_block.restype = I
             lib.oracle_mlp_block.argtypes = [dp, dp, dp, d, dp, dp, dp, dp, I, dp, L, L, L]
+            lib.oracle_attention_block.restype = I
+            lib.oracle_attention_block.argtypes = [dp, dp, dp, d, dp, dp, dp, dp, d, I, dp, L, L, L]
             lib.oracle_attention_rows.restype = I
             lib.oracle_attention_rows.argtypes = [dp, lp, L, dp, dp, L, L, d, I, dp]
             _lib = lib
@@ -180,4 +182,21 @@ def attention(q, k, v, *, scale, causal):
     for b in range(B):
         for h in range(H):
             out[b, h] = attention_head(q[b, h], k[b, h], v[b, h], scale=scale, causal=causal)
+    return out
+
+
+def attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, num_heads, scale, causal, eps=1e-5):
+    """x [B,S,E] -> x + attention(LN(x) @ w_qkv + b_qkv) @ w_o + b_o; qkv columns are q | k | v, heads contiguous."""
+    x = _f64(x)
+    B, S, E = x.shape
+    gamma, beta, w_qkv, b_qkv, w_o, b_o = (_f64(a) for a in (gamma, beta, w_qkv, b_qkv, w_o, b_o))
+    assert w_qkv.shape == (E, 3 * E) and w_o.shape == (E, E) and E % num_heads == 0
+    out = np.empty((B, S, E), np.float64)
+    for b in range(B):
+        xb, ob = np.ascontiguousarray(x[b]), np.empty((S, E), np.float64)
+        rc = _load().oracle_attention_block(_p(xb), _p(gamma), _p(beta), float(eps), _p(w_qkv), _p(b_qkv), _p(w_o),
+                                            _p(b_o), float(scale), int(bool(causal)), _p(ob), S, E, num_heads)
+        if rc:
+            raise MemoryError("oracle_attention_block: allocation failed")
+        out[b] = ob
     return out

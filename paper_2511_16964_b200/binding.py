@@ -25,7 +25,7 @@ EXPORTS = (
     "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
     "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
-    "pike_attention_chain", "pike_linear_softmax_noalloc",
+    "pike_attention_chain", "pike_linear_softmax_noalloc", "pike_attention_block_workspace", "pike_attention_block",
 )
 
 
@@ -89,6 +89,8 @@ def load_library() -> ctypes.CDLL:
             lib.pike_mlp_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_attention_chain_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
             lib.pike_attention_chain.argtypes = [vp, T, T, T, E, T, vp, sz, vp]
+            lib.pike_attention_block_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
+            lib.pike_attention_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             for name in EXPORTS:
                 if name != "pike_status_string":
                     getattr(lib, name).restype = ctypes.c_int
@@ -285,4 +287,27 @@ def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
     _check(load_library().pike_attention_chain(_handle(q.device), _tensor(q), _tensor(k), _tensor(v),
                                                ctypes.byref(e), _tensor(out), None, 0, _stream(stream)),
            "pike_attention_chain")
+    return out
+
+
+def pike_attention_block_workspace(x, *, scale, causal=True, eps=1e-5, w_is_nk=False) -> int:
+    e = _epilogue("none", scale, "none", eps, torch.bfloat16, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
+    n = ctypes.c_size_t(0)
+    _check(load_library().pike_attention_block_workspace(_handle(x.device), _tensor(x), ctypes.byref(e), ctypes.byref(n)),
+           "pike_attention_block_workspace")
+    return n.value
+
+
+def pike_attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, scale, causal=True, eps=1e-5, w_is_nk=False,
+                         out=None, workspace=None, stream=None):
+    """out = x + attention(LayerNorm(x) @ w_qkv + b_qkv) @ w_o + b_o for x [B,S,E]; see include/pike.h."""
+    if out is None:
+        out = torch.empty_like(x)
+    e = _epilogue("none", scale, "none", eps, torch.bfloat16, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
+    need = pike_attention_block_workspace(x, scale=scale, causal=causal, eps=eps, w_is_nk=w_is_nk)
+    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    _check(load_library().pike_attention_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta),
+                                               _tensor(w_qkv), _tensor(b_qkv), _tensor(w_o), _tensor(b_o),
+                                               ctypes.byref(e), _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
+           "pike_attention_block")
     return out

@@ -1,6 +1,7 @@
 // C ABI of the library: argument validation, TMA tensor-map encoding, kernel
 // selection and launch.  Host code only; every arithmetic step runs in the kernels.
 #include <cuda.h>
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <cudaTypedefs.h>
 #include <math.h>
@@ -574,6 +575,110 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (BH == 0 || S == 0) return PIKE_OK;
     return run_attention(h, q, k, v, out, epi->scale, (epi->flags & PIKE_FLAG_CAUSAL) != 0, stream);
+}
+
+static pike_status_t block_shape(const pike_tensor_t *x, const pike_epilogue_t *epi, int64_t &B, int64_t &S, int64_t &E)
+{
+    if (x == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = check_epilogue(epi)) return st;
+    if (x->ndim != 3) return PIKE_ERR_SHAPE;
+    if (x->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    B = x->shape[0]; S = x->shape[1]; E = x->shape[2];
+    if (B < 0 || S < 0 || E < 1) return PIKE_ERR_SHAPE;
+    if (E % 128 != 0 || E > 4096) return PIKE_ERR_UNSUPPORTED;          // heads of 128; LayerNorm row in one warp
+    if (B * S > 0x7fffffff || B * (E / 128) > 0x7fffff) return PIKE_ERR_UNSUPPORTED;
+    if (!(epi->scale > 0.0f)) return PIKE_ERR_UNSUPPORTED;
+    if (epi->act != PIKE_ACT_NONE || epi->reduce != PIKE_REDUCE_NONE) return PIKE_ERR_UNSUPPORTED;
+    return PIKE_OK;
+}
+
+static pike_status_t check_dense_bse(const pike_tensor_t *t, int64_t B, int64_t S, int64_t E)
+{
+    if (t == nullptr) return PIKE_ERR_NULL;
+    if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (t->ndim != 3 || t->shape[0] != B || t->shape[1] != S || t->shape[2] != E) return PIKE_ERR_SHAPE;
+    if (B * S == 0) return PIKE_OK;
+    if (t->data == nullptr) return PIKE_ERR_NULL;
+    if (t->stride[2] != 1 || (S > 1 && t->stride[1] != E) || (B > 1 && t->stride[0] != S * E)) return PIKE_ERR_STRIDE;
+    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
+    return PIKE_OK;
+}
+
+pike_status_t pike_attention_block_workspace(pike_handle_t h, const pike_tensor_t *x, const pike_epilogue_t *epi,
+                                             size_t *bytes)
+{
+    if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
+    int64_t B, S, E;
+    if (pike_status_t st = block_shape(x, epi, B, S, E)) return st;
+    const size_t M = (size_t)(B * S);
+    *bytes = 2 * align256(M * E * 2) + align256(M * 3 * E * 2);
+    return PIKE_OK;
+}
+
+pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *gamma,
+                                   const pike_tensor_t *beta, const pike_tensor_t *w_qkv, const pike_tensor_t *b_qkv,
+                                   const pike_tensor_t *w_o, const pike_tensor_t *b_o, const pike_epilogue_t *epi,
+                                   pike_tensor_t *out, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (h == nullptr || w_qkv == nullptr || w_o == nullptr || out == nullptr) return PIKE_ERR_NULL;
+    int64_t B, S, E;
+    if (pike_status_t st = block_shape(x, epi, B, S, E)) return st;
+    const bool nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
+    if (pike_status_t st = check_dense_bse(x, B, S, E)) return st;
+    if (pike_status_t st = check_dense_bse(out, B, S, E)) return st;
+    if (w_qkv->dtype != PIKE_BF16 || w_o->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (pike_status_t st = check_matrix(w_qkv, nk ? 3 * E : E, nk ? E : 3 * E)) return st;
+    if (pike_status_t st = check_matrix(w_o, E, E)) return st;
+    if (pike_status_t st = check_vector(gamma, E)) return st;
+    if (pike_status_t st = check_vector(beta, E)) return st;
+    if (pike_status_t st = check_vector(b_qkv, 3 * E)) return st;
+    if (pike_status_t st = check_vector(b_o, E)) return st;
+    const pike_tensor_t *ins[7] = {x, gamma, beta, w_qkv, b_qkv, w_o, b_o};
+    for (const pike_tensor_t *t : ins)
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    const int64_t M = B * S, H = E / 128;
+    const size_t z_bytes = align256((size_t)M * E * 2), qkv_bytes = align256((size_t)M * 3 * E * 2);
+    if (M > 0 && (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 ||
+                  workspace_bytes < 2 * z_bytes + qkv_bytes))
+        return PIKE_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (M == 0) return PIKE_OK;
+
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    void *z = ws, *qkv = ws + z_bytes, *att = ws + z_bytes + qkv_bytes;
+    {   // z = LayerNorm(x)
+        TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
+        if (pike::launch_layernorm_bf16(x->data, E, z, E, gamma ? gamma->data : nullptr, gamma && gamma->dtype == PIKE_F32,
+                                        beta ? beta->data : nullptr, beta && beta->dtype == PIKE_F32, epi->eps, (int)M,
+                                        (int)E, stream) != cudaSuccess)
+            return PIKE_ERR_CUDA;
+    }
+    // qkv = z @ w_qkv + b_qkv, laid out [B, S, 3, H, 128]
+    if (pike_status_t st = run_gemm(h, z, E, w_qkv, nk, M, E, 3 * E, b_qkv, nullptr, false, 0, qkv, false, 3 * E,
+                                    PIKE_ACT_NONE, 1.0f, nullptr, stream))
+        return st;
+    // attention straight on the packed buffer: q, k, v are [B,H,S,128] views of it, the result is written as [B,S,H,128]
+    pike_tensor_t view[4];
+    for (int i = 0; i < 4; ++i) {
+        view[i].dtype = PIKE_BF16;
+        view[i].ndim = 4;
+        view[i].shape[0] = B; view[i].shape[1] = H; view[i].shape[2] = S; view[i].shape[3] = 128;
+        view[i].stride[3] = 1; view[i].stride[1] = 128;
+        if (i < 3) {
+            view[i].data = static_cast<__nv_bfloat16 *>(qkv) + (int64_t)i * E;
+            view[i].stride[0] = S * 3 * E; view[i].stride[2] = 3 * E;
+        } else {
+            view[i].data = att;
+            view[i].stride[0] = S * E; view[i].stride[2] = E;
+        }
+    }
+    if (pike_status_t st = run_attention(h, &view[0], &view[1], &view[2], &view[3], epi->scale,
+                                         (epi->flags & PIKE_FLAG_CAUSAL) != 0, stream))
+        return st;
+    // out = x + att @ w_o + b_o
+    return run_gemm(h, att, E, w_o, nk, M, E, E, b_o, x->data, false, E, out->data, false, E, PIKE_ACT_NONE, 1.0f, nullptr,
+                    stream);
 }
 
 }  // extern "C"

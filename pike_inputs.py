@@ -163,3 +163,21 @@ def config5(B=8, H=32, S=2048, D=128, seed=0):
         v=normal((B, H, S, D), seed=seed, tensor_id=43, dtype="bf16"),
         scale=1.0 / np.sqrt(D),
     )
+
+
+def attention_block(B=4, S=1024, E=2048, seed=0, affine=True):
+    """bf16 pre-LN attention block with fused projections (heads of 128); weights U(+-1/sqrt(E))."""
+    a = 1.0 / np.sqrt(E)
+    if affine:
+        gamma = round_to_bf16((1.0 + uniform((E,), 0.5, seed=seed, tensor_id=56, dtype="bf16")).astype(np.float32))
+        beta = uniform((E,), 0.1, seed=seed, tensor_id=57, dtype="bf16")
+    else:
+        gamma, beta = np.ones((E,), np.float32), np.zeros((E,), np.float32)
+    return dict(
+        x=normal((B, S, E), seed=seed, tensor_id=51, dtype="bf16"),
+        w_qkv=uniform((E, 3 * E), a, seed=seed, tensor_id=52, dtype="bf16"),
+        b_qkv=uniform((3 * E,), a, seed=seed, tensor_id=53, dtype="bf16"),
+        w_o=uniform((E, E), a, seed=seed, tensor_id=54, dtype="bf16"),
+        b_o=uniform((E,), a, seed=seed, tensor_id=55, dtype="bf16"),
+        gamma=gamma, beta=beta, eps=1e-5, scale=1.0 / np.sqrt(128.0), num_heads=E // 128,
+    )

@@ -292,3 +292,31 @@ def test_mlp_block_special_cases_and_library_composition():
     got = O.mlp_block(x, g, be, w1, b1, w2, b2, act="gelu_tanh", eps=1e-5)
     np.testing.assert_allclose(got, want.numpy(), atol=1e-13)
     np.testing.assert_array_equal(O.mlp_block(x, g, be, w1, b1, w2, b2, rows=[2, 0]), got[[2, 0]])
+
+
+def test_attention_block_special_cases_and_library_composition():
+    B, S, E, H = 2, 7, 12, 3
+    Dh = E // H
+    t = lambda a: torch.from_numpy(a)
+    x = RNG.standard_normal((B, S, E)) * 1.5 + 0.3
+    g, be = RNG.standard_normal(E), RNG.standard_normal(E)
+    wq, bq = RNG.standard_normal((E, 3 * E)) / 3, RNG.standard_normal(3 * E)
+    wo, bo = RNG.standard_normal((E, E)) / 3, RNG.standard_normal(E)
+    kw = dict(num_heads=H, scale=0.4, eps=1e-5)
+    # w_o = 0 -> out = x + b_o: the residual is the un-normalised input and the bias is outside the attention
+    np.testing.assert_allclose(O.attention_block(x, g, be, wq, bq, np.zeros((E, E)), bo, causal=True, **kw), x + bo, atol=1e-15)
+    F = torch.nn.functional
+    for causal in (True, False):
+        z = F.layer_norm(t(x), (E,), t(g), t(be), eps=1e-5)
+        qkv = z @ t(wq) + t(bq)
+        q, k, v = (qkv[..., i * E:(i + 1) * E].reshape(B, S, H, Dh).permute(0, 2, 1, 3) for i in range(3))
+        a = F.scaled_dot_product_attention(q, k, v, is_causal=causal, scale=0.4).permute(0, 2, 1, 3).reshape(B, S, E)
+        want = t(x) + a @ t(wo) + t(bo)
+        got = O.attention_block(x, g, be, wq, bq, wo, bo, causal=causal, **kw)
+        np.testing.assert_allclose(got, want.numpy(), atol=1e-12)
+    # causal: the first position attends to itself only, so its output does not depend on later positions
+    x2 = x.copy()
+    x2[:, 1:] += 1.0
+    a1 = O.attention_block(x, g, be, wq, bq, wo, bo, causal=True, **kw)
+    a2 = O.attention_block(x2, g, be, wq, bq, wo, bo, causal=True, **kw)
+    np.testing.assert_allclose(a1[:, 0], a2[:, 0], atol=1e-13)
