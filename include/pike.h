@@ -144,13 +144,16 @@ pike_status_t pike_profile_end(pike_handle_t handle, pike_kernel_profile_t *out)
  *   FMA on the CUDA cores; any M, K; N <= 1024; every reduce mode.
  * bf16 path (x, w PIKE_BF16; bias/residual/gamma/beta BF16 or F32): tcgen05
  *   tensor-core GEMM with fp32 accumulation; K and N multiples of 8; out BF16 or
- *   F32 for reduce NONE; reduce SOFTMAX needs out F32 (rows are split across N
- *   tiles, partial (max, sum) pairs go to the workspace and a second kernel
- *   normalises in place); reduce LAYERNORM on this path is PIKE_ERR_UNSUPPORTED.
+ *   F32.  A row reduction on this path is split across the GEMM's 256-column
+ *   tiles: the epilogue writes the un-reduced values plus one pair per (row, tile)
+ *   to the workspace - (max, sum exp) for SOFTMAX, (mean, sum of squared
+ *   deviations) for LAYERNORM - and a second kernel combines the pairs and
+ *   finishes the rows in place.  SOFTMAX needs out F32; LAYERNORM takes BF16 or F32
+ *   (with BF16 the un-reduced values are rounded once before normalisation).
  * out must not alias any input (PIKE_ERR_UNSUPPORTED if the ranges overlap).
  *
- * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless
- * the bf16 softmax path is taken); it reads only shapes and dtypes.
+ * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless a
+ * row reduction is requested on the bf16 path); it reads only shapes and dtypes.
  */
 pike_status_t pike_linear_epilogue_workspace(pike_handle_t handle, const pike_tensor_t *x,
                                              const pike_tensor_t *w, const pike_epilogue_t *epi,

@@ -157,7 +157,6 @@ pike_status_t linear_shape(const pike_tensor_t *x, const pike_tensor_t *w, const
         if (epi->out_dtype != PIKE_F32) return PIKE_ERR_DTYPE;
     } else {
         if (s.K % 8 != 0 || s.N % 8 != 0) return PIKE_ERR_UNSUPPORTED;
-        if (epi->reduce == PIKE_REDUCE_LAYERNORM) return PIKE_ERR_UNSUPPORTED;
         if (epi->reduce == PIKE_REDUCE_SOFTMAX && epi->out_dtype != PIKE_F32) return PIKE_ERR_UNSUPPORTED;
     }
     return PIKE_OK;
@@ -173,7 +172,7 @@ size_t softmax_partials_bytes(const LinearShape &s)
 pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pike_tensor_t *w, bool w_is_nk, int64_t M,
                        int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
                        void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
-                       cudaStream_t stream)
+                       cudaStream_t stream, int partials_mode = 1)
 {
     CUtensorMap tmA, tmB;
     if (pike_status_t st = make_map_2d(h, &tmA, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
@@ -196,7 +195,7 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.residual = res_ptr; g.residual_f32 = res_f32 ? 1 : 0; g.ldr = ldr;
     g.out = out_ptr; g.out_f32 = out_f32 ? 1 : 0; g.ldo = ldo;
     g.act = act; g.scale = scale;
-    g.softmax_partials = partials != nullptr;
+    g.row_partials = partials == nullptr ? 0 : partials_mode;
     g.partials = partials;
     g.status = h->status;
     g.limit_ns = h->limit_ns;
@@ -340,7 +339,7 @@ pike_status_t pike_linear_epilogue_workspace(pike_handle_t h, const pike_tensor_
     if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
     LinearShape s;
     if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
-    *bytes = (!s.fp32_path && epi->reduce == PIKE_REDUCE_SOFTMAX) ? softmax_partials_bytes(s) : 0;
+    *bytes = (!s.fp32_path && epi->reduce != PIKE_REDUCE_NONE) ? softmax_partials_bytes(s) : 0;
     return PIKE_OK;
 }
 
@@ -390,24 +389,36 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         return pike::launch_fp32_chain(a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
 
+    // a row reduction on this path is split across the GEMM's column tiles: per-(row, tile) pairs go to the
+    // workspace, a second kernel combines them and finishes the rows in place
     float2 *partials = nullptr;
-    if (epi->reduce == PIKE_REDUCE_SOFTMAX) {
+    if (epi->reduce != PIKE_REDUCE_NONE) {
         const size_t need = softmax_partials_bytes(s);
         if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 || workspace_bytes < need)
             return PIKE_ERR_WORKSPACE;
         partials = static_cast<float2 *>(workspace);
     }
+    const bool layernorm = epi->reduce == PIKE_REDUCE_LAYERNORM;
     if (pike_status_t st = run_gemm(h, x->data, x->stride[0], w, s.w_is_nk, s.M, s.K, s.N, bias,
                                     residual ? residual->data : nullptr, residual && residual->dtype == PIKE_F32,
                                     residual ? residual->stride[0] : 0, out->data, out->dtype == PIKE_F32,
-                                    out->stride[0], (int)epi->act, epi->scale, partials, stream))
+                                    out->stride[0], (int)epi->act, epi->scale, partials, stream, layernorm ? 2 : 1))
         return st;
     if (partials != nullptr) {
         const int num_n = (int)((s.N + pike::GEMM_BN - 1) / pike::GEMM_BN);
-        TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
-        if (pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)s.M,
-                                        (int)s.N, stream) != cudaSuccess)
-            return PIKE_ERR_CUDA;
+        if (layernorm) {
+            TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
+            if (pike::launch_layernorm_finish(out->data, out->dtype == PIKE_F32, out->stride[0], partials, num_n,
+                                              pike::GEMM_BN, (int)s.M, (int)s.N, gamma ? gamma->data : nullptr,
+                                              gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
+                                              beta && beta->dtype == PIKE_F32, epi->eps, stream) != cudaSuccess)
+                return PIKE_ERR_CUDA;
+        } else {
+            TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
+            if (pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)s.M,
+                                            (int)s.N, stream) != cudaSuccess)
+                return PIKE_ERR_CUDA;
+        }
     }
     return PIKE_OK;
 }

@@ -141,7 +141,7 @@ extern "C" pike_status_t pike_linear_softmax_noalloc(pike_handle_t h, const pike
     g.bias_f32 = bias && bias->dtype == PIKE_F32;
     g.out = out->data; g.out_f32 = 1; g.ldo = out->stride[0];
     g.act = (int)epi->act; g.scale = epi->scale;
-    g.softmax_partials = 1;
+    g.row_partials = 1;
     g.partials = partials;
     g.status = h->status;
     g.limit_ns = h->limit_ns;

@@ -13,8 +13,9 @@
 //               (256x256x16) for the pair and commits to mbarriers in both CTAs
 //   warps 2..5  epilogue: tcgen05.ld this CTA's accumulator rows (thread = row, 32
 //               columns at a time), bias/activation/scale/residual in registers, 16-byte
-//               stores; optionally per-row (max, sum exp) partials for a softmax split
-//               across N tiles.  Runs under the next tile's K loop.
+//               stores; optionally per-row partials - (max, sum exp) or (mean, sum of squared
+//               deviations) - for a softmax / LayerNorm split across N tiles.  Runs under the
+//               next tile's K loop.
 // The pair halves the W traffic each SM's shared memory sees compared with a 128x256
 // single-CTA tile, which was shared-memory-bandwidth bound.  No TMA multicast is used.
 // Every mbarrier wait is bounded (see mbar_wait).
@@ -196,7 +197,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_wait(&ctrl->tmem_full[acc], aph, ctx, BAR_TMEM_FULL);
             tc_fence_after();
 
-            float run_m = -INFINITY, run_l = 0.0f;
+            // softmax: running (max, sum exp); LayerNorm: running (mean, sum of squared deviations)
+            float run_m = p.row_partials == 2 ? 0.0f : -INFINITY, run_l = 0.0f;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 const int nc = n0 + c * 32;
@@ -250,7 +252,24 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
 
-                if (p.softmax_partials) {
+                if (p.row_partials == 2) {
+                    // LayerNorm partials: this chunk's (count, mean, sum of squared deviations), merged into
+                    // the running triple of the tile row with the pairwise update (no E[x^2]-E[x]^2 cancellation)
+                    const int cnt = min(32, p.N - nc);
+                    float cs = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < cnt) cs += v[j];
+                    const float cmean = cs / (float)cnt;
+                    float cm2 = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < cnt) cm2 += (v[j] - cmean) * (v[j] - cmean);
+                    const float n_old = (float)(nc - n0), n_new = n_old + (float)cnt;
+                    const float delta = cmean - run_m;
+                    run_m += delta * ((float)cnt / n_new);             // run_m: running mean
+                    run_l += cm2 + delta * delta * (n_old * (float)cnt / n_new);   // run_l: running M2
+                } else if (p.row_partials) {
                     float cm = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
@@ -288,7 +307,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctrl->tmem_empty[acc]), 0));
 
-            if (p.softmax_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
+            if (p.row_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
         }
     }
 

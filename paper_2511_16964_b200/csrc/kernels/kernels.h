@@ -32,7 +32,8 @@ struct GemmArgs {
     void *out;             int out_f32;       long long ldo;
     int act;
     float scale;
-    int softmax_partials;  // 1: also write per-(row, n-tile) (max, sum exp) pairs
+    int row_partials;      // per-(row, n-tile) pairs for a row reduction split across tiles: 0 none,
+                           // 1 softmax (max, sum exp), 2 LayerNorm (mean, sum of squared deviations)
     float2 *partials;
     unsigned int *status;
     unsigned long long limit_ns;
@@ -53,6 +54,12 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
                                   cudaStream_t stream);
+
+// out = (v - mean)/sqrt(var + eps)*gamma + beta in place (v bf16 or f32), statistics combined from the
+// per-(row, n-tile) (mean, sum of squared deviations) pairs; tile_n = columns per tile
+cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
+                                    int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
+                                    int beta_f32, float eps, cudaStream_t stream);
 
 // ---- attention ---------------------------------------------------------------------
 struct AttnArgs {

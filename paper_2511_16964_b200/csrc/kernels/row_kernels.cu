@@ -234,7 +234,87 @@ softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__rest
     }
 }
 
+// Second half of a LayerNorm split across GEMM tiles.  One CTA per row: combine the per-tile
+// (mean_t, M2_t) pairs (tile t holds n_t = min(tile_n, N - t*tile_n) columns)
+//   mean = sum_t n_t mean_t / N,   M2 = sum_t M2_t + sum_t n_t (mean_t - mean)^2,   var = M2 / N
+// then out = (v - mean) / sqrt(var + eps) * gamma + beta in place (one read and one write of the row).
+template <bool OUT_F32>
+__global__ void __launch_bounds__(SM_THREADS)
+layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__restrict__ partials, int num_n_tiles,
+                        int tile_n, int N, const void *gamma, int gamma_f32, const void *beta, int beta_f32, float eps)
+{
+    __shared__ float red[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long row = blockIdx.x;
+    const float2 *pr = partials + row * num_n_tiles;
+    auto block_sum256 = [&](float x) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        if (lane == 0) red[warp] = x;
+        __syncthreads();
+        x = (lane < SM_THREADS / 32) ? red[lane] : 0.0f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        __syncthreads();
+        return x;
+    };
+    float a = 0.0f;
+    for (int t = tid; t < num_n_tiles; t += SM_THREADS) a += (float)min(tile_n, N - t * tile_n) * pr[t].x;
+    const float mean = block_sum256(a) / (float)N;
+    float b = 0.0f;
+    for (int t = tid; t < num_n_tiles; t += SM_THREADS) {
+        const float2 pt = pr[t];
+        const float d = pt.x - mean;
+        b += pt.y + (float)min(tile_n, N - t * tile_n) * d * d;
+    }
+    const float rstd = rsqrtf(block_sum256(b) / (float)N + eps);
+
+    if (OUT_F32) {
+        float4 *vr = reinterpret_cast<float4 *>(static_cast<float *>(vout) + row * ldv);
+        for (int i = tid; i < N / 4; i += SM_THREADS) {
+            float4 x = vr[i];
+            const int e = i * 4;
+            x.x = (x.x - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f) + load_param(beta, beta_f32, e, 0.0f);
+            x.y = (x.y - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f) + load_param(beta, beta_f32, e + 1, 0.0f);
+            x.z = (x.z - mean) * rstd * load_param(gamma, gamma_f32, e + 2, 1.0f) + load_param(beta, beta_f32, e + 2, 0.0f);
+            x.w = (x.w - mean) * rstd * load_param(gamma, gamma_f32, e + 3, 1.0f) + load_param(beta, beta_f32, e + 3, 0.0f);
+            vr[i] = x;
+        }
+    } else {
+        uint4 *vr = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(vout) + row * ldv);
+        for (int i = tid; i < N / 8; i += SM_THREADS) {
+            const uint4 x = vr[i];
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const int e = i * 8 + 2 * h;
+                const float lo = (bf16_lo(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f) +
+                                 load_param(beta, beta_f32, e, 0.0f);
+                const float hi = (bf16_hi(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f) +
+                                 load_param(beta, beta_f32, e + 1, 0.0f);
+                o[h] = pack_bf16x2(lo, hi);
+            }
+            vr[i] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
+                                    int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
+                                    int beta_f32, float eps, cudaStream_t stream)
+{
+    if (M <= 0) return cudaSuccess;
+    if (out_f32)
+        layernorm_finish_kernel<true><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
+                                                                    gamma_f32, beta, beta_f32, eps);
+    else
+        layernorm_finish_kernel<false><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
+                                                                     gamma_f32, beta, beta_f32, eps);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D,

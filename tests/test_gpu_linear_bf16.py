@@ -16,17 +16,18 @@ BF16, F32 = torch.bfloat16, torch.float32
 
 
 def _gemm(c, *, act="none", scale=1.0, bias=True, residual=True, w_is_nk=False, out_dtype=BF16, rows=None,
-          reduce="none"):
+          reduce="none", gamma=None, beta=None, eps=1e-5):
     import paper_2511_16964_b200 as P
     w = np.ascontiguousarray(c["w"].T) if w_is_nk else c["w"]
     b = c["b"] if bias else None
     r = c["r"] if residual else None
-    out = P.pike_linear_epilogue(dev(c["x"], BF16), dev(w, BF16), dev(b, BF16), dev(r, BF16), act=act, scale=scale,
-                                 reduce=reduce, out_dtype=out_dtype, w_is_nk=w_is_nk)
+    out = P.pike_linear_epilogue(dev(c["x"], BF16), dev(w, BF16), dev(b, BF16), dev(r, BF16), dev(gamma, BF16),
+                                 dev(beta, BF16), act=act, scale=scale, reduce=reduce, eps=eps, out_dtype=out_dtype,
+                                 w_is_nk=w_is_nk)
     torch.cuda.synchronize()
     st, where = P.pike_get_last_device_status()
     assert st == 0, f"device status {st} at {where:#x}"
-    want = O.linear_epilogue(c["x"], c["w"], b, r, act=act, scale=scale, reduce=reduce, rows=rows)
+    want = O.linear_epilogue(c["x"], c["w"], b, r, gamma, beta, act=act, scale=scale, reduce=reduce, eps=eps, rows=rows)
     got = host64(out)
     return (got if rows is None else got[rows]), want
 
@@ -102,13 +103,33 @@ def test_config4_full_size_sampled_rows():
     _softmax_gates(got, want, "config 4")
 
 
+@pytest.mark.parametrize("out_dtype", [BF16, F32])
+@pytest.mark.parametrize("M,K,N,w_is_nk", [(130, 64, 1000, False), (300, 192, 264, True), (5, 256, 8, False),
+                                             (512, 256, 2048, False)])
+def test_split_row_layernorm(M, K, N, w_is_nk, out_dtype):
+    c = G.config2(M=M, K=K, N=N, seed=7)
+    aff = G.config3(M=1, D=N, F=8, seed=7, affine=True)           # bf16 gamma ~ 1 +- 0.5, beta ~ +-0.1
+    got, want = _gemm(c, act="gelu_erf", scale=0.5, w_is_nk=w_is_nk, out_dtype=out_dtype, reduce="layernorm",
+                      gamma=aff["gamma"], beta=aff["beta"], eps=1e-5)
+    check_bf16(got, want, what=f"layernorm {M}x{K}x{N} {out_dtype}")
+    if out_dtype == F32:                                           # fp32 out: only fp32 statistics rounding is left
+        assert np.abs(got - want).max() < 2e-3
+
+
+def test_split_row_layernorm_with_a_large_common_offset():
+    # rows whose mean is far larger than their spread: a sum-of-squares formula would cancel, the
+    # pairwise (mean, M2) merge does not
+    c = G.config2(M=64, K=64, N=1024, seed=8)
+    c = dict(c, r=(c["r"] * 0.25 + 100.0).astype(np.float32))
+    c["r"] = G.round_to_bf16(c["r"])
+    got, want = _gemm(c, out_dtype=F32, reduce="layernorm")
+    assert np.abs(got - want).max() < 2e-2 and np.abs(got.mean(axis=1)).max() < 1e-3
+
+
 def test_rejections():
     import paper_2511_16964_b200 as P
     x = torch.zeros((16, 64), device="cuda", dtype=BF16)
     w = torch.zeros((64, 64), device="cuda", dtype=BF16)
-    with pytest.raises(P.PikeError) as e:                 # LayerNorm epilogue is not on the bf16 path
-        P.pike_linear_epilogue(x, w, reduce="layernorm")
-    assert e.value.code == 6
     with pytest.raises(P.PikeError) as e:                 # softmax needs fp32 output
         P.pike_linear_epilogue(x, w, reduce="softmax", out_dtype=BF16)
     assert e.value.code == 6
