@@ -38,7 +38,6 @@ constexpr int TMEM_COLS = NUM_ACC * BN;         // 512
 constexpr int THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr int EPI_WARPS = 4;
-constexpr int GROUP_M = 4;                      // rasterisation: 4 pair-row-blocks (1024 rows) per column sweep
 
 struct __align__(8) Ctrl {
     uint64_t full[STAGES];        // used in the leader: both CTAs' TMA bytes land here
@@ -53,12 +52,16 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_
 
 enum : uint32_t { BAR_EMPTY = 1, BAR_FULL = 2, BAR_TMEM_EMPTY = 3, BAR_TMEM_FULL = 4 };
 
-__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int &m_blk, int &n_blk)
+// Rasterisation: tiles are walked in groups of group_m pair-row-blocks, all column blocks of a group
+// before the next group, row-block fastest.  The clusters that run together therefore share a few row
+// blocks and a few column blocks (their k-slices meet in L2), and the group's rows of A stay in L2 for
+// the whole column sweep, so W is streamed from HBM once per group.
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int group_m, int &m_blk, int &n_blk)
 {
-    const int per_group = GROUP_M * num_n;
+    const int per_group = group_m * num_n;
     const int g = t / per_group;
-    const int first_m = g * GROUP_M;
-    const int gsz = min(GROUP_M, num_m - first_m);
+    const int first_m = g * group_m;
+    const int gsz = min(group_m, num_m - first_m);
     const int r = t - g * per_group;
     m_blk = first_m + r % gsz;
     n_blk = r / gsz;
@@ -106,7 +109,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t ph = 0;
             for (int t = cluster_id; t < num_tiles && !p.test_withhold_loads; t += num_clusters) {
                 int m_blk, n_blk;
-                tile_coords(t, num_m, num_n, m_blk, n_blk);
+                tile_coords(t, num_m, num_n, p.group_m, m_blk, n_blk);
                 const int row0 = m_blk * 2 * BM + (int)rank * BM;
                 const int col0 = n_blk * BN + (int)rank * BN_HALF;
                 for (int kb = 0; kb < num_kb; ++kb) {
@@ -176,7 +179,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         int it = 0;
         for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
             int m_blk, n_blk;
-            tile_coords(t, num_m, num_n, m_blk, n_blk);
+            tile_coords(t, num_m, num_n, p.group_m, m_blk, n_blk);
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int n0 = n_blk * BN;
@@ -330,6 +333,19 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
     const int num_m = (a.M + 2 * BM - 1) / (2 * BM), num_n = (a.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     if (num_tiles <= 0) return cudaSuccess;
+    // Row blocks per rasterisation group.  Measured on B200 (DRAM bytes of the two MLP GEMMs): HBM reads
+    // are lowest when the group's rows of A (group_m x 256 x K bf16) stay within about 32 MB - a quarter
+    // of the 126 MB L2, which is split over two dies and shared with the streaming W and output traffic -
+    // and never below 8 groups rows, where the clusters running together (74 = about 8 x 9 tiles) share
+    // the fewest distinct k-slices: 1169 -> 402 MB for 8192x4096x16384, 1501 -> 1322 MB for 8192x16384x4096.
+    GemmArgs args = a;
+    {
+        const long long row_block_bytes = 2ll * BM * a.K * 2;
+        long long g = (33ll << 20) / (row_block_bytes > 0 ? row_block_bytes : 1);
+        if (g < 8) g = 8;
+        if (g > num_m) g = num_m;
+        args.group_m = (int)g;
+    }
     auto go = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         if (e != cudaSuccess) return e;
@@ -353,7 +369,7 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
             max_clusters = n < num_sms / 2 ? n : num_sms / 2;
         }
         const int clusters = num_tiles < max_clusters ? num_tiles : max_clusters;
-        kern<<<dim3(2 * clusters), dim3(THREADS), SMEM_BYTES, stream>>>(tmA, tmB, a);
+        kern<<<dim3(2 * clusters), dim3(THREADS), SMEM_BYTES, stream>>>(tmA, tmB, args);
         return cudaGetLastError();
     };
     switch (a.act) {

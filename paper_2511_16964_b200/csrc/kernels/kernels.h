@@ -37,6 +37,7 @@ struct GemmArgs {
     float2 *partials;
     unsigned int *status;
     unsigned long long limit_ns;
+    int group_m;              // set by the launcher: pair-row-blocks per rasterisation group
     int test_withhold_loads;  // test hook: the producers issue no loads, so the first "full" wait runs out
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
