@@ -33,6 +33,10 @@ if ROOT not in sys.path:
 METRIC = "fused_chain_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the four gemm_bf16_kernel launches of one step
+GEMM_DRAM_BYTES_PER_STEP = 2.671e9
+# x, W, residual and output once each: C2 134.2 MB, C3 GEMM1 469.8 MB, C3 GEMM2 469.8 MB, C4 541.1 MB
+GEMM_ALGORITHMIC_BYTES_PER_STEP = 1.615e9
 
 
 # ----------------------------------------------------------------------------
@@ -376,7 +380,12 @@ def run_ours(args):
         "kernel": "gemm_bf16_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": peak, "unit": "TFLOP/s",
         "frac": (gemm_tflops / peak) if gemm_tflops else None, "peak_source": f"{peaks['source']} cuBLAS bf16, {'sustained' if sustained else 'burst'} figure",
         "frac_of_nominal_2250": (gemm_tflops / NOMINAL_BF16_TFLOPS) if gemm_tflops else None,
-        "launches": gemm_launches, "traffic": None,
+        "launches": gemm_launches,
+        # DRAM bytes of the kernel's four launches of one step, from the ncu capture summarised in
+        # profiles/gemm_bf16_kernel_dram_per_step.md (null for partial suites, and to be reset to null
+        # whenever the kernel changes after that capture)
+        "traffic": GEMM_DRAM_BYTES_PER_STEP if tuple(only) == ALL else None,
+        "traffic_unit": "bytes per step (4 launches)", "algorithmic_bytes": GEMM_ALGORITHMIC_BYTES_PER_STEP,
     }
 
     eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5 or x1, names)
