@@ -222,9 +222,9 @@ pike_status_t pike_mlp_block(pike_handle_t handle, const pike_tensor_t *x, const
  *   s[i,j]  = epi->scale * sum_d q[i,d] * k[j,d]
  *   out[i,:] = sum_j softmax_j(s[i,.])[j] * v[j,:]   (j <= i only with PIKE_FLAG_CAUSAL)
  *
- * per (batch, head).  q, k, v, out are [B,H,S,D] PIKE_BF16 views, D == 128, S_q == S_k, any
- * S >= 1.  Rows must be contiguous (stride[3] == 1); the batch, head and row strides may be anything
- * that is a multiple of 8 elements and at least 128, so dense [B,H,S,D], a [B,S,H,D] tensor viewed as
+ * per (batch, head).  q, out are [B,H,S,D] and k, v [B,H,Sk,D] PIKE_BF16 views, D == 128 or 64, any
+ * S, Sk >= 1; Sk != S (cross attention) only without PIKE_FLAG_CAUSAL.  Rows must be contiguous (stride[3] == 1); the batch, head and row strides may be anything
+ * that is a multiple of 8 elements and at least D, so dense [B,H,S,D], a [B,S,H,D] tensor viewed as
  * [B,H,S,D], or the q / k / v slices of a packed [B,S,3,H,D] projection output all work without a copy.  The score matrix lives in tensor memory and registers
  * only; probabilities are rounded to bf16 before the second GEMM.  Workspace: 0
  * bytes (the query exists for symmetry).

@@ -118,11 +118,11 @@ pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, const void *ptr, ui
 }
 
 // bf16 attention operand, element (b, h, s, d) at ptr + b*sb + h*sh + s*ss + d (strides in elements, multiples
-// of 8) -> 4-D map {128, S, H, B} with a (64 x 128 x 1 x 1) box
+// of 8) -> 4-D map {D, S, H, B} with a (64 x 128 x 1 x 1) box
 pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t B, uint64_t H, uint64_t S,
-                            uint64_t sb, uint64_t sh, uint64_t ss)
+                            uint64_t D, uint64_t sb, uint64_t sh, uint64_t ss)
 {
-    const cuuint64_t dims[4] = {128, S, H, B};
+    const cuuint64_t dims[4] = {D, S, H, B};
     const cuuint64_t strides[3] = {ss * 2, sh * 2, sb * 2};
     const cuuint32_t box[4] = {64, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -507,7 +507,7 @@ static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *e
     if (pike_status_t st = check_epilogue(epi)) return st;
     if (q->ndim != 4) return PIKE_ERR_SHAPE;
     if (q->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
-    if (q->shape[3] != 128) return PIKE_ERR_UNSUPPORTED;
+    if (q->shape[3] != 128 && q->shape[3] != 64) return PIKE_ERR_UNSUPPORTED;
     if (q->shape[0] < 0 || q->shape[1] < 0 || q->shape[2] < 0) return PIKE_ERR_SHAPE;
     if (q->shape[0] * q->shape[1] > 0x7fffff || q->shape[2] > 0x7fffff00) return PIKE_ERR_UNSUPPORTED;
     if (!(epi->scale > 0.0f)) return PIKE_ERR_UNSUPPORTED;
@@ -515,20 +515,20 @@ static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *e
     return PIKE_OK;
 }
 
-static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *like)
+static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *like, bool own_length = false)
 {
     if (t == nullptr) return PIKE_ERR_NULL;
     if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
     if (t->ndim != 4) return PIKE_ERR_SHAPE;
     for (int i = 0; i < 4; ++i)
-        if (t->shape[i] != like->shape[i]) return PIKE_ERR_SHAPE;
+        if (t->shape[i] != like->shape[i] && !(own_length && i == 2)) return PIKE_ERR_SHAPE;   // keys may have their own length
     if (t->shape[0] * t->shape[1] * t->shape[2] == 0) return PIKE_OK;  // empty: no storage needed
     if (t->data == nullptr) return PIKE_ERR_NULL;
     // any [B,H,S,D] view whose rows are contiguous and whose other strides keep 16-byte alignment
     // (dense [B,H,S,D], [B,S,H,D] seen as [B,H,S,D], a slice of a packed qkv buffer, ...)
     if (t->stride[3] != 1) return PIKE_ERR_STRIDE;
     for (int i = 0; i < 3; ++i)
-        if (t->shape[i] > 1 && (t->stride[i] < 128 || t->stride[i] % 8 != 0)) return PIKE_ERR_STRIDE;
+        if (t->shape[i] > 1 && (t->stride[i] < t->shape[3] || t->stride[i] % 8 != 0)) return PIKE_ERR_STRIDE;
     if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
     return PIKE_OK;
 }
@@ -539,14 +539,14 @@ static uint64_t eff_stride(const pike_tensor_t *t, int i) { return t->shape[i] >
 static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, const pike_tensor_t *k, const pike_tensor_t *v,
                                    const pike_tensor_t *out, float scale, bool causal, cudaStream_t stream)
 {
-    const uint64_t B = q->shape[0], H = q->shape[1], S = q->shape[2];
+    const uint64_t B = q->shape[0], H = q->shape[1], S = q->shape[2], Sk = k->shape[2], D = q->shape[3];
     CUtensorMap tmQ, tmK, tmV;
-    if (pike_status_t st = make_map_bhsd(h, &tmQ, q->data, B, H, S, eff_stride(q, 0), eff_stride(q, 1), eff_stride(q, 2))) return st;
-    if (pike_status_t st = make_map_bhsd(h, &tmK, k->data, B, H, S, eff_stride(k, 0), eff_stride(k, 1), eff_stride(k, 2))) return st;
-    if (pike_status_t st = make_map_bhsd(h, &tmV, v->data, B, H, S, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmQ, q->data, B, H, S, D, eff_stride(q, 0), eff_stride(q, 1), eff_stride(q, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmK, k->data, B, H, Sk, D, eff_stride(k, 0), eff_stride(k, 1), eff_stride(k, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmV, v->data, B, H, Sk, D, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
     pike::AttnArgs a;
     memset(&a, 0, sizeof(a));
-    a.BH = (int)(B * H); a.H = (int)H; a.S = (int)S;
+    a.BH = (int)(B * H); a.H = (int)H; a.S = (int)S; a.Sk = (int)Sk; a.D = (int)D;
     a.scale = scale;
     a.causal = causal ? 1 : 0;
     a.out = out->data;
@@ -575,9 +575,12 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     if (h == nullptr) return PIKE_ERR_NULL;
     if (pike_status_t st = attn_shape(q, epi)) return st;
     if (pike_status_t st = check_bhsd(q, q)) return st;
-    if (pike_status_t st = check_bhsd(k, q)) return st;
-    if (pike_status_t st = check_bhsd(v, q)) return st;
+    if (pike_status_t st = check_bhsd(k, q, true)) return st;
+    if (pike_status_t st = check_bhsd(v, k)) return st;
     if (pike_status_t st = check_bhsd(out, q)) return st;
+    // keys of another length (cross attention) have no causal alignment with the queries
+    if (k->shape[2] != q->shape[2] && (epi->flags & PIKE_FLAG_CAUSAL)) return PIKE_ERR_UNSUPPORTED;
+    if (k->shape[2] > 0x7fffff00) return PIKE_ERR_UNSUPPORTED;
     const pike_tensor_t *ins[3] = {q, k, v};
     for (const pike_tensor_t *t : ins)
         if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
@@ -585,6 +588,7 @@ pike_status_t pike_attention_chain(pike_handle_t h, const pike_tensor_t *q, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (BH == 0 || S == 0) return PIKE_OK;
+    if (k->shape[2] == 0) return PIKE_ERR_SHAPE;               // a softmax over no keys is undefined
     return run_attention(h, q, k, v, out, epi->scale, (epi->flags & PIKE_FLAG_CAUSAL) != 0, stream);
 }
 

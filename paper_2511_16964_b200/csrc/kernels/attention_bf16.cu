@@ -28,7 +28,6 @@
 namespace pike {
 namespace {
 
-constexpr int D = 128;
 constexpr int BQ = 128, BKV = 128;
 constexpr int KV_STAGES = 2;
 constexpr int SUB_BYTES = 128 * 64 * 2;       // one 128-row x 64-element swizzled sub-tile: 16 KiB
@@ -61,6 +60,8 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// D = head dimension (64 or 128): one or two 64-wide swizzled sub-tiles per operand tile
+template <int D>
 __global__ void __launch_bounds__(THREADS, 1)
 attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, const AttnArgs p)
@@ -75,7 +76,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_tiles = (p.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
-    const int num_kv_all = (p.S + BKV - 1) / BKV;
+    const int num_kv_all = (p.Sk + BKV - 1) / BKV;          // Sk == S unless this is cross attention
+    constexpr int OPERAND_BYTES = (D / 64) * SUB_BYTES;     // bytes of one Q / K / V tile
     // Work order.  A "slot" is one head's longest remaining pair of query tiles together with its shortest
     // (under the causal mask pair u costs 4u+3 tile-MMAs, so every slot of a head costs the same); slots
     // are dealt round-robin to the persistent CTAs.  All CTAs get equal work, CTAs running at the same
@@ -140,12 +142,13 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 const int Jmax = J[0] > J[1] ? J[0] : J[1];
                 mbar_wait(&ctrl->q_empty, (it & 1) ^ 1, ctx, BAR_Q_EMPTY);   // the previous item's S MMAs are done
                 if (leader) {
-                    mbar_arrive_expect_tx(&ctrl->q_full, 2 * TILE_BYTES);
+                    mbar_arrive_expect_tx(&ctrl->q_full, 2 * OPERAND_BYTES);
 #pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        tma_load_4d(q_s + t * TILE_BYTES, &tmQ, &ctrl->q_full, 0, (2 * pair + t) * BQ, bh % p.H, bh / p.H);
-                        tma_load_4d(q_s + t * TILE_BYTES + SUB_BYTES, &tmQ, &ctrl->q_full, 64, (2 * pair + t) * BQ, bh % p.H, bh / p.H);
-                    }
+                    for (int t = 0; t < 2; ++t)
+#pragma unroll
+                        for (int h2 = 0; h2 < D / 64; ++h2)
+                            tma_load_4d(q_s + t * TILE_BYTES + h2 * SUB_BYTES, &tmQ, &ctrl->q_full, h2 * 64,
+                                        (2 * pair + t) * BQ, bh % p.H, bh / p.H);
                 }
                 __syncwarp();
                 for (int j = 0; j < Jmax; ++j, ++g) {
@@ -153,16 +156,20 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     const uint32_t ph = (g / KV_STAGES) & 1;
                     mbar_wait(&ctrl->k_empty[s], ph ^ 1, ctx, BAR_K_EMPTY);
                     if (leader) {
-                        mbar_arrive_expect_tx(&ctrl->k_full[s], TILE_BYTES);
-                        tma_load_4d(k_s + s * TILE_BYTES, &tmK, &ctrl->k_full[s], 0, j * BKV, bh % p.H, bh / p.H);
-                        tma_load_4d(k_s + s * TILE_BYTES + SUB_BYTES, &tmK, &ctrl->k_full[s], 64, j * BKV, bh % p.H, bh / p.H);
+                        mbar_arrive_expect_tx(&ctrl->k_full[s], OPERAND_BYTES);
+#pragma unroll
+                        for (int h2 = 0; h2 < D / 64; ++h2)
+                            tma_load_4d(k_s + s * TILE_BYTES + h2 * SUB_BYTES, &tmK, &ctrl->k_full[s], h2 * 64, j * BKV,
+                                        bh % p.H, bh / p.H);
                     }
                     __syncwarp();
                     mbar_wait(&ctrl->v_empty[s], ph ^ 1, ctx, BAR_V_EMPTY);
                     if (leader) {
-                        mbar_arrive_expect_tx(&ctrl->v_full[s], TILE_BYTES);
-                        tma_load_4d(v_s + s * TILE_BYTES, &tmV, &ctrl->v_full[s], 0, j * BKV, bh % p.H, bh / p.H);
-                        tma_load_4d(v_s + s * TILE_BYTES + SUB_BYTES, &tmV, &ctrl->v_full[s], 64, j * BKV, bh % p.H, bh / p.H);
+                        mbar_arrive_expect_tx(&ctrl->v_full[s], OPERAND_BYTES);
+#pragma unroll
+                        for (int h2 = 0; h2 < D / 64; ++h2)
+                            tma_load_4d(v_s + s * TILE_BYTES + h2 * SUB_BYTES, &tmV, &ctrl->v_full[s], h2 * 64, j * BKV,
+                                        bh % p.H, bh / p.H);
                     }
                     __syncwarp();
                 }
@@ -303,7 +310,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
                     for (int i = 0; i < BKV; ++i) {
                         const int kidx = k0 + i;
-                        const bool ok = kidx < p.S && (!p.causal || kidx <= qidx);
+                        const bool ok = kidx < p.Sk && (!p.causal || kidx <= qidx);
                         const float v = ok ? __uint_as_float(s[i]) : -INFINITY;
                         s[i] = __float_as_uint(v);
                         pm[i & 7] = fmaxf(pm[i & 7], v);
@@ -395,18 +402,16 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     }
 }
 
-}  // namespace
-
-cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
-                                  const AttnArgs &a, int num_sms, cudaStream_t stream)
+template <int D>
+static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
+                                      const AttnArgs &a, int num_sms, cudaStream_t stream)
 {
-    if (a.BH <= 0 || a.S <= 0) return cudaSuccess;
     // The in-kernel setmaxnreg split draws on threads x registers-at-launch; refuse to launch
     // (rather than wait forever inside the kernel) if the compiled kernel was given fewer.
     static int regs_ok = -1;
     if (regs_ok < 0) {
         cudaFuncAttributes attr;
-        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel);
+        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel<D>);
         if (e != cudaSuccess) return e;
         regs_ok = (attr.numRegs * THREADS >= 128 * REGS_WG0 + 256 * REGS_SOFTMAX) ? 1 : 0;
     }
@@ -414,12 +419,23 @@ cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK
     const int num_q_tiles = (a.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
     const long long num_items = (long long)((num_pairs + 1) / 2) * a.BH;   // slots: two items each
-    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(num_items < num_sms ? num_items : num_sms);   // persistent: one CTA per SM
-    attention_bf16_kernel<<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
+    attention_bf16_kernel<D><<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
+                                  const AttnArgs &a, int num_sms, cudaStream_t stream)
+{
+    if (a.BH <= 0 || a.S <= 0 || a.Sk <= 0) return cudaSuccess;
+    if (a.D == 64) return launch_attention_d<64>(tmQ, tmK, tmV, a, num_sms, stream);
+    if (a.D == 128) return launch_attention_d<128>(tmQ, tmK, tmV, a, num_sms, stream);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace pike

@@ -64,7 +64,8 @@ cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const f
 
 // ---- attention ---------------------------------------------------------------------
 struct AttnArgs {
-    int BH, H, S;   // BH = batch * H; tensor maps are 4-D {128, S, H, batch}
+    int BH, H, S;   // BH = batch * H; tensor maps are 4-D {D, S or Sk, H, batch}
+    int Sk, D;      // key/value length (== S unless cross attention) and head dimension (64 or 128)
     float scale;
     int causal;
     void *out;      // bf16; element (b, h, s, d) at out + b*out_b + h*out_h + s*out_s + d

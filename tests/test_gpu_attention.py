@@ -44,6 +44,32 @@ def test_structural_properties_on_the_gpu_output():
     assert np.array_equal(got, _run(c, True))
 
 
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("B,H,S", [(1, 2, 128), (2, 3, 300), (1, 1, 1), (1, 2, 513)])
+def test_head_dimension_64(B, H, S, causal):
+    c = G.config5(B=B, H=H, S=S, D=64, seed=15)
+    got = _run(c, causal)
+    want = O.attention(c["q"], c["k"], c["v"], scale=c["scale"], causal=causal)
+    check_bf16(got, want, what=f"attention D=64 B{B} H{H} S{S} causal={causal}")
+
+
+@pytest.mark.parametrize("D", [128, 64])
+@pytest.mark.parametrize("Sq,Sk", [(128, 384), (200, 77), (1, 300), (300, 1)])
+def test_cross_attention_keys_of_another_length(Sq, Sk, D):
+    import paper_2511_16964_b200 as P
+    cq = G.config5(B=2, H=2, S=Sq, D=D, seed=16)
+    ck = G.config5(B=2, H=2, S=Sk, D=D, seed=17)
+    out = P.pike_attention_chain(dev(cq["q"], BF16), dev(ck["k"], BF16), dev(ck["v"], BF16), scale=cq["scale"],
+                                 causal=False)
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    want = O.attention(cq["q"], ck["k"], ck["v"], scale=cq["scale"], causal=False)
+    check_bf16(host64(out), want, what=f"cross attention Sq{Sq} Sk{Sk} D{D}")
+    with pytest.raises(P.PikeError) as e:                 # no causal alignment is defined for Sq != Sk
+        P.pike_attention_chain(dev(cq["q"], BF16), dev(ck["k"], BF16), dev(ck["v"], BF16), scale=1.0, causal=True)
+    assert e.value.code == 6
+
+
 def test_strided_views_of_a_packed_projection_buffer():
     """q, k, v as slices of one [B,S,3,H,D] buffer and the output written as [B,S,H,D]: no copies."""
     import paper_2511_16964_b200 as P
@@ -80,13 +106,14 @@ def test_config5_full_size_sampled_rows():
 
 def test_rejections():
     import paper_2511_16964_b200 as P
-    q = torch.zeros((1, 1, 16, 64), device="cuda", dtype=BF16)
-    with pytest.raises(P.PikeError) as e:                 # head dimension other than 128
+    q = torch.zeros((1, 1, 16, 96), device="cuda", dtype=BF16)
+    with pytest.raises(P.PikeError) as e:                 # head dimension other than 64 or 128
         P.pike_attention_chain(q, q.clone(), q.clone(), scale=1.0)
     assert e.value.code == 6
     q = torch.zeros((1, 1, 16, 128), device="cuda", dtype=BF16)
-    with pytest.raises(P.PikeError) as e:                 # k has another sequence length
-        P.pike_attention_chain(q, torch.zeros((1, 1, 32, 128), device="cuda", dtype=BF16), q.clone(), scale=1.0)
+    with pytest.raises(P.PikeError) as e:                 # v does not have k's sequence length
+        P.pike_attention_chain(q, torch.zeros((1, 1, 32, 128), device="cuda", dtype=BF16), q.clone(), scale=1.0,
+                               causal=False)
     assert e.value.code == 2
     with pytest.raises(P.PikeError) as e:                 # non-positive scale
         P.pike_attention_chain(q, q.clone(), q.clone(), scale=0.0)
