@@ -196,6 +196,26 @@ pike_status_t pike_linear_softmax_noalloc(pike_handle_t handle, const pike_tenso
                                           void *cuda_stream);
 
 /*
+ * Grouped linear + epilogue: many small GEMMs with different weights in ONE launch (Appendix C,
+ * "DeepSeek3MOESmallBatch": the per-expert loop of a mixture-of-experts layer replaced by one
+ * grouped matrix multiplication over packed expert weights):
+ *
+ *   for group g and every row r in [group_offsets[g], group_offsets[g+1]):
+ *     out[r,:] = scale * act( x[r,:] @ w[g] + bias[g,:] ) + residual[r,:]
+ *
+ * x [T,K] PIKE_BF16 with the rows of one group stored together; w [G,K,N] (or [G,N,K] with
+ * PIKE_FLAG_W_IS_NK) PIKE_BF16; bias [G,N] BF16/F32 or NULL; residual, out [T,N] (out BF16 or F32);
+ * K and N multiples of 8; reduce must be NONE.  group_offsets points to G+1 int32 values in DEVICE
+ * memory (non-decreasing, first 0, last T; empty groups are fine): the kernel reads them itself, so
+ * the host never has to wait for a router's counts.  No workspace.  Rows outside
+ * [0, group_offsets[G]) are not written.
+ */
+pike_status_t pike_grouped_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
+                                           const pike_tensor_t *bias, const pike_tensor_t *residual,
+                                           const int32_t *group_offsets, const pike_epilogue_t *epi, pike_tensor_t *out,
+                                           void *cuda_stream);
+
+/*
  * Pre-LayerNorm transformer MLP block (sub-graph fusion, Section 5.3):
  *
  *   z   = LayerNorm(x; gamma, beta, eps)            over the last dimension D

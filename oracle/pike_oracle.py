@@ -200,3 +200,21 @@ def attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, num_heads, scale,
             raise MemoryError("oracle_attention_block: allocation failed")
         out[b] = ob
     return out
+
+
+def grouped_linear_epilogue(x, w, bias, residual, offsets, *, act="none", scale=1.0):
+    """Rows offsets[g]..offsets[g+1] of x go through weight matrix w[g] ([G,K,N]) and bias row bias[g]:
+    out[r] = scale*act(x[r] @ w[g] + bias[g]) + residual[r].  Each group is one call of the linear chain."""
+    x, w = np.asarray(x), np.asarray(w)
+    offsets = [int(o) for o in offsets]
+    G, K, N = w.shape
+    assert len(offsets) == G + 1 and offsets[0] == 0 and offsets[-1] == x.shape[0]
+    out = np.zeros((x.shape[0], N), np.float64)
+    for g in range(G):
+        lo, hi = offsets[g], offsets[g + 1]
+        assert lo <= hi
+        if hi > lo:
+            out[lo:hi] = linear_epilogue(x[lo:hi], w[g], None if bias is None else np.asarray(bias)[g],
+                                         None if residual is None else np.asarray(residual)[lo:hi],
+                                         act=act, scale=scale)
+    return out

@@ -26,6 +26,7 @@ EXPORTS = (
     "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
     "pike_attention_chain", "pike_linear_softmax_noalloc", "pike_attention_block_workspace", "pike_attention_block",
+    "pike_grouped_linear_epilogue",
 )
 
 
@@ -89,6 +90,7 @@ def load_library() -> ctypes.CDLL:
             lib.pike_mlp_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_attention_chain_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
             lib.pike_attention_chain.argtypes = [vp, T, T, T, E, T, vp, sz, vp]
+            lib.pike_grouped_linear_epilogue.argtypes = [vp, T, T, T, T, vp, E, T, vp]
             lib.pike_attention_block_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
             lib.pike_attention_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             for name in EXPORTS:
@@ -310,4 +312,22 @@ def pike_attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, scale, causa
                                                _tensor(w_qkv), _tensor(b_qkv), _tensor(w_o), _tensor(b_o),
                                                ctypes.byref(e), _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
            "pike_attention_block")
+    return out
+
+
+def pike_grouped_linear_epilogue(x, w, bias, residual, group_offsets, *, act="none", scale=1.0, out_dtype=None,
+                                 w_is_nk=False, out=None, stream=None):
+    """out[r] = scale*act(x[r] @ w[g] + bias[g]) + residual[r] for rows r of group g; group_offsets is a CUDA
+    int32 tensor with G+1 entries.  See include/pike.h."""
+    if group_offsets.dtype != torch.int32 or not group_offsets.is_cuda or not group_offsets.is_contiguous():
+        raise TypeError("group_offsets must be a contiguous CUDA int32 tensor")
+    out_dtype = (out.dtype if out is not None else x.dtype) if out_dtype is None else out_dtype
+    N = w.shape[1] if w_is_nk else w.shape[2]
+    if out is None:
+        out = torch.zeros((x.shape[0], N), dtype=out_dtype, device=x.device)
+    e = _epilogue(act, scale, "none", 0.0, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
+    _check(load_library().pike_grouped_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
+                                                       _tensor(residual), ctypes.c_void_p(group_offsets.data_ptr()),
+                                                       ctypes.byref(e), _tensor(out), _stream(stream)),
+           "pike_grouped_linear_epilogue")
     return out

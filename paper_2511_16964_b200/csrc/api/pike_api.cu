@@ -132,6 +132,21 @@ pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, const void *ptr, 
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
+// bf16 weights [groups, rows, cols] (dense matrices `group_pitch` elements apart; groups == 1 for a plain
+// GEMM) -> 3-D map with a (box_cols x box_rows x 1) box, 128-byte swizzle
+pike_status_t make_map_w(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t groups, uint64_t rows,
+                         uint64_t cols, uint64_t pitch_elems, uint64_t group_pitch, uint32_t box_cols, uint32_t box_rows)
+{
+    const cuuint64_t dims[3] = {cols, rows, groups};
+    const cuuint64_t strides[2] = {pitch_elems * 2, (groups > 1 ? group_pitch : rows * pitch_elems) * 2};
+    const cuuint32_t box[3] = {box_cols, box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
 struct LinearShape {
     int64_t M, K, N;
     bool w_is_nk;
@@ -172,18 +187,21 @@ size_t softmax_partials_bytes(const LinearShape &s)
 pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pike_tensor_t *w, bool w_is_nk, int64_t M,
                        int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
                        void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
-                       cudaStream_t stream, int partials_mode = 1)
+                       cudaStream_t stream, int partials_mode = 1, const int *group_offsets = nullptr, int num_groups = 0)
 {
     CUtensorMap tmA, tmB;
     if (pike_status_t st = make_map_2d(h, &tmA, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
         return st;
+    // w is [K,N] / [N,K], or [groups,K,N] / [groups,N,K] in grouped mode (the last two dimensions are the matrix)
+    const int wd = w->ndim - 2;
+    const uint64_t groups = wd == 1 ? (uint64_t)w->shape[0] : 1, gpitch = wd == 1 ? (uint64_t)w->stride[0] : 0;
     if (w_is_nk) {
-        if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
-                                           pike::GEMM_BK, pike::GEMM_BN / 2))
+        if (pike_status_t st = make_map_w(h, &tmB, w->data, groups, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[wd],
+                                          gpitch, pike::GEMM_BK, pike::GEMM_BN / 2))
             return st;
     } else {
-        if (pike_status_t st = make_map_2d(h, &tmB, w->data, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0], 64,
-                                           pike::GEMM_BK))
+        if (pike_status_t st = make_map_w(h, &tmB, w->data, groups, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[wd],
+                                          gpitch, 64, pike::GEMM_BK))
             return st;
     }
     pike::GemmArgs g;
@@ -196,6 +214,8 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.out = out_ptr; g.out_f32 = out_f32 ? 1 : 0; g.ldo = ldo;
     g.act = act; g.scale = scale;
     g.row_partials = partials == nullptr ? 0 : partials_mode;
+    g.group_offsets = group_offsets;
+    g.num_groups = num_groups;
     g.partials = partials;
     g.status = h->status;
     g.limit_ns = h->limit_ns;
@@ -421,6 +441,51 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         }
     }
     return PIKE_OK;
+}
+
+pike_status_t pike_grouped_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
+                                           const pike_tensor_t *bias, const pike_tensor_t *residual,
+                                           const int32_t *group_offsets, const pike_epilogue_t *epi, pike_tensor_t *out,
+                                           void *cuda_stream)
+{
+    if (h == nullptr || x == nullptr || w == nullptr || out == nullptr || group_offsets == nullptr) return PIKE_ERR_NULL;
+    if (pike_status_t st = check_epilogue(epi)) return st;
+    if (x->ndim != 2 || w->ndim != 3) return PIKE_ERR_SHAPE;
+    if (x->dtype != PIKE_BF16 || w->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (epi->reduce != PIKE_REDUCE_NONE) return PIKE_ERR_UNSUPPORTED;
+    const bool nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
+    const int64_t T = x->shape[0], K = x->shape[1], G = w->shape[0];
+    const int64_t N = nk ? w->shape[1] : w->shape[2];
+    if ((nk ? w->shape[2] : w->shape[1]) != K) return PIKE_ERR_SHAPE;
+    if (T < 0 || K < 1 || N < 1 || G < 1) return PIKE_ERR_SHAPE;
+    if (T > 0x7fffffff || K > 0x7fffffff || N > 0x7fffffff || G > 65536 || K % 8 != 0 || N % 8 != 0)
+        return PIKE_ERR_UNSUPPORTED;
+    if (pike_status_t st = check_matrix(x, T, K)) return st;
+    if (pike_status_t st = check_matrix(out, T, N)) return st;
+    if (out->dtype != epi->out_dtype) return PIKE_ERR_DTYPE;
+    if (residual != nullptr)
+        if (pike_status_t st = check_matrix(residual, T, N)) return st;
+    // weights: G dense matrices, innermost stride 1, 16-byte aligned pitches
+    if (w->data == nullptr) return PIKE_ERR_NULL;
+    if (w->stride[2] != 1 || w->stride[1] < w->shape[2] || w->stride[0] < w->shape[1] * w->stride[1]) return PIKE_ERR_STRIDE;
+    if (reinterpret_cast<uintptr_t>(w->data) % 16 != 0 || (w->stride[1] * 2) % 16 != 0 || (w->stride[0] * 2) % 16 != 0)
+        return PIKE_ERR_ALIGNMENT;
+    if (bias != nullptr) {
+        if (bias->data == nullptr) return PIKE_ERR_NULL;
+        if (!valid_dtype(bias->dtype)) return PIKE_ERR_DTYPE;
+        if (bias->ndim != 2 || bias->shape[0] != G || bias->shape[1] != N) return PIKE_ERR_SHAPE;
+        if (bias->stride[1] != 1 || bias->stride[0] != N) return PIKE_ERR_STRIDE;
+    }
+    const pike_tensor_t *ins[4] = {x, w, bias, residual};
+    for (const pike_tensor_t *t : ins)
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (T == 0) return PIKE_OK;
+    return run_gemm(h, x->data, x->stride[0], w, nk, T, K, N, bias, residual ? residual->data : nullptr,
+                    residual && residual->dtype == PIKE_F32, residual ? residual->stride[0] : 0, out->data,
+                    out->dtype == PIKE_F32, out->stride[0], (int)epi->act, epi->scale, nullptr, stream, 0, group_offsets,
+                    (int)G);
 }
 
 static pike_status_t mlp_shape(const pike_tensor_t *x, const pike_tensor_t *w1, const pike_epilogue_t *epi, int64_t &M,

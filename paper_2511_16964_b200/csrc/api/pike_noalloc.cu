@@ -59,14 +59,15 @@ pike_status_t check_bf16_matrix(const pike_tensor_t *t, int64_t rows, int64_t co
     return PIKE_OK;
 }
 
+// rank 2 for the activations, rank 3 (one matrix) for the weights, as the GEMM kernel expects
 pike_status_t encode_2d(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
-                        uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
+                        uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows, int rank = 2)
 {
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {pitch_elems * 2};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+    const cuuint64_t dims[3] = {cols, rows, 1};
+    const cuuint64_t strides[2] = {pitch_elems * 2, rows * pitch_elems * 2};
+    const cuuint32_t box[3] = {box_cols, box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
@@ -129,9 +130,9 @@ extern "C" pike_status_t pike_linear_softmax_noalloc(pike_handle_t h, const pike
                                      pike::GEMM_BM))
         return st;
     if (pike_status_t st = nk ? encode_2d(h, &tmB, w->data, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
-                                          pike::GEMM_BK, pike::GEMM_BN / 2)
+                                          pike::GEMM_BK, pike::GEMM_BN / 2, 3)
                               : encode_2d(h, &tmB, w->data, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0], 64,
-                                          pike::GEMM_BK))
+                                          pike::GEMM_BK, 3))
         return st;
     pike::GemmArgs g;
     memset(&g, 0, sizeof(g));

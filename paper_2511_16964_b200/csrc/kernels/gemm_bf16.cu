@@ -67,6 +67,31 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int gro
     n_blk = r / gsz;
 }
 
+// Rows covered by the pair-row-tile with linear index m_lin.  Plain mode: 256 consecutive rows of A.
+// Grouped mode: row tiles are counted group by group (a group's last tile may be partly empty), the
+// tile's rows stop at the end of its group, and `group` selects the weight matrix and bias row.
+struct RowTile { int row0, row_end, group; };
+__device__ __forceinline__ RowTile row_tile(const GemmArgs &p, int m_lin)
+{
+    if (p.group_offsets == nullptr) return RowTile{m_lin * 2 * BM, p.M, 0};
+    int first = 0;
+    for (int e = 0; e < p.num_groups; ++e) {
+        const int lo = __ldg(p.group_offsets + e), hi = __ldg(p.group_offsets + e + 1);
+        const int tiles = (hi - lo + 2 * BM - 1) / (2 * BM);
+        if (m_lin < first + tiles) return RowTile{lo + (m_lin - first) * 2 * BM, hi, e};
+        first += tiles;
+    }
+    return RowTile{p.M, p.M, 0};   // past the end: nothing to store
+}
+__device__ __forceinline__ int count_row_tiles(const GemmArgs &p)
+{
+    if (p.group_offsets == nullptr) return (p.M + 2 * BM - 1) / (2 * BM);
+    int n = 0;
+    for (int e = 0; e < p.num_groups; ++e)
+        n += (__ldg(p.group_offsets + e + 1) - __ldg(p.group_offsets + e) + 2 * BM - 1) / (2 * BM);
+    return n;
+}
+
 template <int ACT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs p)
@@ -78,7 +103,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();           // 0 = leader
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
-    const int num_m = (p.M + 2 * BM - 1) / (2 * BM), num_n = (p.N + BN - 1) / BN;
+    const int num_m = count_row_tiles(p), num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
 
@@ -110,7 +135,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int t = cluster_id; t < num_tiles && !p.test_withhold_loads; t += num_clusters) {
                 int m_blk, n_blk;
                 tile_coords(t, num_m, num_n, p.group_m, m_blk, n_blk);
-                const int row0 = m_blk * 2 * BM + (int)rank * BM;
+                const RowTile rt = row_tile(p, m_blk);
+                const int row0 = rt.row0 + (int)rank * BM;
                 const int col0 = n_blk * BN + (int)rank * BN_HALF;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     mbar_wait(&ctrl->empty[s], ph ^ 1, ctx, BAR_EMPTY);
@@ -121,11 +147,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (rank == 0) mbar_arrive_expect_tx(&ctrl->full[s], 2 * STAGE_BYTES);
                         tma_load_2d_pair(a_s, &tmA, full_leader, kb * BK, row0);
                         if (p.w_is_nk) {
-                            tma_load_2d_pair(b_s, &tmB, full_leader, kb * BK, col0);
+                            tma_load_3d_pair(b_s, &tmB, full_leader, kb * BK, col0, rt.group);
                         } else {
 #pragma unroll
                             for (int i = 0; i < BN_HALF / 64; ++i)
-                                tma_load_2d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK);
+                                tma_load_3d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK, rt.group);
                         }
                     }
                     __syncwarp();
@@ -183,16 +209,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int n0 = n_blk * BN;
-            const int row = m_blk * 2 * BM + (int)rank * BM + q * 32 + lane;
-            const bool row_ok = row < p.M;
+            const RowTile rt = row_tile(p, m_blk);
+            const int row = rt.row0 + (int)rank * BM + q * 32 + lane;
+            const bool row_ok = row < rt.row_end;
+            const long long bias0 = (long long)rt.group * p.N + n0;    // bias is [num_groups, N] in grouped mode
 
             // stage the tile's bias as fp32
             named_bar_sync(1, EPI_THREADS);
             for (int i = et; i < BN; i += EPI_THREADS) {
                 float b = 0.0f;
                 if (p.bias != nullptr && n0 + i < p.N)
-                    b = p.bias_f32 ? static_cast<const float *>(p.bias)[n0 + i]
-                                   : __bfloat162float(static_cast<const __nv_bfloat16 *>(p.bias)[n0 + i]);
+                    b = p.bias_f32 ? static_cast<const float *>(p.bias)[bias0 + i]
+                                   : __bfloat162float(static_cast<const __nv_bfloat16 *>(p.bias)[bias0 + i]);
                 ctrl->bias[i] = b;
             }
             named_bar_sync(1, EPI_THREADS);
@@ -330,9 +358,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
                              cudaStream_t stream)
 {
-    const int num_m = (a.M + 2 * BM - 1) / (2 * BM), num_n = (a.N + BN - 1) / BN;
+    // grouped mode: the device counts the row tiles itself; this is the host's upper bound for sizing
+    const int num_m = (a.M + 2 * BM - 1) / (2 * BM) + (a.group_offsets != nullptr ? a.num_groups : 0);
+    const int num_n = (a.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
-    if (num_tiles <= 0) return cudaSuccess;
+    if (num_tiles <= 0 || a.M <= 0) return cudaSuccess;
     // Row blocks per rasterisation group.  Measured on B200 (DRAM bytes of the two MLP GEMMs): HBM reads
     // are lowest when the group's rows of A (group_m x 256 x K bf16) stay within about 32 MB - a quarter
     // of the 126 MB L2, which is split over two dies and shared with the streaming W and output traffic -

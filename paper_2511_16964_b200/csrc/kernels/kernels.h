@@ -37,6 +37,10 @@ struct GemmArgs {
     float2 *partials;
     unsigned int *status;
     unsigned long long limit_ns;
+    // grouped mode (group_offsets != nullptr): rows [group_offsets[e], group_offsets[e+1]) of A use weight
+    // matrix e (third coordinate of the W tensor map) and bias row e; M is the total row count
+    const int *group_offsets;  // device, num_groups + 1 ints
+    int num_groups;
     int group_m;              // set by the launcher: pair-row-blocks per rasterisation group
     int test_withhold_loads;  // test hook: the producers issue no loads, so the first "full" wait runs out
 };

@@ -181,3 +181,23 @@ def attention_block(B=4, S=1024, E=2048, seed=0, affine=True):
         b_o=uniform((E,), a, seed=seed, tensor_id=55, dtype="bf16"),
         gamma=gamma, beta=beta, eps=1e-5, scale=1.0 / np.sqrt(128.0), num_heads=E // 128,
     )
+
+
+def grouped_linear(T=16384, K=2048, N=4096, G=32, seed=0):
+    """bf16 mixture-of-experts style grouped linear: T rows split over G groups of uneven size (one group is
+    empty, sizes are not multiples of the tile), weights U(+-1/sqrt(K))."""
+    a = 1.0 / np.sqrt(K)
+    # group sizes: seeded uniform weights, one group forced empty, remainder to the last group
+    wts = uniform((G,), 0.5, seed=seed, tensor_id=66, dtype="f32").astype(np.float64) + 0.6
+    if G > 2:
+        wts[G // 2] = 0.0
+    sizes = np.floor(wts / wts.sum() * T).astype(np.int64)
+    sizes[-1] += T - sizes.sum()
+    offsets = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    return dict(
+        x=normal((T, K), seed=seed, tensor_id=61, dtype="bf16"),
+        w=uniform((G, K, N), a, seed=seed, tensor_id=62, dtype="bf16"),
+        b=uniform((G, N), a, seed=seed, tensor_id=63, dtype="bf16"),
+        r=normal((T, N), seed=seed, tensor_id=64, dtype="bf16"),
+        offsets=offsets,
+    )

@@ -320,3 +320,21 @@ def test_attention_block_special_cases_and_library_composition():
     a1 = O.attention_block(x, g, be, wq, bq, wo, bo, causal=True, **kw)
     a2 = O.attention_block(x2, g, be, wq, bq, wo, bo, causal=True, **kw)
     np.testing.assert_allclose(a1[:, 0], a2[:, 0], atol=1e-13)
+
+
+def test_grouped_linear_matches_per_group_library_matmul_and_single_group_case():
+    T, K, N, Gn = 11, 6, 5, 4
+    x, w = RNG.standard_normal((T, K)), RNG.standard_normal((Gn, K, N))
+    b, r = RNG.standard_normal((Gn, N)), RNG.standard_normal((T, N))
+    offsets = [0, 3, 3, 9, 11]                                   # one empty group
+    got = O.grouped_linear_epilogue(x, w, b, r, offsets, act="silu", scale=0.5)
+    for g in range(Gn):
+        lo, hi = offsets[g], offsets[g + 1]
+        y = torch.from_numpy(x[lo:hi]) @ torch.from_numpy(w[g]) + torch.from_numpy(b[g])
+        want = 0.5 * torch.nn.functional.silu(y) + torch.from_numpy(r[lo:hi])
+        np.testing.assert_allclose(got[lo:hi], want.numpy(), atol=1e-13)
+    # a row moved to another group changes (only) that row
+    got2 = O.grouped_linear_epilogue(x, w, b, r, [0, 2, 3, 9, 11], act="silu", scale=0.5)
+    assert np.abs(got2[2] - got[2]).max() > 1e-3 and np.array_equal(np.delete(got2, 2, 0), np.delete(got, 2, 0))
+    one = O.grouped_linear_epilogue(x, w[:1], b[:1], r, [0, T], act="gelu_tanh")
+    np.testing.assert_array_equal(one, O.linear_epilogue(x, w[0], b[0], r, act="gelu_tanh"))
