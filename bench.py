@@ -51,6 +51,8 @@ def flops_per_config():
         "C5": 4.0 * 8 * 32 * 128 * (2048 * 2049 / 2),
         # X1 (not part of the default step): attention block with fused projections, B8 S2048 E4096 (32 heads)
         "X1": 2.0 * 16384 * 4096 * (3 * 4096) + 4.0 * 8 * 32 * 128 * (2048 * 2049 / 2) + 2.0 * 16384 * 4096 * 4096,
+        # X2 (not part of the default step): grouped linear + SiLU, 16384 rows over 32 weight matrices 2048 x 4096
+        "X2": 2.0 * 16384 * 2048 * 4096,
     }
 
 
@@ -150,7 +152,7 @@ def oracle_sample_text():
 
 
 ALL = ("C1", "C2", "C3", "C4", "C5")          # the step
-EXTRA = ("X1",)                                 # further workloads, only with --only
+EXTRA = ("X1", "X2")                         # further workloads, only with --only
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -172,7 +174,7 @@ def job_tflops(step_flops: float, world: int, ms_per_step: float) -> float:
 def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
-           "X1": lambda: G.attention_block(B=8, S=2048, E=4096)}
+           "X1": lambda: G.attention_block(B=8, S=2048, E=4096), "X2": G.grouped_linear}
     return {k: gen[k]() for k in only}
 
 
@@ -258,10 +260,14 @@ def run_ours(args):
         host_act.update(x1x=pin(x1["x"], BF16))
         wts.update(x1wq=pin(x1["w_qkv"], BF16), x1bq=pin(x1["b_qkv"], BF16), x1wo=pin(x1["w_o"], BF16),
                    x1bo=pin(x1["b_o"], BF16), x1g=pin(x1["gamma"], BF16), x1be=pin(x1["beta"], BF16))
+    x2 = inputs.get("X2")
+    if x2:
+        host_act.update(x2x=pin(x2["x"], BF16))
+        wts.update(x2w=pin(x2["w"], BF16), x2b=pin(x2["b"], BF16))
     d = {k: v.to(device) for k, v in host_act.items()}
     d.update({k: v.to(device) for k, v in wts.items()})
     shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
-              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16)}
+              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16), "X2": ((16384, 4096), BF16)}
     out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in only}
     host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
     ws0 = torch.empty(256, dtype=torch.uint8, device=device)
@@ -275,6 +281,7 @@ def run_ours(args):
         ws4 = torch.empty(P.pike_linear_epilogue_workspace(d["c4x"], d["c4w"], reduce="softmax", out_dtype=F32),
                           dtype=torch.uint8, device=device)
 
+    x2off = torch.from_numpy(x2["offsets"]).to(device) if x2 else None
     chains = {
         "C1": lambda: P.pike_linear_epilogue(d["c1x"], d["c1w"], d["c1b"], None, d["c1g"], d["c1be"], act="gelu_erf",
                                              reduce="layernorm", eps=c1["eps"], out=out["C1"], workspace=ws0),
@@ -289,6 +296,8 @@ def run_ours(args):
         "X1": lambda: P.pike_attention_block(d["x1x"], d["x1g"], d["x1be"], d["x1wq"], d["x1bq"], d["x1wo"], d["x1bo"],
                                              scale=float(x1["scale"]), causal=True, eps=x1["eps"], out=out["X1"],
                                              workspace=wsx),
+        "X2": lambda: P.pike_grouped_linear_epilogue(d["x2x"], d["x2w"], d["x2b"], None, x2off, act="silu",
+                                                     out=out["X2"]),
     }
     names = [n for n in chains if n in only]
 
@@ -372,6 +381,7 @@ def run_ours(args):
     gemm_flops = sum(f.get(k, 0.0) for k in ("C2", "C3", "C4"))      # the launches of the bf16 GEMM kernel
     if "X1" in f:
         gemm_flops += 2.0 * 16384 * 4096 * (4 * 4096)
+    gemm_flops += f.get("X2", 0.0)
     gemm_tflops = gemm_flops * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     # a long timed region runs under the power cap: compare with the sustained library figure
     sustained = total_ms > 500.0 or "sw_power_cap" in (clocks or {}).get("reasons", [])
@@ -388,6 +398,8 @@ def run_ours(args):
         "traffic_unit": "bytes per step (4 launches)", "algorithmic_bytes": GEMM_ALGORITHMIC_BYTES_PER_STEP,
     }
 
+    if x2:
+        d["x2off_host"] = [int(o) for o in x2["offsets"]]
     eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5 or x1, names)
     library_gemm = None if args.no_eager else library_gemm_context(torch, device, sampler.__class__(local_rank))
     if tuple(only) != ALL:
@@ -459,7 +471,14 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         "C4": lambda: torch.softmax(d["c4x"] @ d["c4w"], dim=-1, dtype=torch.float32),
         "C5": attn,
         "X1": lambda: x1_eager(),
+        "X2": lambda: x2_eager(),
     }
+
+    def x2_eager():     # the per-expert loop the grouped kernel replaces
+        off = d["x2off_host"]
+        outs = [F.silu(d["x2x"][off[g]:off[g + 1]] @ d["x2w"][g] + d["x2b"][g]) for g in range(len(off) - 1)
+                if off[g + 1] > off[g]]
+        return torch.cat(outs)
 
     def x1_eager():
         x = d["x1x"]
@@ -472,7 +491,7 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         mask = torch.ones((S, S), dtype=torch.bool, device=x.device).tril()
         a = (torch.softmax(sc.masked_fill(~mask, float("-inf")), dim=-1) @ v).permute(0, 2, 1, 3).reshape(B, S, E)
         return x + a @ d["x1wo"] + d["x1bo"]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=next(iter(d.values())).device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=next(v for v in d.values() if hasattr(v, "device")).device)
     res = {}
     for n in names:
         ops[n]()
