@@ -52,7 +52,13 @@ typedef enum {
     PIKE_ERR_TIMEOUT = 10     /* device status only: a bounded in-kernel wait ran out    */
 } pike_status_t;
 
-typedef enum { PIKE_F32 = 0, PIKE_BF16 = 1 } pike_dtype_t;
+/* Element types.  PIKE_BF16 and PIKE_F16 (IEEE binary16, the reduced precision the paper's winning
+ * solutions use: Section 5.3 and Appendix C, "VisionAttention", "MinGPT") select the same tensor-core
+ * kernels with fp32 accumulation; wherever the text below says "16-bit" either may be used, but one
+ * call never mixes the two: every 16-bit tensor of a call has the dtype of x (or q), anything else
+ * is PIKE_ERR_DTYPE.  F16 has the narrower range (largest finite value 65504): values that overflow
+ * it on output become infinities, as in any f16 computation. */
+typedef enum { PIKE_F32 = 0, PIKE_BF16 = 1, PIKE_F16 = 2 } pike_dtype_t;
 
 /* A view of caller-owned device memory.  stride[] is in elements. */
 typedef struct {
@@ -142,18 +148,18 @@ pike_status_t pike_profile_end(pike_handle_t handle, pike_kernel_profile_t *out)
  *
  * fp32 path (x, w, out all PIKE_F32; bias/residual/gamma/beta F32): true fp32
  *   FMA on the CUDA cores; any M, K; N <= 1024; every reduce mode.
- * bf16 path (x, w PIKE_BF16; bias/residual/gamma/beta BF16 or F32): tcgen05
- *   tensor-core GEMM with fp32 accumulation; K and N multiples of 8; out BF16 or
- *   F32.  A row reduction on this path is split across the GEMM's 256-column
+ * 16-bit path (x, w both PIKE_BF16 or both PIKE_F16; bias/residual/gamma/beta of
+ *   that type or F32): tcgen05 tensor-core GEMM with fp32 accumulation; K and N
+ *   multiples of 8; out of that 16-bit type or F32.  A row reduction on this path is split across the GEMM's 256-column
  *   tiles: the epilogue writes the un-reduced values plus one pair per (row, tile)
  *   to the workspace - (max, sum exp) for SOFTMAX, (mean, sum of squared
  *   deviations) for LAYERNORM - and a second kernel combines the pairs and
- *   finishes the rows in place.  SOFTMAX needs out F32; LAYERNORM takes BF16 or F32
- *   (with BF16 the un-reduced values are rounded once before normalisation).
+ *   finishes the rows in place.  SOFTMAX needs out F32; LAYERNORM takes 16-bit or F32
+ *   (with a 16-bit out the un-reduced values are rounded once before normalisation).
  * out must not alias any input (PIKE_ERR_UNSUPPORTED if the ranges overlap).
  *
  * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless a
- * row reduction is requested on the bf16 path); it reads only shapes and dtypes.
+ * row reduction is requested on the 16-bit path); it reads only shapes and dtypes.
  */
 pike_status_t pike_linear_epilogue_workspace(pike_handle_t handle, const pike_tensor_t *x,
                                              const pike_tensor_t *w, const pike_epilogue_t *epi,
@@ -203,8 +209,8 @@ pike_status_t pike_linear_softmax_noalloc(pike_handle_t handle, const pike_tenso
  *   for group g and every row r in [group_offsets[g], group_offsets[g+1]):
  *     out[r,:] = scale * act( x[r,:] @ w[g] + bias[g,:] ) + residual[r,:]
  *
- * x [T,K] PIKE_BF16 with the rows of one group stored together; w [G,K,N] (or [G,N,K] with
- * PIKE_FLAG_W_IS_NK) PIKE_BF16; bias [G,N] BF16/F32 or NULL; residual, out [T,N] (out BF16 or F32);
+ * x [T,K] 16-bit (BF16 or F16) with the rows of one group stored together; w [G,K,N] (or [G,N,K] with
+ * PIKE_FLAG_W_IS_NK) of the same type; bias [G,N] that type or F32, or NULL; residual, out [T,N] (that type or F32);
  * K and N multiples of 8; reduce must be NONE.  group_offsets points to G+1 int32 values in DEVICE
  * memory (non-decreasing, first 0, last T; empty groups are fine): the kernel reads them itself, so
  * the host never has to wait for a router's counts.  No workspace.  Rows outside
@@ -222,10 +228,10 @@ pike_status_t pike_grouped_linear_epilogue(pike_handle_t handle, const pike_tens
  *   h   = act( z @ w1 + b1 )                         [M,F]
  *   out = x + h @ w2 + b2                            [M,D]   (residual = un-normalised x)
  *
- * All tensors PIKE_BF16 (gamma, beta, b1, b2 may be F32); x, out [M,D]; w1 [D,F];
+ * All tensors 16-bit, all BF16 or all F16 (gamma, beta, b1, b2 may be F32); x, out [M,D]; w1 [D,F];
  * w2 [F,D] (or transposed with PIKE_FLAG_W_IS_NK); D, F multiples of 8, D <= 16384.
  * epi->act selects the activation, epi->eps the LayerNorm epsilon; scale must be 1
- * and reduce NONE.  z and h are rounded to bf16 and live in the workspace
+ * and reduce NONE.  z and h are rounded to the 16-bit type and live in the workspace
  * (M*D*2 + M*F*2 bytes, each part 256-byte aligned).  Three kernels are enqueued
  * on the stream.
  */
@@ -242,11 +248,11 @@ pike_status_t pike_mlp_block(pike_handle_t handle, const pike_tensor_t *x, const
  *   s[i,j]  = epi->scale * sum_d q[i,d] * k[j,d]
  *   out[i,:] = sum_j softmax_j(s[i,.])[j] * v[j,:]   (j <= i only with PIKE_FLAG_CAUSAL)
  *
- * per (batch, head).  q, out are [B,H,S,D] and k, v [B,H,Sk,D] PIKE_BF16 views, D == 128 or 64, any
+ * per (batch, head).  q, out are [B,H,S,D] and k, v [B,H,Sk,D] 16-bit views (all BF16 or all F16), D == 128 or 64, any
  * S, Sk >= 1; Sk != S (cross attention) only without PIKE_FLAG_CAUSAL.  Rows must be contiguous (stride[3] == 1); the batch, head and row strides may be anything
  * that is a multiple of 8 elements and at least D, so dense [B,H,S,D], a [B,S,H,D] tensor viewed as
  * [B,H,S,D], or the q / k / v slices of a packed [B,S,3,H,D] projection output all work without a copy.  The score matrix lives in tensor memory and registers
- * only; probabilities are rounded to bf16 before the second GEMM.  Workspace: 0
+ * only; probabilities are rounded to the 16-bit type before the second GEMM.  Workspace: 0
  * bytes (the query exists for symmetry).
  */
 pike_status_t pike_attention_chain_workspace(pike_handle_t handle, const pike_tensor_t *q,
@@ -264,12 +270,12 @@ pike_status_t pike_attention_chain(pike_handle_t handle, const pike_tensor_t *q,
  *   a   = softmax(scale * q k^T [+ causal mask]) v           per (batch, head), written as [B,S,H,128]
  *   out = x + a @ w_o + b_o                                  [B,S,E]
  *
- * x, out dense [B,S,E] PIKE_BF16 with E = H*128 <= 4096; w_qkv [E,3E], w_o [E,E] PIKE_BF16 (or transposed
- * with PIKE_FLAG_W_IS_NK); gamma, beta [E], b_qkv [3E], b_o [E] BF16 or F32, each may be NULL.  epi->eps is
+ * x, out dense [B,S,E] 16-bit (BF16 or F16) with E = H*128 <= 4096; w_qkv [E,3E], w_o [E,E] of that type (or transposed
+ * with PIKE_FLAG_W_IS_NK); gamma, beta [E], b_qkv [3E], b_o [E] of that type or F32, each may be NULL.  epi->eps is
  * the LayerNorm epsilon, epi->scale (> 0) the factor on q.k, PIKE_FLAG_CAUSAL the mask; act must be NONE and
  * reduce NONE.  The attention kernel reads q, k, v as strided views of the projection output and writes its
  * result in the layout the output projection reads, so no transpose or copy kernel runs: four kernels are
- * enqueued (LayerNorm, GEMM+bias, attention, GEMM+bias+residual).  z, qkv and a are bf16 in the workspace
+ * enqueued (LayerNorm, GEMM+bias, attention, GEMM+bias+residual).  z, qkv and a are 16-bit in the workspace
  * (2*B*S*E*2 + B*S*3E*2 bytes, each part 256-byte aligned).
  */
 pike_status_t pike_attention_block_workspace(pike_handle_t handle, const pike_tensor_t *x, const pike_epilogue_t *epi,

@@ -16,7 +16,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libpike.so")
 
-PIKE_F32, PIKE_BF16 = 0, 1
+PIKE_F32, PIKE_BF16, PIKE_F16 = 0, 1, 2
 ACT = {"none": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 REDUCE = {"none": 0, "layernorm": 1, "softmax": 2}
 FLAG_W_IS_NK, FLAG_CAUSAL = 0x1, 0x2
@@ -124,6 +124,8 @@ def _dtype_code(t: torch.Tensor) -> int:
         return PIKE_F32
     if t.dtype == torch.bfloat16:
         return PIKE_BF16
+    if t.dtype == torch.float16:
+        return PIKE_F16
     raise TypeError(f"unsupported dtype {t.dtype}")
 
 
@@ -150,7 +152,7 @@ def _epilogue(act, scale, reduce, eps, out_dtype, flags) -> pike_epilogue_t:
     e.scale = float(scale)
     e.reduce = REDUCE[reduce]
     e.eps = float(eps)
-    e.out_dtype = PIKE_F32 if out_dtype == torch.float32 else PIKE_BF16
+    e.out_dtype = {torch.float32: PIKE_F32, torch.bfloat16: PIKE_BF16, torch.float16: PIKE_F16}[out_dtype]
     e.flags = flags
     return e
 
@@ -252,7 +254,7 @@ def pike_linear_softmax_noalloc(x, w, bias=None, *, out, act="none", scale=1.0, 
 
 
 def pike_mlp_block_workspace(x, w1, *, act="gelu_tanh", eps=1e-5, w_is_nk=False) -> int:
-    e = _epilogue(act, 1.0, "none", eps, torch.bfloat16, FLAG_W_IS_NK if w_is_nk else 0)
+    e = _epilogue(act, 1.0, "none", eps, x.dtype, FLAG_W_IS_NK if w_is_nk else 0)
     n = ctypes.c_size_t(0)
     _check(load_library().pike_mlp_block_workspace(_handle(x.device), _tensor(x), _tensor(w1), ctypes.byref(e),
                                                    ctypes.byref(n)), "pike_mlp_block_workspace")
@@ -264,7 +266,7 @@ def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5,
     """out = x + act(LayerNorm(x) @ w1 + b1) @ w2 + b2; see include/pike.h."""
     if out is None:
         out = torch.empty_like(x)
-    e = _epilogue(act, 1.0, "none", eps, torch.bfloat16, FLAG_W_IS_NK if w_is_nk else 0)
+    e = _epilogue(act, 1.0, "none", eps, x.dtype, FLAG_W_IS_NK if w_is_nk else 0)
     need = pike_mlp_block_workspace(x, w1, act=act, eps=eps, w_is_nk=w_is_nk)
     ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
     _check(load_library().pike_mlp_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta), _tensor(w1),
@@ -274,7 +276,7 @@ def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5,
 
 
 def pike_attention_chain_workspace(q, *, scale, causal=True) -> int:
-    e = _epilogue("none", scale, "none", 0.0, torch.bfloat16, FLAG_CAUSAL if causal else 0)
+    e = _epilogue("none", scale, "none", 0.0, q.dtype, FLAG_CAUSAL if causal else 0)
     n = ctypes.c_size_t(0)
     _check(load_library().pike_attention_chain_workspace(_handle(q.device), _tensor(q), ctypes.byref(e),
                                                          ctypes.byref(n)), "pike_attention_chain_workspace")
@@ -285,7 +287,7 @@ def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
     """out = softmax(scale * q k^T [+ causal mask]) v per (batch, head); see include/pike.h."""
     if out is None:
         out = torch.empty_like(q)
-    e = _epilogue("none", scale, "none", 0.0, torch.bfloat16, FLAG_CAUSAL if causal else 0)
+    e = _epilogue("none", scale, "none", 0.0, q.dtype, FLAG_CAUSAL if causal else 0)
     _check(load_library().pike_attention_chain(_handle(q.device), _tensor(q), _tensor(k), _tensor(v),
                                                ctypes.byref(e), _tensor(out), None, 0, _stream(stream)),
            "pike_attention_chain")
@@ -293,7 +295,7 @@ def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
 
 
 def pike_attention_block_workspace(x, *, scale, causal=True, eps=1e-5, w_is_nk=False) -> int:
-    e = _epilogue("none", scale, "none", eps, torch.bfloat16, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
+    e = _epilogue("none", scale, "none", eps, x.dtype, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
     n = ctypes.c_size_t(0)
     _check(load_library().pike_attention_block_workspace(_handle(x.device), _tensor(x), ctypes.byref(e), ctypes.byref(n)),
            "pike_attention_block_workspace")
@@ -305,7 +307,7 @@ def pike_attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, scale, causa
     """out = x + attention(LayerNorm(x) @ w_qkv + b_qkv) @ w_o + b_o for x [B,S,E]; see include/pike.h."""
     if out is None:
         out = torch.empty_like(x)
-    e = _epilogue("none", scale, "none", eps, torch.bfloat16, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
+    e = _epilogue("none", scale, "none", eps, x.dtype, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
     need = pike_attention_block_workspace(x, scale=scale, causal=causal, eps=eps, w_is_nk=w_is_nk)
     ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
     _check(load_library().pike_attention_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta),

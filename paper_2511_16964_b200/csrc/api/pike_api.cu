@@ -49,7 +49,14 @@ struct TimedLaunch {
 size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 size_t elem_size(pike_dtype_t t) { return t == PIKE_F32 ? 4 : 2; }
 
-bool valid_dtype(pike_dtype_t t) { return t == PIKE_F32 || t == PIKE_BF16; }
+bool valid_dtype(pike_dtype_t t) { return t == PIKE_F32 || t == PIKE_BF16 || t == PIKE_F16; }
+bool is_16bit(pike_dtype_t t) { return t == PIKE_BF16 || t == PIKE_F16; }
+// an optional side tensor of a 16-bit chain is fp32 or of the chain's own 16-bit type (bf16 and f16 never mix)
+bool side_ok(const pike_tensor_t *t, pike_dtype_t chain) { return t == nullptr || t->dtype == PIKE_F32 || t->dtype == chain; }
+CUtensorMapDataType map_dtype(pike_dtype_t t)
+{
+    return t == PIKE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+}
 
 // a dense-enough 2-D view: innermost stride 1, row pitch >= columns, 16-byte aligned base and pitch
 pike_status_t check_matrix(const pike_tensor_t *t, int64_t rows, int64_t cols, bool pitch16 = true)
@@ -103,45 +110,45 @@ pike_status_t check_epilogue(const pike_epilogue_t *e)
     return PIKE_OK;
 }
 
-// bf16 [rows, cols] row-major matrix -> tensor map with a (box_cols x box_rows) box, 128-byte swizzle
-pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
+// 16-bit [rows, cols] row-major matrix -> tensor map with a (box_cols x box_rows) box, 128-byte swizzle
+pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t rows, uint64_t cols,
                           uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
 {
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {pitch_elems * 2};
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+    const CUresult r = h->encode(map, map_dtype(dt), 2, const_cast<void *>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
-// bf16 attention operand, element (b, h, s, d) at ptr + b*sb + h*sh + s*ss + d (strides in elements, multiples
+// 16-bit attention operand, element (b, h, s, d) at ptr + b*sb + h*sh + s*ss + d (strides in elements, multiples
 // of 8) -> 4-D map {D, S, H, B} with a (64 x 128 x 1 x 1) box
-pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t B, uint64_t H, uint64_t S,
+pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t B, uint64_t H, uint64_t S,
                             uint64_t D, uint64_t sb, uint64_t sh, uint64_t ss)
 {
     const cuuint64_t dims[4] = {D, S, H, B};
     const cuuint64_t strides[3] = {ss * 2, sh * 2, sb * 2};
     const cuuint32_t box[4] = {64, 128, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(ptr), dims, strides, box,
+    const CUresult r = h->encode(map, map_dtype(dt), 4, const_cast<void *>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
-// bf16 weights [groups, rows, cols] (dense matrices `group_pitch` elements apart; groups == 1 for a plain
+// 16-bit weights [groups, rows, cols] (dense matrices `group_pitch` elements apart; groups == 1 for a plain
 // GEMM) -> 3-D map with a (box_cols x box_rows x 1) box, 128-byte swizzle
-pike_status_t make_map_w(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t groups, uint64_t rows,
+pike_status_t make_map_w(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t groups, uint64_t rows,
                          uint64_t cols, uint64_t pitch_elems, uint64_t group_pitch, uint32_t box_cols, uint32_t box_rows)
 {
     const cuuint64_t dims[3] = {cols, rows, groups};
     const cuuint64_t strides[2] = {pitch_elems * 2, (groups > 1 ? group_pitch : rows * pitch_elems) * 2};
     const cuuint32_t box[3] = {box_cols, box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = h->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(ptr), dims, strides, box,
+    const CUresult r = h->encode(map, map_dtype(dt), 3, const_cast<void *>(ptr), dims, strides, box,
                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
@@ -172,6 +179,7 @@ pike_status_t linear_shape(const pike_tensor_t *x, const pike_tensor_t *w, const
         if (epi->out_dtype != PIKE_F32) return PIKE_ERR_DTYPE;
     } else {
         if (s.K % 8 != 0 || s.N % 8 != 0) return PIKE_ERR_UNSUPPORTED;
+        if (epi->out_dtype != PIKE_F32 && epi->out_dtype != x->dtype) return PIKE_ERR_DTYPE;
         if (epi->reduce == PIKE_REDUCE_SOFTMAX && epi->out_dtype != PIKE_F32) return PIKE_ERR_UNSUPPORTED;
     }
     return PIKE_OK;
@@ -183,24 +191,24 @@ size_t softmax_partials_bytes(const LinearShape &s)
     return align256((size_t)s.M * (size_t)num_n * sizeof(float2));
 }
 
-// Launch one bf16 GEMM + epilogue.  All tensors validated by the caller.
+// Launch one 16-bit GEMM + epilogue; w's dtype (bf16 or f16) is the chain's.  All tensors validated by the caller.
 pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pike_tensor_t *w, bool w_is_nk, int64_t M,
                        int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
                        void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
                        cudaStream_t stream, int partials_mode = 1, const int *group_offsets = nullptr, int num_groups = 0)
 {
     CUtensorMap tmA, tmB;
-    if (pike_status_t st = make_map_2d(h, &tmA, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
+    if (pike_status_t st = make_map_2d(h, &tmA, w->dtype, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
         return st;
     // w is [K,N] / [N,K], or [groups,K,N] / [groups,N,K] in grouped mode (the last two dimensions are the matrix)
     const int wd = w->ndim - 2;
     const uint64_t groups = wd == 1 ? (uint64_t)w->shape[0] : 1, gpitch = wd == 1 ? (uint64_t)w->stride[0] : 0;
     if (w_is_nk) {
-        if (pike_status_t st = make_map_w(h, &tmB, w->data, groups, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[wd],
+        if (pike_status_t st = make_map_w(h, &tmB, w->dtype, w->data, groups, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[wd],
                                           gpitch, pike::GEMM_BK, pike::GEMM_BN / 2))
             return st;
     } else {
-        if (pike_status_t st = make_map_w(h, &tmB, w->data, groups, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[wd],
+        if (pike_status_t st = make_map_w(h, &tmB, w->dtype, w->data, groups, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[wd],
                                           gpitch, 64, pike::GEMM_BK))
             return st;
     }
@@ -208,6 +216,7 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     memset(&g, 0, sizeof(g));
     g.M = (int)M; g.N = (int)N; g.K = (int)K;
     g.w_is_nk = w_is_nk ? 1 : 0;
+    g.f16 = w->dtype == PIKE_F16 ? 1 : 0;
     g.bias = bias ? bias->data : nullptr;
     g.bias_f32 = bias && bias->dtype == PIKE_F32;
     g.residual = res_ptr; g.residual_f32 = res_f32 ? 1 : 0; g.ldr = ldr;
@@ -409,6 +418,8 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         return pike::launch_fp32_chain(a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
 
+    for (const pike_tensor_t *t : {bias, residual, gamma, beta})
+        if (!side_ok(t, x->dtype)) return PIKE_ERR_DTYPE;
     // a row reduction on this path is split across the GEMM's column tiles: per-(row, tile) pairs go to the
     // workspace, a second kernel combines them and finishes the rows in place
     float2 *partials = nullptr;
@@ -431,7 +442,8 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
             if (pike::launch_layernorm_finish(out->data, out->dtype == PIKE_F32, out->stride[0], partials, num_n,
                                               pike::GEMM_BN, (int)s.M, (int)s.N, gamma ? gamma->data : nullptr,
                                               gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
-                                              beta && beta->dtype == PIKE_F32, epi->eps, stream) != cudaSuccess)
+                                              beta && beta->dtype == PIKE_F32, epi->eps, x->dtype == PIKE_F16,
+                                              stream) != cudaSuccess)
                 return PIKE_ERR_CUDA;
         } else {
             TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
@@ -451,7 +463,9 @@ pike_status_t pike_grouped_linear_epilogue(pike_handle_t h, const pike_tensor_t 
     if (h == nullptr || x == nullptr || w == nullptr || out == nullptr || group_offsets == nullptr) return PIKE_ERR_NULL;
     if (pike_status_t st = check_epilogue(epi)) return st;
     if (x->ndim != 2 || w->ndim != 3) return PIKE_ERR_SHAPE;
-    if (x->dtype != PIKE_BF16 || w->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (!is_16bit(x->dtype) || w->dtype != x->dtype) return PIKE_ERR_DTYPE;
+    if (epi->out_dtype != PIKE_F32 && epi->out_dtype != x->dtype) return PIKE_ERR_DTYPE;
+    if (!side_ok(bias, x->dtype) || !side_ok(residual, x->dtype)) return PIKE_ERR_DTYPE;
     if (epi->reduce != PIKE_REDUCE_NONE) return PIKE_ERR_UNSUPPORTED;
     const bool nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
     const int64_t T = x->shape[0], K = x->shape[1], G = w->shape[0];
@@ -494,7 +508,7 @@ static pike_status_t mlp_shape(const pike_tensor_t *x, const pike_tensor_t *w1, 
     if (x == nullptr || w1 == nullptr) return PIKE_ERR_NULL;
     if (pike_status_t st = check_epilogue(epi)) return st;
     if (x->ndim != 2 || w1->ndim != 2) return PIKE_ERR_SHAPE;
-    if (x->dtype != PIKE_BF16 || w1->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (!is_16bit(x->dtype) || w1->dtype != x->dtype || epi->out_dtype != x->dtype) return PIKE_ERR_DTYPE;
     if (epi->reduce != PIKE_REDUCE_NONE || epi->scale != 1.0f) return PIKE_ERR_UNSUPPORTED;
     nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
     M = x->shape[0];
@@ -531,7 +545,9 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
     if (pike_status_t st = check_matrix(w1, nk ? F : D, nk ? D : F)) return st;
     if (pike_status_t st = check_matrix(w2, nk ? D : F, nk ? F : D)) return st;
     if (pike_status_t st = check_matrix(out, M, D)) return st;
-    if (w2->dtype != PIKE_BF16 || out->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (w2->dtype != x->dtype || out->dtype != x->dtype) return PIKE_ERR_DTYPE;
+    for (const pike_tensor_t *t : {gamma, beta, b1, b2})
+        if (!side_ok(t, x->dtype)) return PIKE_ERR_DTYPE;
     if (pike_status_t st = check_vector(gamma, D)) return st;
     if (pike_status_t st = check_vector(beta, D)) return st;
     if (pike_status_t st = check_vector(b1, F)) return st;
@@ -554,10 +570,10 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
         if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
                                         gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
                                         beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D,
-                                        stream) != cudaSuccess)
+                                        x->dtype == PIKE_F16, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
-    // h = act(z @ w1 + b1), bf16
+    // h = act(z @ w1 + b1), rounded to the chain's 16-bit type
     if (pike_status_t st = run_gemm(h, z, D, w1, nk, M, D, F, b1, nullptr, false, 0, hbuf, false, F, (int)epi->act,
                                     1.0f, nullptr, stream))
         return st;
@@ -571,7 +587,7 @@ static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *e
     if (q == nullptr) return PIKE_ERR_NULL;
     if (pike_status_t st = check_epilogue(epi)) return st;
     if (q->ndim != 4) return PIKE_ERR_SHAPE;
-    if (q->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (!is_16bit(q->dtype) || epi->out_dtype != q->dtype) return PIKE_ERR_DTYPE;
     if (q->shape[3] != 128 && q->shape[3] != 64) return PIKE_ERR_UNSUPPORTED;
     if (q->shape[0] < 0 || q->shape[1] < 0 || q->shape[2] < 0) return PIKE_ERR_SHAPE;
     if (q->shape[0] * q->shape[1] > 0x7fffff || q->shape[2] > 0x7fffff00) return PIKE_ERR_UNSUPPORTED;
@@ -583,7 +599,7 @@ static pike_status_t attn_shape(const pike_tensor_t *q, const pike_epilogue_t *e
 static pike_status_t check_bhsd(const pike_tensor_t *t, const pike_tensor_t *like, bool own_length = false)
 {
     if (t == nullptr) return PIKE_ERR_NULL;
-    if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (t->dtype != like->dtype) return PIKE_ERR_DTYPE;
     if (t->ndim != 4) return PIKE_ERR_SHAPE;
     for (int i = 0; i < 4; ++i)
         if (t->shape[i] != like->shape[i] && !(own_length && i == 2)) return PIKE_ERR_SHAPE;   // keys may have their own length
@@ -606,14 +622,15 @@ static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, cons
 {
     const uint64_t B = q->shape[0], H = q->shape[1], S = q->shape[2], Sk = k->shape[2], D = q->shape[3];
     CUtensorMap tmQ, tmK, tmV;
-    if (pike_status_t st = make_map_bhsd(h, &tmQ, q->data, B, H, S, D, eff_stride(q, 0), eff_stride(q, 1), eff_stride(q, 2))) return st;
-    if (pike_status_t st = make_map_bhsd(h, &tmK, k->data, B, H, Sk, D, eff_stride(k, 0), eff_stride(k, 1), eff_stride(k, 2))) return st;
-    if (pike_status_t st = make_map_bhsd(h, &tmV, v->data, B, H, Sk, D, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmQ, q->dtype, q->data, B, H, S, D, eff_stride(q, 0), eff_stride(q, 1), eff_stride(q, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmK, q->dtype, k->data, B, H, Sk, D, eff_stride(k, 0), eff_stride(k, 1), eff_stride(k, 2))) return st;
+    if (pike_status_t st = make_map_bhsd(h, &tmV, q->dtype, v->data, B, H, Sk, D, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
     pike::AttnArgs a;
     memset(&a, 0, sizeof(a));
     a.BH = (int)(B * H); a.H = (int)H; a.S = (int)S; a.Sk = (int)Sk; a.D = (int)D;
     a.scale = scale;
     a.causal = causal ? 1 : 0;
+    a.f16 = q->dtype == PIKE_F16 ? 1 : 0;
     a.out = out->data;
     a.out_b = (long long)eff_stride(out, 0); a.out_h = (long long)eff_stride(out, 1); a.out_s = (long long)eff_stride(out, 2);
     a.status = h->status;
@@ -662,7 +679,7 @@ static pike_status_t block_shape(const pike_tensor_t *x, const pike_epilogue_t *
     if (x == nullptr) return PIKE_ERR_NULL;
     if (pike_status_t st = check_epilogue(epi)) return st;
     if (x->ndim != 3) return PIKE_ERR_SHAPE;
-    if (x->dtype != PIKE_BF16 || epi->out_dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (!is_16bit(x->dtype) || epi->out_dtype != x->dtype) return PIKE_ERR_DTYPE;
     B = x->shape[0]; S = x->shape[1]; E = x->shape[2];
     if (B < 0 || S < 0 || E < 1) return PIKE_ERR_SHAPE;
     if (E % 128 != 0 || E > 4096) return PIKE_ERR_UNSUPPORTED;          // heads of 128; LayerNorm row in one warp
@@ -672,10 +689,10 @@ static pike_status_t block_shape(const pike_tensor_t *x, const pike_epilogue_t *
     return PIKE_OK;
 }
 
-static pike_status_t check_dense_bse(const pike_tensor_t *t, int64_t B, int64_t S, int64_t E)
+static pike_status_t check_dense_bse(const pike_tensor_t *t, pike_dtype_t dt, int64_t B, int64_t S, int64_t E)
 {
     if (t == nullptr) return PIKE_ERR_NULL;
-    if (t->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (t->dtype != dt) return PIKE_ERR_DTYPE;
     if (t->ndim != 3 || t->shape[0] != B || t->shape[1] != S || t->shape[2] != E) return PIKE_ERR_SHAPE;
     if (B * S == 0) return PIKE_OK;
     if (t->data == nullptr) return PIKE_ERR_NULL;
@@ -704,9 +721,11 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
     int64_t B, S, E;
     if (pike_status_t st = block_shape(x, epi, B, S, E)) return st;
     const bool nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
-    if (pike_status_t st = check_dense_bse(x, B, S, E)) return st;
-    if (pike_status_t st = check_dense_bse(out, B, S, E)) return st;
-    if (w_qkv->dtype != PIKE_BF16 || w_o->dtype != PIKE_BF16) return PIKE_ERR_DTYPE;
+    if (pike_status_t st = check_dense_bse(x, x->dtype, B, S, E)) return st;
+    if (pike_status_t st = check_dense_bse(out, x->dtype, B, S, E)) return st;
+    if (w_qkv->dtype != x->dtype || w_o->dtype != x->dtype) return PIKE_ERR_DTYPE;
+    for (const pike_tensor_t *t : {gamma, beta, b_qkv, b_o})
+        if (!side_ok(t, x->dtype)) return PIKE_ERR_DTYPE;
     if (pike_status_t st = check_matrix(w_qkv, nk ? 3 * E : E, nk ? E : 3 * E)) return st;
     if (pike_status_t st = check_matrix(w_o, E, E)) return st;
     if (pike_status_t st = check_vector(gamma, E)) return st;
@@ -731,7 +750,7 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
         TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
         if (pike::launch_layernorm_bf16(x->data, E, z, E, gamma ? gamma->data : nullptr, gamma && gamma->dtype == PIKE_F32,
                                         beta ? beta->data : nullptr, beta && beta->dtype == PIKE_F32, epi->eps, (int)M,
-                                        (int)E, stream) != cudaSuccess)
+                                        (int)E, x->dtype == PIKE_F16, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // qkv = z @ w_qkv + b_qkv, laid out [B, S, 3, H, 128]
@@ -741,12 +760,12 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
     // attention straight on the packed buffer: q, k, v are [B,H,S,128] views of it, the result is written as [B,S,H,128]
     pike_tensor_t view[4];
     for (int i = 0; i < 4; ++i) {
-        view[i].dtype = PIKE_BF16;
+        view[i].dtype = x->dtype;
         view[i].ndim = 4;
         view[i].shape[0] = B; view[i].shape[1] = H; view[i].shape[2] = S; view[i].shape[3] = 128;
         view[i].stride[3] = 1; view[i].stride[1] = 128;
         if (i < 3) {
-            view[i].data = static_cast<__nv_bfloat16 *>(qkv) + (int64_t)i * E;
+            view[i].data = static_cast<uint16_t *>(qkv) + (int64_t)i * E;
             view[i].stride[0] = S * 3 * E; view[i].stride[2] = 3 * E;
         } else {
             view[i].data = att;

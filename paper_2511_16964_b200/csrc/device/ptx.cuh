@@ -4,6 +4,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -368,13 +369,13 @@ __device__ __forceinline__ constexpr uint64_t desc_advance(uint64_t desc, uint32
     return desc + static_cast<uint64_t>(bytes >> 4);
 }
 
-// Instruction descriptor for kind::f16 with bf16 operands and fp32 accumulator:
-//   [4,6) D format (1 = f32)  [7,10) A format (1 = bf16)  [10,13) B format (1 = bf16)
+// Instruction descriptor for kind::f16 with 16-bit operands (both bf16, or both f16) and fp32 accumulator:
+//   [4,6) D format (1 = f32)  [7,10) A format (0 = f16, 1 = bf16)  [10,13) B format (same as A)
 //   bit 15 A is MN-major   bit 16 B is MN-major   [17,23) N >> 3   [24,29) M >> 4
-__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major)
+__host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major, bool f16 = false)
 {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u) |
-           (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+    return (1u << 4) | (f16 ? 0u : ((1u << 7) | (1u << 10))) | (a_mn_major ? (1u << 15) : 0u) |
+           (b_mn_major ? (1u << 16) : 0u) | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
 // ------------------------------------------------------------------ misc ----
@@ -402,6 +403,30 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (low 16 bits)
     return *reinterpret_cast<uint32_t *>(&v);
+}
+// The 16-bit storage type of a tensor is bf16 or IEEE half (f16 == true); both are computed in fp32.
+__device__ __forceinline__ float h16_lo(uint32_t u, bool f16)
+{
+    return f16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(u & 0xFFFFu))) : bf16_lo(u);
+}
+__device__ __forceinline__ float h16_hi(uint32_t u, bool f16)
+{
+    return f16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(u >> 16))) : bf16_hi(u);
+}
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
+{
+    __half2 v = __floats2half2_rn(lo, hi);             // .x = lo (low 16 bits)
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint32_t pack_h16x2(float lo, float hi, bool f16)
+{
+    return f16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
+}
+// element i of a 16-bit vector as fp32
+__device__ __forceinline__ float h16_at(const void *p, long long i, bool f16)
+{
+    const unsigned short u = static_cast<const unsigned short *>(p)[i];
+    return f16 ? __half2float(__ushort_as_half(u)) : __uint_as_float(static_cast<uint32_t>(u) << 16);
 }
 
 }  // namespace pike

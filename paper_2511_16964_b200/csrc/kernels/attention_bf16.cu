@@ -11,7 +11,7 @@
 //   WG1  softmax for query tile 0        WG2  softmax for query tile 1   (thread = row)
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each.
 //   S_t(j) = Q_t K_j^T      both operands K-major from shared memory
-//   P_t(j) = bf16 probabilities, written by the softmax threads over the first 64
+//   P_t(j) = 16-bit probabilities (the type of Q/K/V: bf16 or f16), written by the softmax threads over the first 64
 //            columns of S_t (two per 32-bit column) and read by the second MMA as its
 //            A operand straight from tensor memory
 //   O_t   += P_t(j) V_j     V is the MN-major B operand; accumulates in tensor memory
@@ -60,8 +60,9 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
+// F16 = the tensors are IEEE half instead of bf16 (operand format of both MMAs, P and the output).
 // D = head dimension (64 or 128): one or two 64-wide swizzled sub-tiles per operand tile
-template <int D>
+template <int D, bool F16>
 __global__ void __launch_bounds__(THREADS, 1)
 attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, const AttnArgs p)
@@ -180,8 +181,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             // The whole warp runs this loop (uniform control flow keeps descriptors and counters in
             // uniform registers); one elected lane issues the MMAs and commits.
             const bool leader = elect_one();
-            const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false);   // Q, K both K-major (d contiguous)
-            const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true);      // P K-major (TMEM), V MN-major
+            const uint32_t idesc_s = make_idesc_bf16(BQ, BKV, false, false, F16);   // Q, K both K-major (d contiguous)
+            const uint32_t idesc_o = make_idesc_bf16(BQ, D, false, true, F16);     // P K-major (TMEM), V MN-major
             // Descriptors are built once; the issue loops only add constants to them (this single thread's
             // instruction stream is on the critical path of every hand-off).
             const uint64_t q_desc0 = make_smem_desc_sw128(smem_u32(q_s), 0, 1024);
@@ -354,7 +355,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                         const float e0 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i]), c, neg_m));
                         const float e1 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i + 1]), c, neg_m));
                         ls[i & 3] += e0 + e1;
-                        pk[i] = pack_bf16x2(e0, e1);
+                        pk[i] = pack_h16x2(e0, e1, F16);
                     }
                     tmem_st32(s_addr + cc * 32, pk);
                 }
@@ -369,7 +370,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             ++n_o;
             tc_fence_after();
             const float inv_l = 1.0f / l_run;
-            __nv_bfloat16 *orow = static_cast<__nv_bfloat16 *>(p.out) + (long long)(bh / p.H) * p.out_b +
+            uint16_t *orow = static_cast<uint16_t *>(p.out) + (long long)(bh / p.H) * p.out_b +
                                   (long long)(bh % p.H) * p.out_h + (long long)qidx * p.out_s;
 #pragma unroll 1
             for (int cc = 0; cc < D / 32; ++cc) {
@@ -383,8 +384,8 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
                         for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[g * 8 + i]) * inv_l;
                         *reinterpret_cast<uint4 *>(orow + cc * 32 + g * 8) =
-                            make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]),
-                                       pack_bf16x2(f[6], f[7]));
+                            make_uint4(pack_h16x2(f[0], f[1], F16), pack_h16x2(f[2], f[3], F16),
+                                       pack_h16x2(f[4], f[5], F16), pack_h16x2(f[6], f[7], F16));
                     }
                 }
             }
@@ -402,7 +403,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     }
 }
 
-template <int D>
+template <int D, bool F16>
 static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                                       const AttnArgs &a, int num_sms, cudaStream_t stream)
 {
@@ -411,7 +412,7 @@ static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap 
     static int regs_ok = -1;
     if (regs_ok < 0) {
         cudaFuncAttributes attr;
-        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel<D>);
+        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel<D, F16>);
         if (e != cudaSuccess) return e;
         regs_ok = (attr.numRegs * THREADS >= 128 * REGS_WG0 + 256 * REGS_SOFTMAX) ? 1 : 0;
     }
@@ -419,11 +420,11 @@ static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap 
     const int num_q_tiles = (a.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
     const long long num_items = (long long)((num_pairs + 1) / 2) * a.BH;   // slots: two items each
-    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SMEM_BYTES);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(num_items < num_sms ? num_items : num_sms);   // persistent: one CTA per SM
-    attention_bf16_kernel<D><<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
+    attention_bf16_kernel<D, F16><<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError();
 }
 
@@ -433,8 +434,12 @@ cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK
                                   const AttnArgs &a, int num_sms, cudaStream_t stream)
 {
     if (a.BH <= 0 || a.S <= 0 || a.Sk <= 0) return cudaSuccess;
-    if (a.D == 64) return launch_attention_d<64>(tmQ, tmK, tmV, a, num_sms, stream);
-    if (a.D == 128) return launch_attention_d<128>(tmQ, tmK, tmV, a, num_sms, stream);
+    if (a.D == 64)
+        return a.f16 ? launch_attention_d<64, true>(tmQ, tmK, tmV, a, num_sms, stream)
+                     : launch_attention_d<64, false>(tmQ, tmK, tmV, a, num_sms, stream);
+    if (a.D == 128)
+        return a.f16 ? launch_attention_d<128, true>(tmQ, tmK, tmV, a, num_sms, stream)
+                     : launch_attention_d<128, false>(tmQ, tmK, tmV, a, num_sms, stream);
     return cudaErrorInvalidValue;
 }
 

@@ -163,7 +163,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------- MMA issuer (leader CTA only; warp-uniform loop, one elected lane issues)
         if (rank == 0) {
             const bool leader = elect_one();
-            const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk);
+            const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk, p.f16 != 0);
             const uint32_t a_addr0 = smem_u32(tiles), b_addr0 = a_addr0 + A_BYTES;
             const uint64_t adesc0 = make_smem_desc_sw128(a_addr0, 0, 1024);
             const uint64_t bdesc0 = p.w_is_nk ? make_smem_desc_sw128(b_addr0, 0, 1024)
@@ -202,6 +202,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------------------------------------------------------------- epilogue
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int et = threadIdx.x - 64;        // 0..127
+        const bool f16 = p.f16 != 0;            // 16-bit tensors are IEEE half instead of bf16
         int it = 0;
         for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
             int m_blk, n_blk;
@@ -220,7 +221,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 float b = 0.0f;
                 if (p.bias != nullptr && n0 + i < p.N)
                     b = p.bias_f32 ? static_cast<const float *>(p.bias)[bias0 + i]
-                                   : __bfloat162float(static_cast<const __nv_bfloat16 *>(p.bias)[bias0 + i]);
+                                   : h16_at(p.bias, bias0 + i, p.f16 != 0);
                 ctrl->bias[i] = b;
             }
             named_bar_sync(1, EPI_THREADS);
@@ -249,8 +250,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             res32[g] = (nc + g * 4 < p.N) ? *reinterpret_cast<const float4 *>(rp + g * 4)
                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
                     } else {
-                        const __nv_bfloat16 *rp =
-                            static_cast<const __nv_bfloat16 *>(p.residual) + (long long)row * p.ldr + nc;
+                        const uint16_t *rp = static_cast<const uint16_t *>(p.residual) + (long long)row * p.ldr + nc;
 #pragma unroll
                         for (int g = 0; g < 4; ++g)
                             res16[g] = (nc + g * 8 < p.N) ? *reinterpret_cast<const uint4 *>(rp + g * 8)
@@ -276,8 +276,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             const uint32_t w4[4] = {res16[g].x, res16[g].y, res16[g].z, res16[g].w};
 #pragma unroll
                             for (int h = 0; h < 4; ++h) {
-                                v[g * 8 + 2 * h] += bf16_lo(w4[h]);
-                                v[g * 8 + 2 * h + 1] += bf16_hi(w4[h]);
+                                v[g * 8 + 2 * h] += h16_lo(w4[h], f16);
+                                v[g * 8 + 2 * h + 1] += h16_hi(w4[h], f16);
                             }
                         }
                     }
@@ -323,13 +323,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                 *reinterpret_cast<float4 *>(op + g * 4) =
                                     make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
                     } else {
-                        __nv_bfloat16 *op = static_cast<__nv_bfloat16 *>(p.out) + (long long)row * p.ldo + nc;
+                        uint16_t *op = static_cast<uint16_t *>(p.out) + (long long)row * p.ldo + nc;
 #pragma unroll
                         for (int g = 0; g < 4; ++g)
                             if (nc + g * 8 < p.N)
                                 *reinterpret_cast<uint4 *>(op + g * 8) =
-                                    make_uint4(pack_bf16x2(v[g * 8 + 0], v[g * 8 + 1]), pack_bf16x2(v[g * 8 + 2], v[g * 8 + 3]),
-                                               pack_bf16x2(v[g * 8 + 4], v[g * 8 + 5]), pack_bf16x2(v[g * 8 + 6], v[g * 8 + 7]));
+                                    make_uint4(pack_h16x2(v[g * 8 + 0], v[g * 8 + 1], f16),
+                                               pack_h16x2(v[g * 8 + 2], v[g * 8 + 3], f16),
+                                               pack_h16x2(v[g * 8 + 4], v[g * 8 + 5], f16),
+                                               pack_h16x2(v[g * 8 + 6], v[g * 8 + 7], f16));
                     }
                 }
             }

@@ -23,10 +23,11 @@ struct Fp32ChainArgs {
 };
 cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, cudaStream_t stream);
 
-// ---- bf16 tcgen05 GEMM + epilogue ------------------------------------------------
+// ---- 16-bit (bf16 or f16) tcgen05 GEMM + epilogue --------------------------------
 struct GemmArgs {
     int M, N, K;
     int w_is_nk;
+    int f16;               // every 16-bit tensor (x, w and any 16-bit bias/residual/out) is IEEE half, not bf16
     const void *bias;      int bias_f32;
     const void *residual;  int residual_f32;  long long ldr;
     void *out;             int out_f32;       long long ldo;
@@ -52,19 +53,20 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
                              cudaStream_t stream);
 
 // ---- row kernels -------------------------------------------------------------------
-// z = LayerNorm(x) rows, bf16 in/out, fp32 statistics; gamma/beta bf16 or f32 or null.
+// z = LayerNorm(x) rows, 16-bit in/out (f16 != 0: IEEE half, else bf16), fp32 statistics; gamma/beta of
+// the same 16-bit type or f32 or null.
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
-                                  int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D,
+                                  int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
                                   cudaStream_t stream);
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
                                   cudaStream_t stream);
 
-// out = (v - mean)/sqrt(var + eps)*gamma + beta in place (v bf16 or f32), statistics combined from the
+// out = (v - mean)/sqrt(var + eps)*gamma + beta in place (v 16-bit or f32), statistics combined from the
 // per-(row, n-tile) (mean, sum of squared deviations) pairs; tile_n = columns per tile
 cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
                                     int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
-                                    int beta_f32, float eps, cudaStream_t stream);
+                                    int beta_f32, float eps, int f16, cudaStream_t stream);
 
 // ---- attention ---------------------------------------------------------------------
 struct AttnArgs {
@@ -72,7 +74,8 @@ struct AttnArgs {
     int Sk, D;      // key/value length (== S unless cross attention) and head dimension (64 or 128)
     float scale;
     int causal;
-    void *out;      // bf16; element (b, h, s, d) at out + b*out_b + h*out_h + s*out_s + d
+    int f16;        // q, k, v and out are IEEE half instead of bf16
+    void *out;      // 16-bit; element (b, h, s, d) at out + b*out_b + h*out_h + s*out_s + d
     long long out_b, out_h, out_s;
     unsigned int *status;
     unsigned long long limit_ns;

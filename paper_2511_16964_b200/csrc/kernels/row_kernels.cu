@@ -1,4 +1,4 @@
-// Bandwidth-bound row kernels: bf16 LayerNorm (the MLP block's prologue) and the
+// Bandwidth-bound row kernels: 16-bit (bf16 or f16) LayerNorm (the MLP block's prologue) and the
 // second half of the split-row softmax (combine per-tile partials, normalise in place).
 #include "../device/ptx.cuh"
 #include "kernels.h"
@@ -23,20 +23,21 @@ __device__ __forceinline__ float block_sum(float x, float *red, int tid)
     return x;
 }
 
-__device__ __forceinline__ float load_param(const void *p, int is_f32, int i, float dflt)
+__device__ __forceinline__ float load_param(const void *p, int is_f32, int i, float dflt, bool f16)
 {
     if (p == nullptr) return dflt;
-    return is_f32 ? static_cast<const float *>(p)[i] : __bfloat162float(static_cast<const __nv_bfloat16 *>(p)[i]);
+    return is_f32 ? static_cast<const float *>(p)[i] : h16_at(p, i, f16);
 }
 
 // One CTA per row; the row stays in registers between the mean pass, the
 // variance pass (sum of squared deviations, not E[x^2]-E[x]^2) and the store, so
 // HBM sees one read and one write per element.
 __global__ void __launch_bounds__(LN_THREADS)
-layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_bfloat16 *__restrict__ z,
+layernorm_bf16_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *__restrict__ z,
                       long long ldz, const void *gamma, int gamma_f32, const void *beta, int beta_f32, float eps,
-                      int D)
+                      int D, int f16_flag)
 {
+    const bool f16 = f16_flag != 0;
     __shared__ float red[32];
     const int tid = threadIdx.x;
     const long long row = blockIdx.x;
@@ -52,7 +53,7 @@ layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_b
             c[i] = xr[ci];
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
-            for (int h = 0; h < 4; ++h) sum += bf16_lo(w[h]) + bf16_hi(w[h]);
+            for (int h = 0; h < 4; ++h) sum += h16_lo(w[h], f16) + h16_hi(w[h], f16);
         }
     }
     const float mean = block_sum(sum, red, tid) / (float)D;
@@ -64,7 +65,7 @@ layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_b
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float a = bf16_lo(w[h]) - mean, b = bf16_hi(w[h]) - mean;
+                const float a = h16_lo(w[h], f16) - mean, b = h16_hi(w[h], f16) - mean;
                 ss += a * a + b * b;
             }
         }
@@ -80,11 +81,11 @@ layernorm_bf16_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_b
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
                 const int e = ci * 8 + 2 * h;
-                const float a = (bf16_lo(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f) +
-                                load_param(beta, beta_f32, e, 0.0f);
-                const float b = (bf16_hi(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f) +
-                                load_param(beta, beta_f32, e + 1, 0.0f);
-                o[h] = pack_bf16x2(a, b);
+                const float a = (h16_lo(w[h], f16) - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f, f16) +
+                                load_param(beta, beta_f32, e, 0.0f, f16);
+                const float b = (h16_hi(w[h], f16) - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f, f16) +
+                                load_param(beta, beta_f32, e + 1, 0.0f, f16);
+                o[h] = pack_h16x2(a, b, f16);
             }
             zr[ci] = make_uint4(o[0], o[1], o[2], o[3]);
         }
@@ -104,8 +105,9 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
-// eight consecutive parameters starting at element e (e % 8 == 0) as fp32; KIND 0 = absent, 1 = bf16, 2 = f32
-template <int KIND>
+// eight consecutive parameters starting at element e (e % 8 == 0) as fp32; KIND 0 = absent, 1 = 16-bit
+// (the type of x), 2 = f32
+template <int KIND, bool F16>
 __device__ __forceinline__ void load_param8(const void *p, int e, float dflt, float (&out)[8])
 {
     if constexpr (KIND == 0) {
@@ -117,16 +119,16 @@ __device__ __forceinline__ void load_param8(const void *p, int e, float dflt, fl
         out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
         out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
     } else {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p) + e));
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(p) + e));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int h = 0; h < 4; ++h) { out[2 * h] = bf16_lo(w[h]); out[2 * h + 1] = bf16_hi(w[h]); }
+        for (int h = 0; h < 4; ++h) { out[2 * h] = h16_lo(w[h], F16); out[2 * h + 1] = h16_hi(w[h], F16); }
     }
 }
 
-template <int GK, int BK>
+template <int GK, int BK, bool F16>
 __global__ void __launch_bounds__(LNW_WARPS * 32, 2)
-layernorm_bf16_warp_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, __nv_bfloat16 *__restrict__ z,
+layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *__restrict__ z,
                            long long ldz, const void *gamma, const void *beta, float eps, int M, int D)
 {
     const int lane = threadIdx.x & 31;
@@ -146,7 +148,7 @@ layernorm_bf16_warp_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, _
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
         const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
-        for (int h = 0; h < 4; ++h) sum += bf16_lo(w[h]) + bf16_hi(w[h]);   // padding chunks are zero
+        for (int h = 0; h < 4; ++h) sum += h16_lo(w[h], F16) + h16_hi(w[h], F16);   // padding chunks are zero
     }
     const float mean = warp_sum(sum) / (float)D;
     float ss = 0.0f;
@@ -156,7 +158,7 @@ layernorm_bf16_warp_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, _
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float a = bf16_lo(w[h]) - mean, b = bf16_hi(w[h]) - mean;
+                const float a = h16_lo(w[h], F16) - mean, b = h16_hi(w[h], F16) - mean;
                 ss += a * a + b * b;
             }
         }
@@ -169,14 +171,14 @@ layernorm_bf16_warp_kernel(const __nv_bfloat16 *__restrict__ x, long long ldx, _
         if (ci < nchunks) {
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
             float g[8], be[8];
-            load_param8<GK>(gamma, ci * 8, 1.0f, g);
-            load_param8<BK>(beta, ci * 8, 0.0f, be);
+            load_param8<GK, F16>(gamma, ci * 8, 1.0f, g);
+            load_param8<BK, F16>(beta, ci * 8, 0.0f, be);
             uint32_t o[4];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float a = (bf16_lo(w[h]) - mean) * rstd * g[2 * h] + be[2 * h];
-                const float b = (bf16_hi(w[h]) - mean) * rstd * g[2 * h + 1] + be[2 * h + 1];
-                o[h] = pack_bf16x2(a, b);
+                const float a = (h16_lo(w[h], F16) - mean) * rstd * g[2 * h] + be[2 * h];
+                const float b = (h16_hi(w[h], F16) - mean) * rstd * g[2 * h + 1] + be[2 * h + 1];
+                o[h] = pack_h16x2(a, b, F16);
             }
             zr[ci] = make_uint4(o[0], o[1], o[2], o[3]);
         }
@@ -241,9 +243,11 @@ softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__rest
 template <bool OUT_F32>
 __global__ void __launch_bounds__(SM_THREADS)
 layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__restrict__ partials, int num_n_tiles,
-                        int tile_n, int N, const void *gamma, int gamma_f32, const void *beta, int beta_f32, float eps)
+                        int tile_n, int N, const void *gamma, int gamma_f32, const void *beta, int beta_f32, float eps,
+                        int f16_flag)
 {
     __shared__ float red[32];
+    const bool f16 = f16_flag != 0;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long row = blockIdx.x;
     const float2 *pr = partials + row * num_n_tiles;
@@ -274,14 +278,18 @@ layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__
         for (int i = tid; i < N / 4; i += SM_THREADS) {
             float4 x = vr[i];
             const int e = i * 4;
-            x.x = (x.x - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f) + load_param(beta, beta_f32, e, 0.0f);
-            x.y = (x.y - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f) + load_param(beta, beta_f32, e + 1, 0.0f);
-            x.z = (x.z - mean) * rstd * load_param(gamma, gamma_f32, e + 2, 1.0f) + load_param(beta, beta_f32, e + 2, 0.0f);
-            x.w = (x.w - mean) * rstd * load_param(gamma, gamma_f32, e + 3, 1.0f) + load_param(beta, beta_f32, e + 3, 0.0f);
+            x.x = (x.x - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f, f16) +
+                  load_param(beta, beta_f32, e, 0.0f, f16);
+            x.y = (x.y - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f, f16) +
+                  load_param(beta, beta_f32, e + 1, 0.0f, f16);
+            x.z = (x.z - mean) * rstd * load_param(gamma, gamma_f32, e + 2, 1.0f, f16) +
+                  load_param(beta, beta_f32, e + 2, 0.0f, f16);
+            x.w = (x.w - mean) * rstd * load_param(gamma, gamma_f32, e + 3, 1.0f, f16) +
+                  load_param(beta, beta_f32, e + 3, 0.0f, f16);
             vr[i] = x;
         }
     } else {
-        uint4 *vr = reinterpret_cast<uint4 *>(static_cast<__nv_bfloat16 *>(vout) + row * ldv);
+        uint4 *vr = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(vout) + row * ldv);
         for (int i = tid; i < N / 8; i += SM_THREADS) {
             const uint4 x = vr[i];
             const uint32_t w[4] = {x.x, x.y, x.z, x.w};
@@ -289,11 +297,11 @@ layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
                 const int e = i * 8 + 2 * h;
-                const float lo = (bf16_lo(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f) +
-                                 load_param(beta, beta_f32, e, 0.0f);
-                const float hi = (bf16_hi(w[h]) - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f) +
-                                 load_param(beta, beta_f32, e + 1, 0.0f);
-                o[h] = pack_bf16x2(lo, hi);
+                const float lo = (h16_lo(w[h], f16) - mean) * rstd * load_param(gamma, gamma_f32, e, 1.0f, f16) +
+                                 load_param(beta, beta_f32, e, 0.0f, f16);
+                const float hi = (h16_hi(w[h], f16) - mean) * rstd * load_param(gamma, gamma_f32, e + 1, 1.0f, f16) +
+                                 load_param(beta, beta_f32, e + 1, 0.0f, f16);
+                o[h] = pack_h16x2(lo, hi, f16);
             }
             vr[i] = make_uint4(o[0], o[1], o[2], o[3]);
         }
@@ -304,20 +312,20 @@ layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__
 
 cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
                                     int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
-                                    int beta_f32, float eps, cudaStream_t stream)
+                                    int beta_f32, float eps, int f16, cudaStream_t stream)
 {
     if (M <= 0) return cudaSuccess;
     if (out_f32)
         layernorm_finish_kernel<true><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
-                                                                    gamma_f32, beta, beta_f32, eps);
+                                                                    gamma_f32, beta, beta_f32, eps, f16);
     else
         layernorm_finish_kernel<false><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
-                                                                     gamma_f32, beta, beta_f32, eps);
+                                                                     gamma_f32, beta, beta_f32, eps, f16);
     return cudaGetLastError();
 }
 
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
-                                  int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D,
+                                  int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
                                   cudaStream_t stream)
 {
     if (M <= 0) return cudaSuccess;
@@ -325,18 +333,21 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
     if (D <= 32 * LNW_MAX_CHUNKS * 8) {
         const int gk = gamma == nullptr ? 0 : (gamma_f32 ? 2 : 1), bk = beta == nullptr ? 0 : (beta_f32 ? 2 : 1);
         const dim3 grid((M + LNW_WARPS - 1) / LNW_WARPS), block(LNW_WARPS * 32);
-        const __nv_bfloat16 *xp = static_cast<const __nv_bfloat16 *>(x);
-        __nv_bfloat16 *zp = static_cast<__nv_bfloat16 *>(z);
-#define PIKE_LN_CASE(G, B) \
-    if (gk == G && bk == B) layernorm_bf16_warp_kernel<G, B><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D);
+        const uint16_t *xp = static_cast<const uint16_t *>(x);
+        uint16_t *zp = static_cast<uint16_t *>(z);
+#define PIKE_LN_CASE(G, B)                                                                                          \
+    if (gk == G && bk == B) {                                                                                       \
+        if (f16) layernorm_bf16_warp_kernel<G, B, true><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D); \
+        else layernorm_bf16_warp_kernel<G, B, false><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D);   \
+    }
         PIKE_LN_CASE(0, 0) PIKE_LN_CASE(0, 1) PIKE_LN_CASE(0, 2) PIKE_LN_CASE(1, 0) PIKE_LN_CASE(1, 1)
         PIKE_LN_CASE(1, 2) PIKE_LN_CASE(2, 0) PIKE_LN_CASE(2, 1) PIKE_LN_CASE(2, 2)
 #undef PIKE_LN_CASE
         return cudaGetLastError();
     }
-    layernorm_bf16_kernel<<<M, LN_THREADS, 0, stream>>>(static_cast<const __nv_bfloat16 *>(x), ldx,
-                                                         static_cast<__nv_bfloat16 *>(z), ldz, gamma, gamma_f32, beta,
-                                                         beta_f32, eps, D);
+    layernorm_bf16_kernel<<<M, LN_THREADS, 0, stream>>>(static_cast<const uint16_t *>(x), ldx,
+                                                         static_cast<uint16_t *>(z), ldz, gamma, gamma_f32, beta,
+                                                         beta_f32, eps, D, f16);
     return cudaGetLastError();
 }
 

@@ -16,9 +16,10 @@ Generator (counter based, stateless, so any element can be produced alone):
     normal  element i  = sqrt(-2 ln u1(2i)) * cos(2 pi u0(2i+1))   (Box-Muller)
 
 Values are computed in fp64, rounded to fp32 (round-to-nearest-even) and, for
-bf16 tensors, rounded again to bf16 (RNE).  The rounded value *is* the input:
-bf16 tensors are returned as float32 arrays whose low 16 mantissa bits are
-zero, so an fp64 consumer can upcast them exactly.
+16-bit tensors, rounded again to bf16 or to IEEE binary16 ("f16") (RNE).  The
+rounded value *is* the input: 16-bit tensors are returned as float32 arrays
+holding exactly representable values, so an fp64 consumer can upcast them
+exactly.
 
 The paper measures on KernelBench models, whose task files are not reproduced
 here; the five workloads below are synthetic stand-ins with the shapes and
@@ -63,13 +64,23 @@ def round_to_bf16(x32: np.ndarray) -> np.ndarray:
     return rounded.view(np.float32)
 
 
-def _finish(v64: np.ndarray, dtype: str) -> np.ndarray:
-    v32 = v64.astype(np.float32)
+def round_to_f16(x32: np.ndarray) -> np.ndarray:
+    """Round float32 values to the nearest IEEE binary16 (ties to even); result is float32."""
+    return np.ascontiguousarray(x32, dtype=np.float32).astype(np.float16).astype(np.float32)
+
+
+def round_to(x32: np.ndarray, dtype: str) -> np.ndarray:
     if dtype == "bf16":
-        return round_to_bf16(v32)
+        return round_to_bf16(x32)
+    if dtype == "f16":
+        return round_to_f16(x32)
     if dtype == "f32":
-        return v32
-    raise ValueError(f"dtype must be 'f32' or 'bf16', got {dtype!r}")
+        return np.ascontiguousarray(x32, dtype=np.float32)
+    raise ValueError(f"dtype must be 'f32', 'bf16' or 'f16', got {dtype!r}")
+
+
+def _finish(v64: np.ndarray, dtype: str) -> np.ndarray:
+    return round_to(v64.astype(np.float32), dtype)
 
 
 def uniform(shape, a: float, *, seed: int, tensor_id: int, dtype: str) -> np.ndarray:
@@ -117,74 +128,74 @@ def config1(M=128, K=256, N=256, seed=0):
     )
 
 
-def config2(M=4096, K=4096, N=4096, seed=0):
-    """bf16 Linear + bias + SiLU + scale(0.5) + residual."""
+def config2(M=4096, K=4096, N=4096, seed=0, dtype="bf16"):
+    """16-bit (bf16 unless dtype="f16") Linear + bias + SiLU + scale(0.5) + residual."""
     return dict(
-        x=normal((M, K), seed=seed, tensor_id=11, dtype="bf16"),
-        w=uniform((K, N), 1.0 / 64, seed=seed, tensor_id=12, dtype="bf16"),
-        b=uniform((N,), 1.0 / 64, seed=seed, tensor_id=13, dtype="bf16"),
-        r=normal((M, N), seed=seed, tensor_id=14, dtype="bf16"),
+        x=normal((M, K), seed=seed, tensor_id=11, dtype=dtype),
+        w=uniform((K, N), 1.0 / 64, seed=seed, tensor_id=12, dtype=dtype),
+        b=uniform((N,), 1.0 / 64, seed=seed, tensor_id=13, dtype=dtype),
+        r=normal((M, N), seed=seed, tensor_id=14, dtype=dtype),
         scale=0.5,
     )
 
 
-def config3(M=8192, D=4096, F=16384, seed=0, affine=False):
-    """bf16 pre-LN transformer MLP block; weights U(+-1/sqrt(fan_in))."""
+def config3(M=8192, D=4096, F=16384, seed=0, affine=False, dtype="bf16"):
+    """16-bit pre-LN transformer MLP block; weights U(+-1/sqrt(fan_in))."""
     if affine:
-        gamma = 1.0 + uniform((D,), 0.5, seed=seed, tensor_id=26, dtype="bf16")
-        beta = uniform((D,), 0.1, seed=seed, tensor_id=27, dtype="bf16")
-        gamma = round_to_bf16(gamma.astype(np.float32))
+        gamma = 1.0 + uniform((D,), 0.5, seed=seed, tensor_id=26, dtype=dtype)
+        beta = uniform((D,), 0.1, seed=seed, tensor_id=27, dtype=dtype)
+        gamma = round_to(gamma.astype(np.float32), dtype)
     else:
         gamma = np.ones((D,), np.float32)
         beta = np.zeros((D,), np.float32)
     return dict(
-        x=normal((M, D), seed=seed, tensor_id=21, dtype="bf16"),
-        w1=uniform((D, F), 1.0 / np.sqrt(D), seed=seed, tensor_id=22, dtype="bf16"),
-        b1=uniform((F,), 1.0 / np.sqrt(D), seed=seed, tensor_id=23, dtype="bf16"),
-        w2=uniform((F, D), 1.0 / np.sqrt(F), seed=seed, tensor_id=24, dtype="bf16"),
-        b2=uniform((D,), 1.0 / np.sqrt(F), seed=seed, tensor_id=25, dtype="bf16"),
+        x=normal((M, D), seed=seed, tensor_id=21, dtype=dtype),
+        w1=uniform((D, F), 1.0 / np.sqrt(D), seed=seed, tensor_id=22, dtype=dtype),
+        b1=uniform((F,), 1.0 / np.sqrt(D), seed=seed, tensor_id=23, dtype=dtype),
+        w2=uniform((F, D), 1.0 / np.sqrt(F), seed=seed, tensor_id=24, dtype=dtype),
+        b2=uniform((D,), 1.0 / np.sqrt(F), seed=seed, tensor_id=25, dtype=dtype),
         gamma=gamma, beta=beta, eps=1e-5,
     )
 
 
-def config4(M=2048, K=4096, N=32000, seed=0):
-    """bf16 logits GEMM + fp32 row softmax."""
+def config4(M=2048, K=4096, N=32000, seed=0, dtype="bf16"):
+    """16-bit logits GEMM + fp32 row softmax."""
     return dict(
-        x=normal((M, K), seed=seed, tensor_id=31, dtype="bf16"),
-        w=uniform((K, N), 1.0 / 64, seed=seed, tensor_id=32, dtype="bf16"),
+        x=normal((M, K), seed=seed, tensor_id=31, dtype=dtype),
+        w=uniform((K, N), 1.0 / 64, seed=seed, tensor_id=32, dtype=dtype),
     )
 
 
-def config5(B=8, H=32, S=2048, D=128, seed=0):
-    """bf16 causal attention."""
+def config5(B=8, H=32, S=2048, D=128, seed=0, dtype="bf16"):
+    """16-bit causal attention."""
     return dict(
-        q=normal((B, H, S, D), seed=seed, tensor_id=41, dtype="bf16"),
-        k=normal((B, H, S, D), seed=seed, tensor_id=42, dtype="bf16"),
-        v=normal((B, H, S, D), seed=seed, tensor_id=43, dtype="bf16"),
+        q=normal((B, H, S, D), seed=seed, tensor_id=41, dtype=dtype),
+        k=normal((B, H, S, D), seed=seed, tensor_id=42, dtype=dtype),
+        v=normal((B, H, S, D), seed=seed, tensor_id=43, dtype=dtype),
         scale=1.0 / np.sqrt(D),
     )
 
 
-def attention_block(B=4, S=1024, E=2048, seed=0, affine=True):
-    """bf16 pre-LN attention block with fused projections (heads of 128); weights U(+-1/sqrt(E))."""
+def attention_block(B=4, S=1024, E=2048, seed=0, affine=True, dtype="bf16"):
+    """16-bit pre-LN attention block with fused projections (heads of 128); weights U(+-1/sqrt(E))."""
     a = 1.0 / np.sqrt(E)
     if affine:
-        gamma = round_to_bf16((1.0 + uniform((E,), 0.5, seed=seed, tensor_id=56, dtype="bf16")).astype(np.float32))
-        beta = uniform((E,), 0.1, seed=seed, tensor_id=57, dtype="bf16")
+        gamma = round_to((1.0 + uniform((E,), 0.5, seed=seed, tensor_id=56, dtype=dtype)).astype(np.float32), dtype)
+        beta = uniform((E,), 0.1, seed=seed, tensor_id=57, dtype=dtype)
     else:
         gamma, beta = np.ones((E,), np.float32), np.zeros((E,), np.float32)
     return dict(
-        x=normal((B, S, E), seed=seed, tensor_id=51, dtype="bf16"),
-        w_qkv=uniform((E, 3 * E), a, seed=seed, tensor_id=52, dtype="bf16"),
-        b_qkv=uniform((3 * E,), a, seed=seed, tensor_id=53, dtype="bf16"),
-        w_o=uniform((E, E), a, seed=seed, tensor_id=54, dtype="bf16"),
-        b_o=uniform((E,), a, seed=seed, tensor_id=55, dtype="bf16"),
+        x=normal((B, S, E), seed=seed, tensor_id=51, dtype=dtype),
+        w_qkv=uniform((E, 3 * E), a, seed=seed, tensor_id=52, dtype=dtype),
+        b_qkv=uniform((3 * E,), a, seed=seed, tensor_id=53, dtype=dtype),
+        w_o=uniform((E, E), a, seed=seed, tensor_id=54, dtype=dtype),
+        b_o=uniform((E,), a, seed=seed, tensor_id=55, dtype=dtype),
         gamma=gamma, beta=beta, eps=1e-5, scale=1.0 / np.sqrt(128.0), num_heads=E // 128,
     )
 
 
-def grouped_linear(T=16384, K=2048, N=4096, G=32, seed=0):
-    """bf16 mixture-of-experts style grouped linear: T rows split over G groups of uneven size (one group is
+def grouped_linear(T=16384, K=2048, N=4096, G=32, seed=0, dtype="bf16"):
+    """16-bit mixture-of-experts style grouped linear: T rows split over G groups of uneven size (one group is
     empty, sizes are not multiples of the tile), weights U(+-1/sqrt(K))."""
     a = 1.0 / np.sqrt(K)
     # group sizes: seeded uniform weights, one group forced empty, remainder to the last group
@@ -195,9 +206,9 @@ def grouped_linear(T=16384, K=2048, N=4096, G=32, seed=0):
     sizes[-1] += T - sizes.sum()
     offsets = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
     return dict(
-        x=normal((T, K), seed=seed, tensor_id=61, dtype="bf16"),
-        w=uniform((G, K, N), a, seed=seed, tensor_id=62, dtype="bf16"),
-        b=uniform((G, N), a, seed=seed, tensor_id=63, dtype="bf16"),
-        r=normal((T, N), seed=seed, tensor_id=64, dtype="bf16"),
+        x=normal((T, K), seed=seed, tensor_id=61, dtype=dtype),
+        w=uniform((G, K, N), a, seed=seed, tensor_id=62, dtype=dtype),
+        b=uniform((G, N), a, seed=seed, tensor_id=63, dtype=dtype),
+        r=normal((T, N), seed=seed, tensor_id=64, dtype=dtype),
         offsets=offsets,
     )

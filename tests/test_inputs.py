@@ -41,6 +41,22 @@ def test_bf16_values_are_representable_and_nearest_even():
     assert np.array_equal(G.round_to_bf16(t), np.array([1.0, 1 + 2.0 ** -6], np.float32))
 
 
+def test_f16_values_are_representable_and_nearest_even():
+    z = G.normal((4096,), seed=0, tensor_id=1, dtype="f16")
+    # a binary16 normal number has 11 significant bits: the low 13 bits of the fp32 mantissa are zero
+    normal = np.abs(z) >= 2.0 ** -14
+    assert normal.mean() > 0.99 and (z[normal].view(np.uint32) & 0x1FFF == 0).all()
+    f = G.normal((4096,), seed=0, tensor_id=1, dtype="f32")
+    assert np.abs(z - f).max() <= np.abs(f).max() * 2.0 ** -11
+    # ties to even: 1 + 2^-11 -> 1, 1 + 3*2^-11 -> 1 + 2^-9; 2049 -> 2048, 2051 -> 2052
+    t = np.array([1 + 2.0 ** -11, 1 + 3 * 2.0 ** -11, 2049, 2051], np.float32)
+    assert np.array_equal(G.round_to_f16(t), np.array([1.0, 1 + 2.0 ** -9, 2048, 2052], np.float32))
+    # the same draw rounded to bf16 is a different tensor: the two 16-bit recipes are distinct inputs
+    assert (G.normal((4096,), seed=0, tensor_id=1, dtype="bf16") != z).mean() > 0.5
+    c = G.config3(M=4, D=8, F=16, affine=True, dtype="f16")
+    assert np.array_equal(G.round_to_f16(c["gamma"]), c["gamma"]) and np.array_equal(G.round_to_f16(c["w1"]), c["w1"])
+
+
 def test_config_shapes():
     c1 = G.config1()
     assert c1["x"].shape == (128, 256) and c1["w"].shape == (256, 256) and c1["b"].shape == (256,)
