@@ -53,6 +53,9 @@ def flops_per_config():
         "X1": 2.0 * 16384 * 4096 * (3 * 4096) + 4.0 * 8 * 32 * 128 * (2048 * 2049 / 2) + 2.0 * 16384 * 4096 * 4096,
         # X2 (not part of the default step): grouped linear + SiLU, 16384 rows over 32 weight matrices 2048 x 4096
         "X2": 2.0 * 16384 * 2048 * 4096,
+        # X3 (not part of the default step): C4's logits + softmax with the 32000 columns split over the ranks
+        # (whole-job flops; every rank does 1/world of them)
+        "X3": 2.0 * 2048 * 4096 * 32000,
     }
 
 
@@ -152,7 +155,7 @@ def oracle_sample_text():
 
 
 ALL = ("C1", "C2", "C3", "C4", "C5")          # the step
-EXTRA = ("X1", "X2")                         # further workloads, only with --only
+EXTRA = ("X1", "X2", "X3")                   # further workloads, only with --only
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -174,7 +177,8 @@ def job_tflops(step_flops: float, world: int, ms_per_step: float) -> float:
 def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
-           "X1": lambda: G.attention_block(B=8, S=2048, E=4096), "X2": G.grouped_linear}
+           "X1": lambda: G.attention_block(B=8, S=2048, E=4096), "X2": G.grouped_linear,
+           "X3": G.config4}
     return {k: gen[k]() for k in only}
 
 
@@ -232,6 +236,8 @@ def run_ours(args):
     only = args.only
     inputs = make_inputs(only)
     f = {k: v for k, v in flops_per_config().items() if k in only}
+    if "X3" in f:
+        f["X3"] /= world          # strong scaling: job_tflops multiplies the per-rank flops by world again
 
     # ---- host (pinned) and device copies --------------------------------------------
     def pin(a, dtype):
@@ -264,14 +270,23 @@ def run_ours(args):
     if x2:
         host_act.update(x2x=pin(x2["x"], BF16))
         wts.update(x2w=pin(x2["w"], BF16), x2b=pin(x2["b"], BF16))
+    x3 = inputs.get("X3")
+    x3_cols = (0, 0)
+    if x3:
+        x3_cols = P.vocab_shard_range(32000, rank, world)
+        host_act.update(x3x=pin(x3["x"], BF16))
+        wts.update(x3w=pin(x3["w"][:, x3_cols[0]:x3_cols[1]], BF16))
     d = {k: v.to(device) for k, v in host_act.items()}
     d.update({k: v.to(device) for k, v in wts.items()})
     shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
-              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16), "X2": ((16384, 4096), BF16)}
+              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16), "X2": ((16384, 4096), BF16),
+              "X3": ((2048, x3_cols[1] - x3_cols[0]), F32)}
     out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in only}
     host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
     ws0 = torch.empty(256, dtype=torch.uint8, device=device)
-    ws3 = ws4 = wsx = ws0
+    ws3 = ws4 = wsx = wsx3 = ws0
+    if x3:
+        wsx3 = torch.empty(P.pike_linear_softmax_shard_workspace(d["x3x"], d["x3w"]), dtype=torch.uint8, device=device)
     if x1:
         wsx = torch.empty(P.pike_attention_block_workspace(d["x1x"], scale=float(x1["scale"])), dtype=torch.uint8,
                           device=device)
@@ -298,6 +313,8 @@ def run_ours(args):
                                              workspace=wsx),
         "X2": lambda: P.pike_grouped_linear_epilogue(d["x2x"], d["x2w"], d["x2b"], None, x2off, act="silu",
                                                      out=out["X2"]),
+        # the exchange between the two library calls is an all-gather of 16 KiB per rank over the default group
+        "X3": lambda: P.linear_softmax_vocab_sharded(d["x3x"], d["x3w"], out=out["X3"], workspace=wsx3),
     }
     names = [n for n in chains if n in only]
 
@@ -381,7 +398,7 @@ def run_ours(args):
     gemm_flops = sum(f.get(k, 0.0) for k in ("C2", "C3", "C4"))      # the launches of the bf16 GEMM kernel
     if "X1" in f:
         gemm_flops += 2.0 * 16384 * 4096 * (4 * 4096)
-    gemm_flops += f.get("X2", 0.0)
+    gemm_flops += f.get("X2", 0.0) + f.get("X3", 0.0)
     gemm_tflops = gemm_flops * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     # a long timed region runs under the power cap: compare with the sustained library figure
     sustained = total_ms > 500.0 or "sw_power_cap" in (clocks or {}).get("reasons", [])
@@ -400,6 +417,8 @@ def run_ours(args):
 
     if x2:
         d["x2off_host"] = [int(o) for o in x2["offsets"]]
+    if x3 and not args.no_eager:   # the eager comparison is the unsharded chain on one GPU
+        d["x3w_full"] = pin(x3["w"], BF16).to(device)
     eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5 or x1, names)
     library_gemm = None if args.no_eager else library_gemm_context(torch, device, sampler.__class__(local_rank))
     if tuple(only) != ALL:
@@ -424,7 +443,8 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if tuple(only) == ("X3",) else "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": ("" if tuple(only) == ALL else "SUBSET " + ",".join(only) + " of the ") +
                                "C1-C5 chain suite (fp32 linear+GELU+LN 128x256x256; bf16 linear+SiLU+scale+residual "
@@ -472,6 +492,7 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         "C5": attn,
         "X1": lambda: x1_eager(),
         "X2": lambda: x2_eager(),
+        "X3": lambda: torch.softmax(d["x3x"] @ d["x3w_full"], dim=-1, dtype=torch.float32),
     }
 
     def x2_eager():     # the per-expert loop the grouped kernel replaces
@@ -578,7 +599,7 @@ def main():
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--only", type=lambda v: tuple(x for x in ALL + EXTRA if x in v.split(",")), default=ALL,
-                    help="comma-separated subset of C1..C5 and X1 (profiling runs; the default is the whole suite C1..C5)")
+                    help="comma-separated subset of C1..C5 and X1..X3 (profiling runs; the default is the whole suite C1..C5)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-eager", action="store_true")
     ap.add_argument("--no-parity", action="store_true")

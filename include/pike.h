@@ -171,6 +171,45 @@ pike_status_t pike_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x,
                                    size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Logits + row softmax with the columns split over several GPUs (the paper's "Future Work" section names
+ * multi-GPU inference as the next step for these chains; a vocabulary projection is the chain whose
+ * weight is sharded column-wise in practice).  GPU r of R holds the column slice w_r [K,N_r] (and bias_r)
+ * and every GPU holds the same x [M,K]; together they compute
+ *
+ *   out[m, slice r] = exp(v[m,n] - max_n v[m,:]) / sum_n exp(v[m,n] - max_n v[m,:]),
+ *   v[m,n] = scale * act( sum_k x[m,k] * w[k,n] + bias[n] )
+ *
+ * with the maximum and the sum taken over ALL N = sum_r N_r columns.  Two calls per GPU with one
+ * exchange between them (the only data that crosses GPUs is one (max, sum) pair per row and GPU):
+ *
+ *  1. pike_linear_softmax_shard_local: out_r [M,N_r] F32 receives the un-normalised v of this slice and
+ *     row_stats[m] = ( max_n v[m, slice r], sum_n exp(v[m,n] - that max) ), M pairs of floats in DEVICE
+ *     memory (8-byte aligned).  Same kernels, dtypes (x, w both BF16 or both F16; bias that type or F32 or
+ *     NULL) and envelope (K, N_r multiples of 8) as pike_linear_epilogue with reduce == SOFTMAX;
+ *     epi->reduce must be PIKE_REDUCE_SOFTMAX and epi->out_dtype PIKE_F32.  Workspace as returned by
+ *     pike_linear_softmax_shard_workspace (the per-tile pairs).
+ *  2. The caller gathers every GPU's row_stats into all_stats [R, M] pairs, shard-major - exactly what an
+ *     all-gather of the R row_stats arrays produces (8*M bytes per GPU; NCCL or any other transport;
+ *     the library itself does no communication).
+ *  3. pike_linear_softmax_shard_finish: combines the R pairs of each row,
+ *     m = max_r m_r, l = sum_r l_r * exp(m_r - m), and overwrites out_r with exp(out_r - m) / l.
+ *     all_stats is DEVICE memory, 8-byte aligned; num_shards = R >= 1.  out_r must still hold the values
+ *     step 1 wrote.  With R == 1 the two calls compute the same result as pike_linear_epilogue.
+ *
+ * The order of the shards in all_stats does not matter (max and sum commute), but every GPU must use the
+ * same x, scale, act and a disjoint slice of the columns.  Errors as for pike_linear_epilogue.
+ */
+pike_status_t pike_linear_softmax_shard_workspace(pike_handle_t handle, const pike_tensor_t *x,
+                                                  const pike_tensor_t *w, const pike_epilogue_t *epi,
+                                                  size_t *bytes);
+pike_status_t pike_linear_softmax_shard_local(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
+                                              const pike_tensor_t *bias, const pike_epilogue_t *epi,
+                                              pike_tensor_t *out, float *row_stats, void *workspace,
+                                              size_t workspace_bytes, void *cuda_stream);
+pike_status_t pike_linear_softmax_shard_finish(pike_handle_t handle, pike_tensor_t *out, const float *all_stats,
+                                               int32_t num_shards, void *cuda_stream);
+
+/*
  * Logits + row softmax for callers that cannot allocate device memory.  (The paper has
  * no counterpart to this entry point; it exists for how the library gets embedded.)
  *

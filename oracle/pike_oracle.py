@@ -218,3 +218,21 @@ def grouped_linear_epilogue(x, w, bias, residual, offsets, *, act="none", scale=
                                          None if residual is None else np.asarray(residual)[lo:hi],
                                          act=act, scale=scale)
     return out
+
+
+def softmax_shard_stats(x, w_shard, bias_shard=None, *, act="none", scale=1.0, rows=None):
+    """One GPU's half of a softmax whose columns are split over GPUs: the un-normalised values
+    v = scale*act(x @ w_shard + bias_shard) of the slice and, per row, (max_n v, sum_n exp(v - max))."""
+    v = linear_epilogue(x, w_shard, bias_shard, act=act, scale=scale, rows=rows)
+    m = v.max(axis=1)
+    l = np.exp(v - m[:, None]).sum(axis=1)
+    return v, np.stack([m, l], axis=1)
+
+
+def softmax_shard_finish(v, all_stats):
+    """Second half: all_stats [R,M,2] holds every slice's (max, sum) per row;
+    m = max_r m_r, l = sum_r l_r*exp(m_r - m), result exp(v - m)/l for this slice's columns."""
+    all_stats = _f64(all_stats)
+    m = all_stats[:, :, 0].max(axis=0)
+    l = (all_stats[:, :, 1] * np.exp(all_stats[:, :, 0] - m[None, :])).sum(axis=0)
+    return np.exp(_f64(v) - m[:, None]) / l[:, None]

@@ -26,7 +26,8 @@ EXPORTS = (
     "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
     "pike_attention_chain", "pike_linear_softmax_noalloc", "pike_attention_block_workspace", "pike_attention_block",
-    "pike_grouped_linear_epilogue",
+    "pike_grouped_linear_epilogue", "pike_linear_softmax_shard_workspace", "pike_linear_softmax_shard_local",
+    "pike_linear_softmax_shard_finish",
 )
 
 
@@ -86,6 +87,9 @@ def load_library() -> ctypes.CDLL:
             lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
             lib.pike_linear_epilogue.argtypes = [vp, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_linear_softmax_noalloc.argtypes = [vp, T, T, T, E, T, vp]
+            lib.pike_linear_softmax_shard_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
+            lib.pike_linear_softmax_shard_local.argtypes = [vp, T, T, T, E, T, vp, vp, sz, vp]
+            lib.pike_linear_softmax_shard_finish.argtypes = [vp, T, vp, ctypes.c_int32, vp]
             lib.pike_mlp_block_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
             lib.pike_mlp_block.argtypes = [vp, T, T, T, T, T, T, T, E, T, vp, sz, vp]
             lib.pike_attention_chain_workspace.argtypes = [vp, T, E, ctypes.POINTER(sz)]
@@ -233,6 +237,51 @@ def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, 
                                                _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
                                                _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
            "pike_linear_epilogue")
+    return out
+
+
+def pike_linear_softmax_shard_workspace(x, w, *, act="none", scale=1.0, w_is_nk=False) -> int:
+    e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
+    n = ctypes.c_size_t(0)
+    _check(load_library().pike_linear_softmax_shard_workspace(_handle(x.device), _tensor(x), _tensor(w),
+                                                              ctypes.byref(e), ctypes.byref(n)),
+           "pike_linear_softmax_shard_workspace")
+    return n.value
+
+
+def pike_linear_softmax_shard_local(x, w, bias=None, *, act="none", scale=1.0, w_is_nk=False, out=None,
+                                    row_stats=None, workspace=None, stream=None):
+    """First half of a softmax whose columns are split over GPUs: this GPU's un-normalised slice
+    out [M,N_r] fp32 and row_stats [M,2] fp32 = (max, sum exp) of the slice; see include/pike.h."""
+    N = w.shape[0] if w_is_nk else w.shape[1]
+    if out is None:
+        out = torch.empty((x.shape[0], N), dtype=torch.float32, device=x.device)
+    if row_stats is None:
+        row_stats = torch.empty((x.shape[0], 2), dtype=torch.float32, device=x.device)
+    if row_stats.dtype != torch.float32 or not row_stats.is_cuda or not row_stats.is_contiguous() \
+            or row_stats.numel() != 2 * x.shape[0]:
+        raise TypeError("row_stats must be a contiguous CUDA float32 tensor of M pairs")
+    e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
+    need = pike_linear_softmax_shard_workspace(x, w, act=act, scale=scale, w_is_nk=w_is_nk)
+    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    _check(load_library().pike_linear_softmax_shard_local(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
+                                                          ctypes.byref(e), _tensor(out),
+                                                          ctypes.c_void_p(row_stats.data_ptr()), ws_ptr, ws_bytes,
+                                                          _stream(stream)),
+           "pike_linear_softmax_shard_local")
+    return out, row_stats
+
+
+def pike_linear_softmax_shard_finish(out, all_stats, *, stream=None):
+    """Second half: all_stats [R,M,2] fp32 (every GPU's row_stats, gathered shard-major) normalises this
+    GPU's slice `out` in place; see include/pike.h."""
+    if all_stats.dtype != torch.float32 or not all_stats.is_cuda or not all_stats.is_contiguous() \
+            or all_stats.dim() != 3 or all_stats.shape[1] != out.shape[0] or all_stats.shape[2] != 2:
+        raise TypeError("all_stats must be a contiguous CUDA float32 tensor [R, M, 2]")
+    _check(load_library().pike_linear_softmax_shard_finish(_handle(out.device), _tensor(out),
+                                                           ctypes.c_void_p(all_stats.data_ptr()),
+                                                           int(all_stats.shape[0]), _stream(stream)),
+           "pike_linear_softmax_shard_finish")
     return out
 
 

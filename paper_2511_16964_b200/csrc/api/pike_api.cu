@@ -455,6 +455,81 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
     return PIKE_OK;
 }
 
+// Validation shared by the two halves of the column-sharded softmax.
+static pike_status_t shard_shape(const pike_tensor_t *x, const pike_tensor_t *w, const pike_epilogue_t *epi,
+                                 LinearShape &s)
+{
+    if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
+    if (s.fp32_path) return PIKE_ERR_DTYPE;
+    if (epi->reduce != PIKE_REDUCE_SOFTMAX || epi->out_dtype != PIKE_F32) return PIKE_ERR_UNSUPPORTED;
+    return PIKE_OK;
+}
+
+pike_status_t pike_linear_softmax_shard_workspace(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
+                                                  const pike_epilogue_t *epi, size_t *bytes)
+{
+    if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
+    LinearShape s;
+    if (pike_status_t st = shard_shape(x, w, epi, s)) return st;
+    *bytes = softmax_partials_bytes(s);
+    return PIKE_OK;
+}
+
+pike_status_t pike_linear_softmax_shard_local(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
+                                              const pike_tensor_t *bias, const pike_epilogue_t *epi,
+                                              pike_tensor_t *out, float *row_stats, void *workspace,
+                                              size_t workspace_bytes, void *cuda_stream)
+{
+    if (h == nullptr || out == nullptr || row_stats == nullptr) return PIKE_ERR_NULL;
+    LinearShape s;
+    if (pike_status_t st = shard_shape(x, w, epi, s)) return st;
+    if (pike_status_t st = check_matrix(x, s.M, s.K)) return st;
+    if (pike_status_t st = check_matrix(w, s.w_is_nk ? s.N : s.K, s.w_is_nk ? s.K : s.N)) return st;
+    if (pike_status_t st = check_matrix(out, s.M, s.N)) return st;
+    if (out->dtype != PIKE_F32) return PIKE_ERR_DTYPE;
+    if (pike_status_t st = check_vector(bias, s.N)) return st;
+    if (!side_ok(bias, x->dtype)) return PIKE_ERR_DTYPE;
+    if (reinterpret_cast<uintptr_t>(row_stats) % 8 != 0) return PIKE_ERR_ALIGNMENT;
+    for (const pike_tensor_t *t : {x, w, bias})
+        if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
+    const size_t need = softmax_partials_bytes(s);
+    if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 || workspace_bytes < need)
+        return PIKE_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    if (s.M == 0) return PIKE_OK;
+    float2 *partials = static_cast<float2 *>(workspace);
+    if (pike_status_t st = run_gemm(h, x->data, x->stride[0], w, s.w_is_nk, s.M, s.K, s.N, bias, nullptr, false, 0,
+                                    out->data, true, out->stride[0], (int)epi->act, epi->scale, partials, stream, 1))
+        return st;
+    const int num_n = (int)((s.N + pike::GEMM_BN - 1) / pike::GEMM_BN);
+    TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
+    return pike::launch_softmax_row_stats(partials, num_n, reinterpret_cast<float2 *>(row_stats), (int)s.M,
+                                          stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+pike_status_t pike_linear_softmax_shard_finish(pike_handle_t h, pike_tensor_t *out, const float *all_stats,
+                                               int32_t num_shards, void *cuda_stream)
+{
+    if (h == nullptr || out == nullptr || all_stats == nullptr) return PIKE_ERR_NULL;
+    if (num_shards < 1) return PIKE_ERR_SHAPE;
+    if (out->ndim != 2 || out->shape[0] < 0 || out->shape[1] < 1) return PIKE_ERR_SHAPE;
+    if (out->shape[0] > 0x7fffffff || out->shape[1] > 0x7fffffff) return PIKE_ERR_UNSUPPORTED;
+    if (out->shape[1] % 8 != 0) return PIKE_ERR_UNSUPPORTED;
+    if (pike_status_t st = check_matrix(out, out->shape[0], out->shape[1])) return st;
+    if (out->dtype != PIKE_F32) return PIKE_ERR_DTYPE;
+    if (reinterpret_cast<uintptr_t>(all_stats) % 8 != 0) return PIKE_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
+    const int64_t M = out->shape[0];
+    if (M == 0) return PIKE_OK;
+    TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
+    // pair of (row m, shard r) at all_stats[(r*M + m)*2]: row stride 1 pair, "tile" stride M pairs
+    return pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0],
+                                       reinterpret_cast<const float2 *>(all_stats), (int)num_shards, (int)M,
+                                       (int)out->shape[1], stream, 1, M) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
 pike_status_t pike_grouped_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
                                            const pike_tensor_t *bias, const pike_tensor_t *residual,
                                            const int32_t *group_offsets, const pike_epilogue_t *epi, pike_tensor_t *out,

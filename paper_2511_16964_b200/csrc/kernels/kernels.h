@@ -59,8 +59,12 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
                                   cudaStream_t stream);
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
+// Pair t of row m sits at partials[m*pair_row_stride + t*pair_tile_stride] (pair_row_stride 0 = num_n_tiles,
+// the layout the GEMM epilogue writes; {1, M} reads pairs stored [t][m], as an all-gather over GPUs lays them).
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, long long pair_row_stride = 0, long long pair_tile_stride = 1);
+// stats[m] = the row's per-tile (max, sum exp) pairs [M, num_n_tiles] folded into one pair
+cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream);
 
 // out = (v - mean)/sqrt(var + eps)*gamma + beta in place (v 16-bit or f32), statistics combined from the
 // per-(row, n-tile) (mean, sum of squared deviations) pairs; tile_n = columns per tile

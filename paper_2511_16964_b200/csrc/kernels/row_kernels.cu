@@ -193,15 +193,16 @@ constexpr int SM_THREADS = 256;
 // then p = exp(v - m) / l in place (one read and one write of the row).
 __global__ void __launch_bounds__(SM_THREADS)
 softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__restrict__ partials, int num_n_tiles,
-                      int N)
+                      long long pair_row_stride, long long pair_tile_stride, int N)
 {
     __shared__ float red[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long row = blockIdx.x;
-    const float2 *pr = partials + row * num_n_tiles;
+    // pair t of this row; [row][tile] for one GEMM's tiles, [shard][row] for pairs gathered from other GPUs
+    const float2 *pr = partials + row * pair_row_stride;
 
     float m = -INFINITY;
-    for (int t = tid; t < num_n_tiles; t += SM_THREADS) m = fmaxf(m, pr[t].x);
+    for (int t = tid; t < num_n_tiles; t += SM_THREADS) m = fmaxf(m, pr[t * pair_tile_stride].x);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if (lane == 0) red[warp] = m;
@@ -213,7 +214,7 @@ softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__rest
 
     float l = 0.0f;
     for (int t = tid; t < num_n_tiles; t += SM_THREADS) {
-        const float2 pt = pr[t];
+        const float2 pt = pr[t * pair_tile_stride];
         l += pt.y * expf(pt.x - m);
     }
 #pragma unroll
@@ -234,6 +235,32 @@ softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__rest
         a.w = expf(a.w - m) * inv;
         vr[i] = a;
     }
+}
+
+constexpr int STATS_THREADS = 256;
+
+// One warp per row: fold the row's per-tile (max, sum exp) pairs into one pair for the whole row,
+//   m = max_t m_t,  l = sum_t l_t * exp(m_t - m),
+// the statistics a GPU publishes for its slice of the columns when a softmax is split over several GPUs.
+__global__ void __launch_bounds__(STATS_THREADS)
+softmax_row_stats_kernel(const float2 *__restrict__ partials, int num_n_tiles, float2 *__restrict__ stats, int M)
+{
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * (STATS_THREADS / 32) + (threadIdx.x >> 5);
+    if (row >= M) return;
+    const float2 *pr = partials + row * num_n_tiles;
+    float m = -INFINITY;
+    for (int t = lane; t < num_n_tiles; t += 32) m = fmaxf(m, pr[t].x);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float l = 0.0f;
+    for (int t = lane; t < num_n_tiles; t += 32) {
+        const float2 pt = pr[t];
+        l += pt.y * expf(pt.x - m);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) stats[row] = make_float2(m, l);
 }
 
 // Second half of a LayerNorm split across GEMM tiles.  One CTA per row: combine the per-tile
@@ -352,10 +379,21 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
 }
 
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
-                                  cudaStream_t stream)
+                                  cudaStream_t stream, long long pair_row_stride, long long pair_tile_stride)
 {
     if (M <= 0) return cudaSuccess;
-    softmax_finish_kernel<<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, N);
+    if (pair_row_stride == 0) pair_row_stride = num_n_tiles;
+    softmax_finish_kernel<<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, pair_row_stride,
+                                                        pair_tile_stride, N);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream)
+{
+    if (M <= 0) return cudaSuccess;
+    const int rows_per_block = STATS_THREADS / 32;
+    softmax_row_stats_kernel<<<(M + rows_per_block - 1) / rows_per_block, STATS_THREADS, 0, stream>>>(
+        partials, num_n_tiles, stats, M);
     return cudaGetLastError();
 }
 
