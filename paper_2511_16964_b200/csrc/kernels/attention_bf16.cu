@@ -16,9 +16,11 @@
 //            A operand straight from tensor memory
 //   O_t   += P_t(j) V_j     V is the MN-major B operand; accumulates in tensor memory
 // The MMA warp interleaves the two tiles (PV0, S0', PV1, S1', ...) so one tile's softmax
-// runs under the other tile's MMAs.  The running maximum is only raised when it grows by
-// more than 2^8 (probabilities stay bounded by 256 in between), so rescaling O in tensor
-// memory is rare; it is done by the softmax threads themselves between two PV MMAs.
+// runs under the other tile's MMAs.  P_t(j) is handed over in two halves of 64 keys (p_full, then
+// p_half2): the first four PV MMAs run while the second half's exponentials are still being computed.
+// The running maximum is only raised when it grows by more than 2^8 (probabilities stay bounded by
+// 256 in between), so rescaling O in tensor memory is rare; it is done by the softmax threads
+// themselves between two PV MMAs.
 // Causal masking comes from indices on the diagonal tile only; tiles above the diagonal
 // are never loaded.  Register budgets are re-partitioned
 // with setmaxnreg (104 for WG0, 200 for the softmax warpgroups; 384 x 168 at launch).
@@ -44,20 +46,45 @@ struct __align__(8) Ctrl {
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
     uint64_t q_empty;
-    uint64_t s_full[2], p_full[2];
+    uint64_t s_full[2], p_full[2], p_half2[2];   // p_full: keys 0..63 of P_t written, p_half2: keys 64..127
     uint64_t o_final[2], o_free[2];
     uint32_t tmem_base;
     uint32_t abort;
 };
 constexpr size_t SMEM_BYTES = 1024 + (size_t)TILE_BYTES * (2 + 2 * KV_STAGES) + sizeof(Ctrl);
 
-enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FINAL, BAR_Q_EMPTY, BAR_O_FREE };
+enum : uint32_t { BAR_Q = 1, BAR_K_EMPTY, BAR_V_EMPTY, BAR_K_FULL, BAR_V_FULL, BAR_S_FULL, BAR_P_FULL, BAR_O_FINAL, BAR_Q_EMPTY, BAR_O_FREE, BAR_P_HALF2 };
 
 __device__ __forceinline__ float ex2(float x)
 {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// Two fp32 lanes per instruction (sm_100 packed arithmetic): halves the issue slots the scale-and-shift
+// and the row sums take in the softmax loop, which is bound by instruction issue, not by a pipe.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
 }
 
 // F16 = the tensors are IEEE half instead of bf16 (operand format of both MMAs, P and the output).
@@ -112,7 +139,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         mbar_init(&ctrl->q_empty, 1);
         for (int t = 0; t < 2; ++t) {
-            mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], SOFTMAX_THREADS);
+            mbar_init(&ctrl->s_full[t], 1); mbar_init(&ctrl->p_full[t], SOFTMAX_THREADS); mbar_init(&ctrl->p_half2[t], SOFTMAX_THREADS);
             mbar_init(&ctrl->o_final[t], 1); mbar_init(&ctrl->o_free[t], SOFTMAX_THREADS);
         }
         ctrl->abort = 0;
@@ -207,15 +234,17 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 }
                 __syncwarp();
             };
-            // O_t (+)= P_t V (V tile in ring stage vs): A = bf16 P in TMEM (8 columns per 16 keys)
-            auto issue_pv = [&](int t, int vs, bool first) {
+            // O_t (+)= P_t V for one half (64 keys) of the V tile in ring stage vs: A = 16-bit P in TMEM (8 columns per 16 keys)
+            auto issue_pv = [&](int t, int vs, bool first, int half) {
                 const uint64_t vd = vs ? v_desc1 : v_desc0;
                 const uint32_t d_tmem = tmem_base + 256 + t * 128, a_tmem = tmem_base + t * 128;
                 if (leader) {
 #pragma unroll
-                    for (int kk = 0; kk < BKV / 16; ++kk)
+                    for (int k4 = 0; k4 < BKV / 32; ++k4) {
+                        const int kk = half * (BKV / 32) + k4;
                         umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o,
                                 (first && kk == 0) ? 0u : 1u);
+                    }
                 }
                 __syncwarp();
             };
@@ -251,9 +280,12 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                             // the first PV of an item overwrites O_t: the previous item's O_t must have been read out
                             if (j == 0 && n_o[t] > 0) mbar_wait(&ctrl->o_free[t], (n_o[t] - 1) & 1, ctx, BAR_O_FREE);
                             mbar_wait(&ctrl->p_full[t], n_s[t] & 1, ctx, BAR_P_FULL);
+                            tc_fence_after();
+                            issue_pv(t, sv, j == 0, 0);
+                            mbar_wait(&ctrl->p_half2[t], n_s[t] & 1, ctx, BAR_P_HALF2);
                             ++n_s[t];
                             tc_fence_after();
-                            issue_pv(t, sv, j == 0);
+                            issue_pv(t, sv, j == 0, 1);
                             if (j == J[t] - 1) commit(&ctrl->o_final[t]);
                         }
                         if (t == 1) commit(&ctrl->v_empty[sv]);
@@ -345,24 +377,30 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     }
                 }
 
-                const float neg_m = -m_used;
-                float ls[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(-m_used, -m_used);
+                uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};      // (0.0f, 0.0f) pairs
 #pragma unroll
                 for (int cc = 0; cc < 2; ++cc) {
                     uint32_t pk[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const float e0 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i]), c, neg_m));
-                        const float e1 = ex2(fmaf(__uint_as_float(s[cc * 64 + 2 * i + 1]), c, neg_m));
-                        ls[i & 3] += e0 + e1;
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 64 + 2 * i]),
+                                                          __uint_as_float(s[cc * 64 + 2 * i + 1])), c2, neg_m2), x0, x1);
+                        const float e0 = ex2(x0), e1 = ex2(x1);
+                        ls2[i & 3] = add_f32x2(ls2[i & 3], pack_f32x2(e0, e1));
                         pk[i] = pack_h16x2(e0, e1, F16);
                     }
                     tmem_st32(s_addr + cc * 32, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    mbar_arrive(cc == 0 ? &ctrl->p_full[t] : &ctrl->p_half2[t]);
                 }
-                l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&ctrl->p_full[t]);
+                {
+                    float a0, a1;
+                    unpack_f32x2(add_f32x2(add_f32x2(ls2[0], ls2[1]), add_f32x2(ls2[2], ls2[3])), a0, a1);
+                    l_run += a0 + a1;
+                }
             }
 
             // this tile's last PV is done: normalise and store, then hand O_t back to the MMA warp
