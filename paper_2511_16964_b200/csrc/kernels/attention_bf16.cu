@@ -339,14 +339,35 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 float pm[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pm[i] = -INFINITY;
+                // chunks of 32 keys that hold a valid key for at least one row of this warp (the same in every lane)
+                uint32_t live = 0xFu;
                 if (edge) {
+                    // A row's valid keys of this tile are its first n_valid: the tile ends at Sk and, under the
+                    // causal mask, at the row's own index.  Masking is decided per 32-key chunk with bounds that
+                    // hold for the whole warp (its rows are consecutive): chunks valid for every row take the plain
+                    // path, chunks valid for none are skipped altogether (their probabilities are zero), and only
+                    // the chunk the diagonal crosses pays for per-element compares.
+                    const int kv_left = p.Sk - k0;
+                    const int warp_row0 = (2 * pair + t) * BQ + q * 32;
+                    const int n_valid = min(kv_left, p.causal ? qidx - k0 + 1 : BKV);
+                    const int nv_min = min(kv_left, p.causal ? warp_row0 - k0 + 1 : BKV);
+                    const int nv_max = min(kv_left, p.causal ? warp_row0 - k0 + 32 : BKV);
 #pragma unroll
-                    for (int i = 0; i < BKV; ++i) {
-                        const int kidx = k0 + i;
-                        const bool ok = kidx < p.Sk && (!p.causal || kidx <= qidx);
-                        const float v = ok ? __uint_as_float(s[i]) : -INFINITY;
-                        s[i] = __float_as_uint(v);
-                        pm[i & 7] = fmaxf(pm[i & 7], v);
+                    for (int cc = 0; cc < BKV / 32; ++cc) {
+                        if ((cc + 1) * 32 <= nv_min) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                pm[i & 7] = fmaxf(pm[i & 7], __uint_as_float(s[cc * 32 + i]));
+                        } else if (cc * 32 >= nv_max) {
+                            live &= ~(1u << cc);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const float v = (cc * 32 + i < n_valid) ? __uint_as_float(s[cc * 32 + i]) : -INFINITY;
+                                s[cc * 32 + i] = __float_as_uint(v);
+                                pm[i & 7] = fmaxf(pm[i & 7], v);
+                            }
+                        }
                     }
                 } else {
 #pragma unroll
@@ -383,13 +404,23 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 for (int cc = 0; cc < 2; ++cc) {
                     uint32_t pk[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        float x0, x1;
-                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[cc * 64 + 2 * i]),
-                                                          __uint_as_float(s[cc * 64 + 2 * i + 1])), c2, neg_m2), x0, x1);
-                        const float e0 = ex2(x0), e1 = ex2(x1);
-                        ls2[i & 3] = add_f32x2(ls2[i & 3], pack_f32x2(e0, e1));
-                        pk[i] = pack_h16x2(e0, e1, F16);
+                    for (int c4 = 0; c4 < 2; ++c4) {
+                        const int ch = 2 * cc + c4;          // 32-key chunk
+                        if (live & (1u << ch)) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                float x0, x1;
+                                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[ch * 32 + 2 * i]),
+                                                                  __uint_as_float(s[ch * 32 + 2 * i + 1])), c2, neg_m2),
+                                             x0, x1);
+                                const float e0 = ex2(x0), e1 = ex2(x1);
+                                ls2[i & 3] = add_f32x2(ls2[i & 3], pack_f32x2(e0, e1));
+                                pk[c4 * 16 + i] = pack_h16x2(e0, e1, F16);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) pk[c4 * 16 + i] = 0u;
+                        }
                     }
                     tmem_st32(s_addr + cc * 32, pk);
                     tmem_st_wait();
