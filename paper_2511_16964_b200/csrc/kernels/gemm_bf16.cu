@@ -67,6 +67,28 @@ __device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int gro
     n_blk = r / gsz;
 }
 
+// Work items.  The tiles are dealt round-robin to the persistent clusters, so the last, partial round leaves
+// most clusters idle when only a few tiles remain.  If that remainder is at most half the cluster count, each
+// of its tiles is split into two 256 x 128 halves (an MMA with N = 128 into the first half of the accumulator
+// columns), which halves the length of the last round: 4096^2 outputs on 74 clusters are 256 tiles = 3 rounds
+// + 34 tiles -> 3 rounds + 68 half tiles (3.5 instead of 4 rounds).  Not used when the epilogue emits one
+// row-reduction pair per 256-column tile.
+struct Work { int tile, col_off, ncols; };
+struct WorkPlan { int full, items; };     // tiles in whole rounds; total work items
+__device__ __forceinline__ WorkPlan work_plan(int num_tiles, int num_clusters, bool may_split)
+{
+    const int full = (num_tiles / num_clusters) * num_clusters;
+    const int tail = num_tiles - full;
+    const bool split = may_split && tail > 0 && 2 * tail <= num_clusters;
+    return WorkPlan{split ? full : num_tiles, split ? full + 2 * tail : num_tiles};
+}
+__device__ __forceinline__ Work work_item(const WorkPlan &wp, int w)
+{
+    if (w < wp.full) return Work{w, 0, BN};
+    const int sub = w - wp.full;
+    return Work{wp.full + (sub >> 1), (sub & 1) * (BN / 2), BN / 2};
+}
+
 // Rows covered by the pair-row-tile with linear index m_lin.  Plain mode: 256 consecutive rows of A.
 // Grouped mode: row tiles are counted group by group (a group's last tile may be partly empty), the
 // tile's rows stop at the end of its group, and `group` selects the weight matrix and bias row.
@@ -106,6 +128,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int num_m = count_row_tiles(p), num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
+    const WorkPlan plan = work_plan(num_tiles, num_clusters, p.row_partials == 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], 1); }
@@ -132,12 +155,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool leader = elect_one();
             int s = 0;
             uint32_t ph = 0;
-            for (int t = cluster_id; t < num_tiles && !p.test_withhold_loads; t += num_clusters) {
+            for (int w = cluster_id; w < plan.items && !p.test_withhold_loads; w += num_clusters) {
+                const Work wk = work_item(plan, w);
                 int m_blk, n_blk;
-                tile_coords(t, num_m, num_n, p.group_m, m_blk, n_blk);
+                tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
                 const RowTile rt = row_tile(p, m_blk);
                 const int row0 = rt.row0 + (int)rank * BM;
-                const int col0 = n_blk * BN + (int)rank * BN_HALF;
+                // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
+                // (the bytes a stage waits for stay the same) and only their first 64 columns are used
+                const int col0 = n_blk * BN + wk.col_off + (int)rank * (wk.ncols / 2);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     mbar_wait(&ctrl->empty[s], ph ^ 1, ctx, BAR_EMPTY);
                     uint8_t *a_s = tiles + (size_t)s * STAGE_BYTES;
@@ -163,7 +189,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // ---------- MMA issuer (leader CTA only; warp-uniform loop, one elected lane issues)
         if (rank == 0) {
             const bool leader = elect_one();
-            const uint32_t idesc = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk, p.f16 != 0);
+            const uint32_t idesc_full = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk, p.f16 != 0);
+            const uint32_t idesc_half = make_idesc_bf16(2 * BM, BN / 2, false, !p.w_is_nk, p.f16 != 0);
             const uint32_t a_addr0 = smem_u32(tiles), b_addr0 = a_addr0 + A_BYTES;
             const uint64_t adesc0 = make_smem_desc_sw128(a_addr0, 0, 1024);
             const uint64_t bdesc0 = p.w_is_nk ? make_smem_desc_sw128(b_addr0, 0, 1024)
@@ -172,7 +199,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             int it = 0;
-            for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
+            for (int w = cluster_id; w < plan.items; w += num_clusters, ++it) {
+                const uint32_t idesc = work_item(plan, w).ncols == BN ? idesc_full : idesc_half;
                 const int acc = it & 1;
                 const uint32_t aph = (it >> 1) & 1;
                 mbar_wait_cluster(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
@@ -204,12 +232,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int et = threadIdx.x - 64;        // 0..127
         const bool f16 = p.f16 != 0;            // 16-bit tensors are IEEE half instead of bf16
         int it = 0;
-        for (int t = cluster_id; t < num_tiles; t += num_clusters, ++it) {
+        for (int w = cluster_id; w < plan.items; w += num_clusters, ++it) {
+            const Work wk = work_item(plan, w);
             int m_blk, n_blk;
-            tile_coords(t, num_m, num_n, p.group_m, m_blk, n_blk);
+            tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
-            const int n0 = n_blk * BN;
+            const int n0 = n_blk * BN + wk.col_off;      // first output column of this item
             const RowTile rt = row_tile(p, m_blk);
             const int row = rt.row0 + (int)rank * BM + q * 32 + lane;
             const bool row_ok = row < rt.row_end;
@@ -232,7 +261,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // softmax: running (max, sum exp); LayerNorm: running (mean, sum of squared deviations)
             float run_m = p.row_partials == 2 ? 0.0f : -INFINITY, run_l = 0.0f;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < wk.ncols / 32; ++c) {
                 const int nc = n0 + c * 32;
                 if (nc >= p.N) break;
                 uint32_t r[32];
@@ -400,7 +429,10 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
             }
             max_clusters = n < num_sms / 2 ? n : num_sms / 2;
         }
-        const int clusters = num_tiles < max_clusters ? num_tiles : max_clusters;
+        // up to two work items per tile (see work_plan): small problems get both halves of a tile onto
+        // different clusters
+        const int most = a.row_partials == 0 ? 2 * num_tiles : num_tiles;
+        const int clusters = most < max_clusters ? most : max_clusters;
         kern<<<dim3(2 * clusters), dim3(THREADS), SMEM_BYTES, stream>>>(tmA, tmB, args);
         return cudaGetLastError();
     };
