@@ -64,6 +64,12 @@ __device__ __forceinline__ float ex2(float x)
 
 // Two fp32 lanes per instruction (sm_100 packed arithmetic): halves the issue slots the scale-and-shift
 // and the row sums take in the softmax loop, which is bound by instruction issue, not by a pipe.
+// one 256-bit store (sm_100); dst must be 32-byte aligned
+__device__ __forceinline__ void st_global_32B(void *dst, const uint32_t *w)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
 {
     uint64_t r;
@@ -441,20 +447,28 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             const float inv_l = 1.0f / l_run;
             uint16_t *orow = static_cast<uint16_t *>(p.out) + (long long)(bh / p.H) * p.out_b +
                                   (long long)(bh % p.H) * p.out_h + (long long)qidx * p.out_s;
+            const bool wide_ok = (reinterpret_cast<uintptr_t>(orow) & 31) == 0;   // rows are only known to be 16-byte aligned
 #pragma unroll 1
             for (int cc = 0; cc < D / 32; ++cc) {
                 uint32_t r[32];
                 tmem_ld32(o_addr + cc * 32, r);
                 tmem_ld_wait();
                 if (qidx < p.S) {
+                    uint32_t w[16];
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        float f[8];
+                    for (int i = 0; i < 16; ++i)
+                        w[i] = pack_h16x2(__uint_as_float(r[2 * i]) * inv_l, __uint_as_float(r[2 * i + 1]) * inv_l, F16);
+                    if (wide_ok) {
+                        // thread = row, so a warp's store touches 32 different rows: 32-byte stores write whole
+                        // sectors and halve the number of store instructions
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[g * 8 + i]) * inv_l;
-                        *reinterpret_cast<uint4 *>(orow + cc * 32 + g * 8) =
-                            make_uint4(pack_h16x2(f[0], f[1], F16), pack_h16x2(f[2], f[3], F16),
-                                       pack_h16x2(f[4], f[5], F16), pack_h16x2(f[6], f[7], F16));
+                        for (int g = 0; g < 2; ++g)
+                            st_global_32B(orow + cc * 32 + g * 16, &w[g * 8]);
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            *reinterpret_cast<uint4 *>(orow + cc * 32 + g * 8) =
+                                make_uint4(w[g * 4], w[g * 4 + 1], w[g * 4 + 2], w[g * 4 + 3]);
                     }
                 }
             }

@@ -87,6 +87,23 @@ def test_strided_views_of_a_packed_projection_buffer():
     check_bf16(host64(out_bshd.permute(0, 2, 1, 3)), want, what="strided attention")
 
 
+@pytest.mark.parametrize("D", [128, 64])
+def test_output_rows_that_are_only_16_byte_aligned(D):
+    """Output rows with a pitch of D + 8 elements: every other row starts 16 bytes off a 32-byte boundary, so the
+    kernel must fall back from its 32-byte stores; the padding columns stay untouched."""
+    import paper_2511_16964_b200 as P
+    B, H, S = 1, 2, 200
+    c = G.config5(B=B, H=H, S=S, D=D, seed=14)
+    padded = torch.full((B, H, S, D + 8), 7.0, dtype=BF16, device="cuda")
+    P.pike_attention_chain(dev(c["q"], BF16), dev(c["k"], BF16), dev(c["v"], BF16), scale=c["scale"], causal=True,
+                           out=padded[..., :D])
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    check_bf16(host64(padded[..., :D]), O.attention(c["q"], c["k"], c["v"], scale=c["scale"], causal=True),
+               what="padded output rows")
+    assert (padded[..., D:] == 7.0).all()
+
+
 @functools.lru_cache(maxsize=1)
 def _config5_full():
     return G.config5()
