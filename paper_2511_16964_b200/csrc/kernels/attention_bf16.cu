@@ -64,12 +64,6 @@ __device__ __forceinline__ float ex2(float x)
 
 // Two fp32 lanes per instruction (sm_100 packed arithmetic): halves the issue slots the scale-and-shift
 // and the row sums take in the softmax loop, which is bound by instruction issue, not by a pipe.
-// one 256-bit store (sm_100); dst must be 32-byte aligned
-__device__ __forceinline__ void st_global_32B(void *dst, const uint32_t *w)
-{
-    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
-                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-}
 __device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
 {
     uint64_t r;

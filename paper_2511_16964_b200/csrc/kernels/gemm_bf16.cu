@@ -343,24 +343,39 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     run_m = nm;
                 }
 
+                // Thread = row, so one store instruction of a warp touches 32 different rows: where the chunk
+                // lies fully inside N and starts on a 32-byte boundary it is written with 32-byte stores (whole
+                // sectors, half as many instructions), else with 16-byte ones.
                 if (row_ok) {
+                    const bool whole = nc + 32 <= p.N;
                     if (p.out_f32) {
                         float *op = static_cast<float *>(p.out) + (long long)row * p.ldo + nc;
+                        if (whole && (reinterpret_cast<uintptr_t>(op) & 31) == 0) {
 #pragma unroll
-                        for (int g = 0; g < 8; ++g)
-                            if (nc + g * 4 < p.N)
-                                *reinterpret_cast<float4 *>(op + g * 4) =
-                                    make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+                            for (int g = 0; g < 4; ++g)
+                                st_global_32B(op + g * 8, reinterpret_cast<const uint32_t *>(&v[g * 8]));
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < 8; ++g)
+                                if (nc + g * 4 < p.N)
+                                    *reinterpret_cast<float4 *>(op + g * 4) =
+                                        make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+                        }
                     } else {
                         uint16_t *op = static_cast<uint16_t *>(p.out) + (long long)row * p.ldo + nc;
+                        uint32_t w[16];
 #pragma unroll
-                        for (int g = 0; g < 4; ++g)
-                            if (nc + g * 8 < p.N)
-                                *reinterpret_cast<uint4 *>(op + g * 8) =
-                                    make_uint4(pack_h16x2(v[g * 8 + 0], v[g * 8 + 1], f16),
-                                               pack_h16x2(v[g * 8 + 2], v[g * 8 + 3], f16),
-                                               pack_h16x2(v[g * 8 + 4], v[g * 8 + 5], f16),
-                                               pack_h16x2(v[g * 8 + 6], v[g * 8 + 7], f16));
+                        for (int i = 0; i < 16; ++i) w[i] = pack_h16x2(v[2 * i], v[2 * i + 1], f16);
+                        if (whole && (reinterpret_cast<uintptr_t>(op) & 31) == 0) {
+                            st_global_32B(op, &w[0]);
+                            st_global_32B(op + 16, &w[8]);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g)
+                                if (nc + g * 8 < p.N)
+                                    *reinterpret_cast<uint4 *>(op + g * 8) =
+                                        make_uint4(w[g * 4], w[g * 4 + 1], w[g * 4 + 2], w[g * 4 + 3]);
+                        }
                     }
                 }
             }
