@@ -34,7 +34,7 @@ METRIC = "fused_chain_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the four gemm_bf16_kernel launches of one step
-GEMM_DRAM_BYTES_PER_STEP = 2.694e9
+GEMM_DRAM_BYTES_PER_STEP = 2.793e9
 # x, W, residual and output once each: C2 134.2 MB, C3 GEMM1 469.8 MB, C3 GEMM2 469.8 MB, C4 541.1 MB
 GEMM_ALGORITHMIC_BYTES_PER_STEP = 1.615e9
 
