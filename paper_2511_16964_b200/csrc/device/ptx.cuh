@@ -422,6 +422,41 @@ __device__ __forceinline__ uint32_t pack_h16x2(float lo, float hi, bool f16)
 {
     return f16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
 }
+// Two fp32 lanes per instruction (sm_100 packed arithmetic): half the issue slots of the scalar forms, which
+// is what row-wise code bound by instruction issue (softmax, LayerNorm) needs.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// the two 16-bit values of a word as an fp32 pair (low half first)
+__device__ __forceinline__ uint64_t h16x2_to_f32x2(uint32_t u, bool f16)
+{
+    return pack_f32x2(h16_lo(u, f16), h16_hi(u, f16));
+}
 // one 256-bit store (sm_100); dst must be 32-byte aligned
 __device__ __forceinline__ void st_global_32B(void *dst, const uint32_t *w)
 {

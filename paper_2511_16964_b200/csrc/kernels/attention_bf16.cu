@@ -62,31 +62,6 @@ __device__ __forceinline__ float ex2(float x)
     return y;
 }
 
-// Two fp32 lanes per instruction (sm_100 packed arithmetic): halves the issue slots the scale-and-shift
-// and the row sums take in the softmax loop, which is bound by instruction issue, not by a pipe.
-__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
-{
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-
 // F16 = the tensors are IEEE half instead of bf16 (operand format of both MMAs, P and the output).
 // D = head dimension (64 or 128): one or two 64-wide swizzled sub-tiles per operand tile
 template <int D, bool F16>

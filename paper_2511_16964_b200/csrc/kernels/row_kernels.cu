@@ -143,27 +143,34 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
         const int ci = lane + i * 32;
         c[i] = ci < nchunks ? __ldg(xr + ci) : make_uint4(0u, 0u, 0u, 0u);
     }
-    float sum = 0.0f;
+    // all arithmetic on fp32 pairs (one 16-bit word = two elements): the kernel moves 4 bytes per element and is
+    // otherwise bound by how many instructions per element the warp has to issue
+    uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
         const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
-        for (int h = 0; h < 4; ++h) sum += h16_lo(w[h], F16) + h16_hi(w[h], F16);   // padding chunks are zero
+        for (int h = 0; h < 4; ++h) sum2[h & 1] = add_f32x2(sum2[h & 1], h16x2_to_f32x2(w[h], F16));   // padding chunks are zero
     }
-    const float mean = warp_sum(sum) / (float)D;
-    float ss = 0.0f;
+    float s0, s1;
+    unpack_f32x2(add_f32x2(sum2[0], sum2[1]), s0, s1);
+    const float mean = warp_sum(s0 + s1) / (float)D;
+    const uint64_t neg_mean2 = pack_f32x2(-mean, -mean);
+    uint64_t ss2[2] = {0ull, 0ull};
 #pragma unroll
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
         if (lane + i * 32 < nchunks) {
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float a = h16_lo(w[h], F16) - mean, b = h16_hi(w[h], F16) - mean;
-                ss += a * a + b * b;
+                const uint64_t d2 = add_f32x2(h16x2_to_f32x2(w[h], F16), neg_mean2);
+                ss2[h & 1] = fma_f32x2(d2, d2, ss2[h & 1]);
             }
         }
     }
-    const float rstd = rsqrtf(warp_sum(ss) / (float)D + eps);
+    unpack_f32x2(add_f32x2(ss2[0], ss2[1]), s0, s1);
+    const float rstd = rsqrtf(warp_sum(s0 + s1) / (float)D + eps);
+    const uint64_t rstd2 = pack_f32x2(rstd, rstd), shift2 = pack_f32x2(-mean * rstd, -mean * rstd);
     uint4 *zr = reinterpret_cast<uint4 *>(z + row * ldz);
 #pragma unroll
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
@@ -176,9 +183,11 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
             uint32_t o[4];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const float a = (h16_lo(w[h], F16) - mean) * rstd * g[2 * h] + be[2 * h];
-                const float b = (h16_hi(w[h], F16) - mean) * rstd * g[2 * h + 1] + be[2 * h + 1];
-                o[h] = pack_h16x2(a, b, F16);
+                // ((v - mean) * rstd) * g + be as two fused multiply-adds: v * rstd + (-mean * rstd), then * g + be
+                const uint64_t n2 = fma_f32x2(h16x2_to_f32x2(w[h], F16), rstd2, shift2);
+                float y0, y1;
+                unpack_f32x2(fma_f32x2(n2, pack_f32x2(g[2 * h], g[2 * h + 1]), pack_f32x2(be[2 * h], be[2 * h + 1])), y0, y1);
+                o[h] = pack_h16x2(y0, y1, F16);
             }
             zr[ci] = make_uint4(o[0], o[1], o[2], o[3]);
         }
