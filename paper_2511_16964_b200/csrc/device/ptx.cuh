@@ -463,6 +463,13 @@ __device__ __forceinline__ void st_global_32B(void *dst, const uint32_t *w)
     asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                  "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
+// one 256-bit load (sm_100); src must be 32-byte aligned
+__device__ __forceinline__ void ld_global_32B(const void *src, uint32_t *w)
+{
+    asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                 : "l"(src));
+}
 // element i of a 16-bit vector as fp32
 __device__ __forceinline__ float h16_at(const void *p, long long i, bool f16)
 {

@@ -280,10 +280,16 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
                     } else {
                         const uint16_t *rp = static_cast<const uint16_t *>(p.residual) + (long long)row * p.ldr + nc;
+                        if (nc + 32 <= p.N && (reinterpret_cast<uintptr_t>(rp) & 31) == 0) {
+                            // whole, 32-byte aligned chunk: two 32-byte loads (thread = row: one sector per row each)
+                            ld_global_32B(rp, reinterpret_cast<uint32_t *>(&res16[0]));
+                            ld_global_32B(rp + 16, reinterpret_cast<uint32_t *>(&res16[2]));
+                        } else {
 #pragma unroll
-                        for (int g = 0; g < 4; ++g)
-                            res16[g] = (nc + g * 8 < p.N) ? *reinterpret_cast<const uint4 *>(rp + g * 8)
-                                                          : make_uint4(0u, 0u, 0u, 0u);
+                            for (int g = 0; g < 4; ++g)
+                                res16[g] = (nc + g * 8 < p.N) ? *reinterpret_cast<const uint4 *>(rp + g * 8)
+                                                              : make_uint4(0u, 0u, 0u, 0u);
+                        }
                     }
                 }
                 tmem_ld_wait();
