@@ -645,7 +645,7 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
         if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
                                         gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
                                         beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D,
-                                        x->dtype == PIKE_F16, stream) != cudaSuccess)
+                                        x->dtype == PIKE_F16, h->status, h->limit_ns, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // h = act(z @ w1 + b1), rounded to the chain's 16-bit type
@@ -825,7 +825,7 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
         TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
         if (pike::launch_layernorm_bf16(x->data, E, z, E, gamma ? gamma->data : nullptr, gamma && gamma->dtype == PIKE_F32,
                                         beta ? beta->data : nullptr, beta && beta->dtype == PIKE_F32, epi->eps, (int)M,
-                                        (int)E, x->dtype == PIKE_F16, stream) != cudaSuccess)
+                                        (int)E, x->dtype == PIKE_F16, h->status, h->limit_ns, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // qkv = z @ w_qkv + b_qkv, laid out [B, S, 3, H, 128]

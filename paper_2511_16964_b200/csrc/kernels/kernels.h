@@ -9,6 +9,7 @@ namespace pike {
 enum : uint32_t {
     KID_GEMM = 1,
     KID_ATTN = 2,
+    KID_LAYERNORM = 3,
 };
 
 // ---- fp32 CUDA-core chain: out = reduce(scale*act(x@w+b)+res) ------------------
@@ -55,9 +56,10 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
 // ---- row kernels -------------------------------------------------------------------
 // z = LayerNorm(x) rows, 16-bit in/out (f16 != 0: IEEE half, else bf16), fp32 statistics; gamma/beta of
 // the same 16-bit type or f32 or null.
+// (status / limit_ns: the device status word and the bound of the kernel's waits for its row copies)
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  cudaStream_t stream);
+                                  unsigned int *status, unsigned long long limit_ns, cudaStream_t stream);
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
 // Pair t of row m sits at partials[m*pair_row_stride + t*pair_tile_stride] (pair_row_stride 0 = num_n_tiles,
 // the layout the GEMM epilogue writes; {1, M} reads pairs stored [t][m], as an all-gather over GPUs lays them).

@@ -92,11 +92,19 @@ layernorm_bf16_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *_
     }
 }
 
-// One WARP per row for rows of at most 4096 elements: the row sits in 16 x 16-byte registers per
-// lane, both reductions are pure shuffles (no block barrier), and eight independent rows per CTA keep
-// many loads in flight.
-constexpr int LNW_WARPS = 8;
+// One WARP per row for rows of at most 4096 elements, in a persistent grid (one CTA per SM, ten warps).
+// Each warp streams its rows through a private two-stage ring in shared memory filled by bulk copies
+// (one elected lane issues them, an mbarrier per stage counts the bytes): while a row is being reduced and
+// normalised in registers, the next two are already in flight, so loads, arithmetic and stores of different
+// rows overlap inside every warp instead of all warps of an SM loading, computing and storing in phase.
+// The row sits in 16 x 16-byte registers per lane and both reductions are pure shuffles.  gamma and beta are
+// copied to shared memory once per CTA (every warp needs all of them for every row).
+constexpr int LNW_WARPS = 10;
+constexpr int LNW_STAGES = 2;
 constexpr int LNW_MAX_CHUNKS = 16;  // D <= 32 * 16 * 8 = 4096
+constexpr int LNW_STAGE_BYTES = LNW_MAX_CHUNKS * 32 * 16;   // 8 KiB: one row of 4096 16-bit elements
+constexpr int LNW_PARAM_BYTES = LNW_MAX_CHUNKS * 32 * 8 * 4;   // 16 KiB: 4096 fp32 values (or 16-bit ones in half of it)
+constexpr size_t LNW_SMEM_BYTES = 128 + (size_t)LNW_WARPS * LNW_STAGES * LNW_STAGE_BYTES + 2 * LNW_PARAM_BYTES;
 
 __device__ __forceinline__ float warp_sum(float x)
 {
@@ -105,21 +113,21 @@ __device__ __forceinline__ float warp_sum(float x)
     return x;
 }
 
-// eight consecutive parameters starting at element e (e % 8 == 0) as fp32; KIND 0 = absent, 1 = 16-bit
-// (the type of x), 2 = f32
+// eight consecutive parameters starting at element e (e % 8 == 0) as fp32, from the CTA's copy in shared memory;
+// KIND 0 = absent, 1 = 16-bit (the type of x), 2 = f32
 template <int KIND, bool F16>
-__device__ __forceinline__ void load_param8(const void *p, int e, float dflt, float (&out)[8])
+__device__ __forceinline__ void smem_param8(const uint8_t *p, int e, float dflt, float (&out)[8])
 {
     if constexpr (KIND == 0) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) out[i] = dflt;
     } else if constexpr (KIND == 2) {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(p) + e));
-        const float4 b = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(p) + e + 4));
+        const float4 a = *reinterpret_cast<const float4 *>(p + (size_t)e * 4);
+        const float4 b = *reinterpret_cast<const float4 *>(p + (size_t)e * 4 + 16);
         out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
         out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
     } else {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(p) + e));
+        const uint4 v = *reinterpret_cast<const uint4 *>(p + (size_t)e * 2);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int h = 0; h < 4; ++h) { out[2 * h] = h16_lo(w[h], F16); out[2 * h + 1] = h16_hi(w[h], F16); }
@@ -127,21 +135,66 @@ __device__ __forceinline__ void load_param8(const void *p, int e, float dflt, fl
 }
 
 template <int GK, int BK, bool F16>
-__global__ void __launch_bounds__(LNW_WARPS * 32, 2)
+__global__ void __launch_bounds__(LNW_WARPS * 32, 1)
 layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *__restrict__ z,
-                           long long ldz, const void *gamma, const void *beta, float eps, int M, int D)
+                           long long ldz, const void *gamma, const void *beta, float eps, int M, int D,
+                           unsigned int *status, unsigned long long limit_ns)
 {
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * LNW_WARPS + (threadIdx.x >> 5);
-    if (row >= M) return;
-    const uint4 *xr = reinterpret_cast<const uint4 *>(x + row * ldx);
+    extern __shared__ uint8_t lnw_smem[];
+    __shared__ uint64_t full[LNW_WARPS][LNW_STAGES];
+    __shared__ uint32_t abort_word;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(lnw_smem) + 127) & ~uintptr_t(127));
+    uint8_t *ring = base + (size_t)warp * LNW_STAGES * LNW_STAGE_BYTES;
+    uint8_t *gamma_s = base + (size_t)LNW_WARPS * LNW_STAGES * LNW_STAGE_BYTES, *beta_s = gamma_s + LNW_PARAM_BYTES;
     const int nchunks = D / 8;
+    const uint32_t row_bytes = (uint32_t)D * 2;
+    if (threadIdx.x == 0) abort_word = 0;
+    // gamma / beta -> shared memory, 16 bytes per thread and turn (D is a multiple of 8, so both sizes are of 16)
+    if constexpr (GK != 0)
+        for (int o = threadIdx.x * 16; o < D * (GK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
+            *reinterpret_cast<uint4 *>(gamma_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(gamma) + o));
+    if constexpr (BK != 0)
+        for (int o = threadIdx.x * 16; o < D * (BK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
+            *reinterpret_cast<uint4 *>(beta_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(beta) + o));
+    if (lane == 0) {
+        for (int k = 0; k < LNW_STAGES; ++k) mbar_init(&full[warp][k], 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    const WaitCtx ctx{status, &abort_word, limit_ns, KID_LAYERNORM};
+    const long long stride = (long long)gridDim.x * LNW_WARPS;
+    const long long first = (long long)blockIdx.x * LNW_WARPS + warp;
+    // the first rows of this warp go into flight at once
+    if (lane == 0) {
+        for (int k = 0; k < LNW_STAGES; ++k) {
+            const long long r = first + k * stride;
+            if (r < M) {
+                mbar_arrive_expect_tx(&full[warp][k], row_bytes);
+                bulk_load_1d(ring + k * LNW_STAGE_BYTES, x + r * ldx, row_bytes, &full[warp][k]);
+            }
+        }
+    }
+    int it = 0;
+    for (long long row = first; row < M; row += stride, ++it) {
+    const int stage = it % LNW_STAGES;
+    mbar_wait(&full[warp][stage], (uint32_t)(it / LNW_STAGES) & 1u, ctx, 1u);
+    const uint4 *xr = reinterpret_cast<const uint4 *>(ring + stage * LNW_STAGE_BYTES);
 
     uint4 c[LNW_MAX_CHUNKS];
 #pragma unroll
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
         const int ci = lane + i * 32;
-        c[i] = ci < nchunks ? __ldg(xr + ci) : make_uint4(0u, 0u, 0u, 0u);
+        c[i] = ci < nchunks ? xr[ci] : make_uint4(0u, 0u, 0u, 0u);
+    }
+    // every lane has taken its chunks out of the stage: refill it with the row two turns ahead
+    __syncwarp();
+    if (lane == 0) {
+        const long long rn = row + LNW_STAGES * stride;
+        if (rn < M) {
+            mbar_arrive_expect_tx(&full[warp][stage], row_bytes);
+            bulk_load_1d(ring + stage * LNW_STAGE_BYTES, x + rn * ldx, row_bytes, &full[warp][stage]);
+        }
     }
     // all arithmetic on fp32 pairs (one 16-bit word = two elements): the kernel moves 4 bytes per element and is
     // otherwise bound by how many instructions per element the warp has to issue
@@ -178,8 +231,8 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
         if (ci < nchunks) {
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
             float g[8], be[8];
-            load_param8<GK, F16>(gamma, ci * 8, 1.0f, g);
-            load_param8<BK, F16>(beta, ci * 8, 0.0f, be);
+            smem_param8<GK, F16>(gamma_s, ci * 8, 1.0f, g);
+            smem_param8<BK, F16>(beta_s, ci * 8, 0.0f, be);
             uint32_t o[4];
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
@@ -191,8 +244,8 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
             }
             zr[ci] = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        asm volatile("" ::: "memory");   // keep the parameter loads of later chunks from being hoisted (registers)
     }
+    }   // rows of this warp
 }
 
 constexpr int SM_THREADS = 256;
@@ -362,19 +415,30 @@ cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const f
 
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  cudaStream_t stream)
+                                  unsigned int *status, unsigned long long limit_ns, cudaStream_t stream)
 {
     if (M <= 0) return cudaSuccess;
     if (D % 8 != 0 || D > LN_THREADS * LN_MAX_CHUNKS * 8) return cudaErrorInvalidValue;
     if (D <= 32 * LNW_MAX_CHUNKS * 8) {
         const int gk = gamma == nullptr ? 0 : (gamma_f32 ? 2 : 1), bk = beta == nullptr ? 0 : (beta_f32 ? 2 : 1);
-        const dim3 grid((M + LNW_WARPS - 1) / LNW_WARPS), block(LNW_WARPS * 32);
+        // persistent: one CTA per SM (the ring takes most of its shared memory), fewer if there are few rows
+        static int num_sms = 0;
+        if (num_sms == 0) {
+            int dev = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess ||
+                cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
+                num_sms = 1;
+        }
+        const int want = (M + LNW_WARPS - 1) / LNW_WARPS;
+        const dim3 grid(want < num_sms ? want : num_sms), block(LNW_WARPS * 32);
         const uint16_t *xp = static_cast<const uint16_t *>(x);
         uint16_t *zp = static_cast<uint16_t *>(z);
 #define PIKE_LN_CASE(G, B)                                                                                          \
     if (gk == G && bk == B) {                                                                                       \
-        if (f16) layernorm_bf16_warp_kernel<G, B, true><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D); \
-        else layernorm_bf16_warp_kernel<G, B, false><<<grid, block, 0, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D);   \
+        auto kern = f16 ? layernorm_bf16_warp_kernel<G, B, true> : layernorm_bf16_warp_kernel<G, B, false>;        \
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LNW_SMEM_BYTES); \
+        if (e != cudaSuccess) return e;                                                                             \
+        kern<<<grid, block, LNW_SMEM_BYTES, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D, status, limit_ns);  \
     }
         PIKE_LN_CASE(0, 0) PIKE_LN_CASE(0, 1) PIKE_LN_CASE(0, 2) PIKE_LN_CASE(1, 0) PIKE_LN_CASE(1, 1)
         PIKE_LN_CASE(1, 2) PIKE_LN_CASE(2, 0) PIKE_LN_CASE(2, 1) PIKE_LN_CASE(2, 2)
