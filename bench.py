@@ -457,6 +457,19 @@ def run_ours(args):
             per_config[n]["eager_ms"] = eager_ms[n]
             per_config[n]["speedup_vs_eager"] = eager_ms[n] / per_cfg_ms[n]
     kernels = {k: {"launches": v[0], "ms_per_step": v[1] / args.steps} for k, v in prof.items()}
+    # the other kernels of the default step against their own bounds (algorithmic bytes / flops per launch)
+    if tuple(only) == ALL:
+        def _bw(name, nbytes):
+            ms = kernels[name]["ms_per_step"]
+            gbs = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else None
+            kernels[name].update(bound="hbm", achieved=gbs, unit="GB/s", peak=peaks["hbm_gbs"],
+                                 frac=(gbs / peaks["hbm_gbs"]) if gbs else None)
+        _bw("layernorm_bf16", 2.0 * 8192 * 4096 * 2)                      # C3 prologue: x in, z out
+        _bw("softmax_finish", 2.0 * 2048 * 32000 * 4 + 2048 * 125 * 8)    # C4: logits in, probabilities out, pairs
+        ms = kernels["attention_bf16"]["ms_per_step"]
+        tf = f["C5"] / (ms * 1e-3) / 1e12 if ms > 0 else None
+        kernels["attention_bf16"].update(bound="tensor + sfu", achieved=tf, unit="TFLOP/s", peak=peak,
+                                         frac=(tf / peak) if tf else None)
 
     parity = None if args.no_parity else parity_spot_check(inputs, out)
 
