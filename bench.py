@@ -434,9 +434,9 @@ def run_ours(args):
         "frac": (gemm_tflops / peak) if gemm_tflops else None, "peak_source": f"{peaks['source']} cuBLAS bf16, {'sustained' if sustained else 'burst'} figure",
         "frac_of_nominal_2250": (gemm_tflops / NOMINAL_BF16_TFLOPS) if gemm_tflops else None,
         "launches": gemm_launches,
-        # DRAM bytes of the kernel's four launches of one step, from the ncu capture summarised in
-        # profiles/gemm_bf16_kernel_dram_per_step.md (null for partial suites, and to be reset to null
-        # whenever the kernel changes after that capture)
+        # DRAM bytes of the kernel's four launches of one step, from the ncu capture summarised under profiles/
+        # (per-step DRAM bytes of this kernel); null for partial suites, and to be reset to null whenever the
+        # kernel changes after that capture
         "traffic": GEMM_DRAM_BYTES_PER_STEP if tuple(only) == ALL else None,
         "traffic_unit": "bytes per step (4 launches)", "algorithmic_bytes": GEMM_ALGORITHMIC_BYTES_PER_STEP,
     }
