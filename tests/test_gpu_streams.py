@@ -1,0 +1,78 @@
+"""Every chain enqueues on the caller's stream: inputs produced on a side stream (after a deliberately long
+kernel) are consumed correctly without any device-wide synchronisation in between, and two chains issued to two
+streams do not disturb each other."""
+import numpy as np
+import pytest
+import torch
+
+import pike_inputs as G
+from oracle import pike_oracle as O
+from util import check_bf16, check_f32, dev, host64
+
+pytestmark = pytest.mark.gpu
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def _busy(stream, n=1 << 26):
+    """Something long-running on `stream`, so that work queued after it really waits for stream order."""
+    with torch.cuda.stream(stream):
+        a = torch.ones(n, device="cuda")
+        for _ in range(8):
+            a = a * 1.0001
+    return a
+
+
+def test_chains_follow_the_order_of_a_side_stream():
+    import paper_2511_16964_b200 as P
+    side = torch.cuda.Stream()
+    c2 = G.config2(M=300, K=192, N=328, seed=31)
+    c5 = G.config5(B=1, H=2, S=300, seed=32)
+    c1 = G.config1(M=40, K=64, N=72, seed=33)
+    # host tensors first; the device copies are made ON the side stream, behind the busy kernel
+    hx, hw, hb, hr = (torch.from_numpy(np.ascontiguousarray(c2[k], np.float32)).to(BF16).pin_memory() for k in "xwbr")
+    hq, hk, hv = (torch.from_numpy(np.ascontiguousarray(c5[k], np.float32)).to(BF16).pin_memory() for k in "qkv")
+    h1 = {k: torch.from_numpy(np.ascontiguousarray(c1[k], np.float32)).pin_memory() for k in ("x", "w", "b", "gamma", "beta")}
+    keep = _busy(side)
+    with torch.cuda.stream(side):
+        x, w, b, r = (t.to("cuda", non_blocking=True) for t in (hx, hw, hb, hr))
+        q, k, v = (t.to("cuda", non_blocking=True) for t in (hq, hk, hv))
+        d1 = {n: t.to("cuda", non_blocking=True) for n, t in h1.items()}
+        got2 = P.pike_linear_epilogue(x, w, b, r, act="silu", scale=0.5, stream=side)
+        got4 = P.pike_linear_epilogue(x, w, reduce="softmax", out_dtype=F32, stream=side)
+        got5 = P.pike_attention_chain(q, k, v, scale=float(c5["scale"]), causal=True, stream=side)
+        got1 = P.pike_linear_epilogue(d1["x"], d1["w"], d1["b"], None, d1["gamma"], d1["beta"], act="gelu_erf",
+                                      reduce="layernorm", eps=c1["eps"], stream=side)
+    side.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    check_bf16(host64(got2), O.linear_epilogue(c2["x"], c2["w"], c2["b"], c2["r"], act="silu", scale=0.5), what="side stream GEMM")
+    want4 = O.linear_epilogue(c2["x"], c2["w"], reduce="softmax")
+    assert np.abs(host64(got4) - want4).max() <= 1e-3 * want4.max() and np.abs(host64(got4).sum(1) - 1).max() <= 1e-5
+    check_bf16(host64(got5), O.attention(c5["q"], c5["k"], c5["v"], scale=c5["scale"], causal=True), what="side stream attention")
+    check_f32(host64(got1), O.linear_epilogue(c1["x"], c1["w"], c1["b"], None, c1["gamma"], c1["beta"], act="gelu_erf",
+                                              reduce="layernorm", eps=c1["eps"]), what="side stream fp32 chain")
+    del keep
+
+
+def test_two_streams_at_once():
+    import paper_2511_16964_b200 as P
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    c3 = G.config3(M=333, D=136, F=1032, seed=34, affine=True)
+    c5 = G.config5(B=2, H=3, S=257, seed=35)
+    t3 = {k: dev(c3[k], BF16) for k in ("x", "gamma", "beta", "w1", "b1", "w2", "b2")}
+    q, k, v = (dev(c5[n], BF16) for n in "qkv")
+    torch.cuda.synchronize()
+    outs3, outs5 = [], []
+    for _ in range(3):      # interleaved submissions; each stream has its own workspace and outputs
+        with torch.cuda.stream(s1):
+            outs3.append(P.pike_mlp_block(t3["x"], t3["gamma"], t3["beta"], t3["w1"], t3["b1"], t3["w2"], t3["b2"],
+                                          act="gelu_tanh", eps=c3["eps"], stream=s1))
+        with torch.cuda.stream(s2):
+            outs5.append(P.pike_attention_chain(q, k, v, scale=float(c5["scale"]), causal=False, stream=s2))
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    want3 = O.mlp_block(c3["x"], c3["gamma"], c3["beta"], c3["w1"], c3["b1"], c3["w2"], c3["b2"], eps=c3["eps"])
+    want5 = O.attention(c5["q"], c5["k"], c5["v"], scale=c5["scale"], causal=False)
+    for o in outs3:
+        check_bf16(host64(o), want3, what="mlp block on stream 1")
+    for o in outs5:
+        check_bf16(host64(o), want5, what="attention on stream 2")
