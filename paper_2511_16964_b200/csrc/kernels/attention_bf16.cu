@@ -16,8 +16,10 @@
 //            A operand straight from tensor memory
 //   O_t   += P_t(j) V_j     V is the MN-major B operand; accumulates in tensor memory
 // The MMA warp interleaves the two tiles (PV0, S0', PV1, S1', ...) so one tile's softmax
-// runs under the other tile's MMAs.  P_t(j) is handed over in two halves of 64 keys (p_full, then
-// p_half2): the first four PV MMAs run while the second half's exponentials are still being computed.
+// runs under the other tile's MMAs.  P_t(j) is handed over in two parts, keys 0..95 (p_full) and keys
+// 96..127 (p_half2): six of the eight PV MMAs run while the last chunk's exponentials are still being
+// computed, and only two are left once it arrives.  (Three or four parts cost more in waits of the MMA
+// warp than they gain.)
 // The running maximum is only raised when it grows by more than 2^8 (probabilities stay bounded by
 // 256 in between), so rescaling O in tensor memory is rare; it is done by the softmax threads
 // themselves between two PV MMAs.
@@ -46,7 +48,7 @@ struct __align__(8) Ctrl {
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
     uint64_t q_empty;
-    uint64_t s_full[2], p_full[2], p_half2[2];   // p_full: keys 0..63 of P_t written, p_half2: keys 64..127
+    uint64_t s_full[2], p_full[2], p_half2[2];   // p_full: keys 0..95 of P_t written, p_half2: keys 96..127
     uint64_t o_final[2], o_free[2];
     uint32_t tmem_base;
     uint32_t abort;
@@ -209,16 +211,17 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                 }
                 __syncwarp();
             };
-            // O_t (+)= P_t V for one half (64 keys) of the V tile in ring stage vs: A = 16-bit P in TMEM (8 columns per 16 keys)
+            // O_t (+)= P_t V for one part of the keys of the V tile in ring stage vs: A = 16-bit P in TMEM (8 columns per 16 keys)
             auto issue_pv = [&](int t, int vs, bool first, int half) {
                 const uint64_t vd = vs ? v_desc1 : v_desc0;
                 const uint32_t d_tmem = tmem_base + 256 + t * 128, a_tmem = tmem_base + t * 128;
                 if (leader) {
 #pragma unroll
-                    for (int k4 = 0; k4 < BKV / 32; ++k4) {
-                        const int kk = half * (BKV / 32) + k4;
-                        umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o,
-                                (first && kk == 0) ? 0u : 1u);
+                    for (int kk = 0; kk < BKV / 16; ++kk) {
+                        // first part: keys 0..95 (six MMAs), second part: keys 96..127 (two)
+                        if ((kk < 6) == (half == 0))
+                            umma_ts(d_tmem, a_tmem + kk * 8, desc_advance(vd, kk * 2048), idesc_o,
+                                    (first && kk == 0) ? 0u : 1u);
                     }
                 }
                 __syncwarp();
@@ -375,32 +378,32 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 
                 const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(-m_used, -m_used);
                 uint64_t ls2[4] = {0ull, 0ull, 0ull, 0ull};      // (0.0f, 0.0f) pairs
+                // 32 keys at a time: their 16 packed probability columns overwrite score columns that are already
+                // in registers; the MMA warp is told after the third chunk (keys 0..95) and after the last
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
-                    uint32_t pk[32];
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t pk[16];
+                    if (live & (1u << ch)) {
 #pragma unroll
-                    for (int c4 = 0; c4 < 2; ++c4) {
-                        const int ch = 2 * cc + c4;          // 32-key chunk
-                        if (live & (1u << ch)) {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                float x0, x1;
-                                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[ch * 32 + 2 * i]),
-                                                                  __uint_as_float(s[ch * 32 + 2 * i + 1])), c2, neg_m2),
-                                             x0, x1);
-                                const float e0 = ex2(x0), e1 = ex2(x1);
-                                ls2[i & 3] = add_f32x2(ls2[i & 3], pack_f32x2(e0, e1));
-                                pk[c4 * 16 + i] = pack_h16x2(e0, e1, F16);
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) pk[c4 * 16 + i] = 0u;
+                        for (int i = 0; i < 16; ++i) {
+                            float x0, x1;
+                            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[ch * 32 + 2 * i]),
+                                                              __uint_as_float(s[ch * 32 + 2 * i + 1])), c2, neg_m2),
+                                         x0, x1);
+                            const float e0 = ex2(x0), e1 = ex2(x1);
+                            ls2[i & 3] = add_f32x2(ls2[i & 3], pack_f32x2(e0, e1));
+                            pk[i] = pack_h16x2(e0, e1, F16);
                         }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) pk[i] = 0u;
                     }
-                    tmem_st32(s_addr + cc * 32, pk);
-                    tmem_st_wait();
-                    tc_fence_before();
-                    mbar_arrive(cc == 0 ? &ctrl->p_full[t] : &ctrl->p_half2[t]);
+                    tmem_st16(s_addr + ch * 16, pk);
+                    if (ch >= 2) {
+                        tmem_st_wait();
+                        tc_fence_before();
+                        mbar_arrive(ch == 2 ? &ctrl->p_full[t] : &ctrl->p_half2[t]);
+                    }
                 }
                 {
                     float a0, a1;
