@@ -89,19 +89,27 @@ typedef struct {
 
 typedef struct pike_handle_s *pike_handle_t;
 
-/* Create / destroy a handle for CUDA device `device`.  The handle caches device
- * properties and owns a 16-byte device status word (its only allocation).  A
- * handle is not thread-safe; use one per host thread.  PIKE_ERR_ARCH if the
- * device is not compute capability 10.x. */
+/* Create / destroy a handle for CUDA device `device`.  pike_create makes that
+ * device current, prepares every kernel for it (shared-memory limits, how many
+ * CTA pairs fit) and stores what it learns in the handle: the library keeps no
+ * per-device state outside handles, so handles on different devices or host
+ * threads never interfere.  The handle owns a 16-byte device status word (its
+ * only device allocation), one non-blocking stream for reading it, and a small
+ * cache of encoded TMA tensor maps keyed by (pointer, extents, pitches, box), so
+ * repeated calls on the same buffers skip the encoding.  A handle is not
+ * thread-safe; use one per host thread.  PIKE_ERR_ARCH if the device is not
+ * compute capability 10.x. */
 pike_status_t pike_create(pike_handle_t *handle, int device);
 pike_status_t pike_destroy(pike_handle_t handle);
 
 /* Static, never-freed description of a status code. */
 const char *pike_status_string(pike_status_t status);
 
-/* Reads (and clears) the device status word.  Synchronises the device.
- * *status is PIKE_OK or PIKE_ERR_TIMEOUT; *where identifies the wait that gave
- * up (kernel id << 16 | barrier id). */
+/* Reads (and clears) the device status word.  It waits for no kernel: the
+ * caller synchronises the stream(s) whose status it wants first; the read
+ * itself travels on the handle's own stream.  *status is PIKE_OK or
+ * PIKE_ERR_TIMEOUT; *where identifies the wait that gave up
+ * (kernel id << 16 | barrier id). */
 pike_status_t pike_get_last_device_status(pike_handle_t handle, pike_status_t *status, uint32_t *where);
 
 /* Test hook: upper bound, in nanoseconds, for every in-kernel wait of kernels
@@ -160,6 +168,8 @@ pike_status_t pike_profile_end(pike_handle_t handle, pike_kernel_profile_t *out)
  *
  * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless a
  * row reduction is requested on the 16-bit path); it reads only shapes and dtypes.
+ * For every entry point that takes one, a workspace that is NULL, not 256-byte
+ * aligned, too small, or that overlaps any tensor of the call is PIKE_ERR_WORKSPACE.
  */
 pike_status_t pike_linear_epilogue_workspace(pike_handle_t handle, const pike_tensor_t *x,
                                              const pike_tensor_t *w, const pike_epilogue_t *epi,
@@ -253,7 +263,10 @@ pike_status_t pike_linear_softmax_noalloc(pike_handle_t handle, const pike_tenso
  * K and N multiples of 8; reduce must be NONE.  group_offsets points to G+1 int32 values in DEVICE
  * memory (non-decreasing, first 0, last T; empty groups are fine): the kernel reads them itself, so
  * the host never has to wait for a router's counts.  No workspace.  Rows outside
- * [0, group_offsets[G]) are not written.
+ * [0, group_offsets[G]) are not written.  The host cannot check the offsets, so the kernel clamps each
+ * one to [0, T] and each group's end to at least its start: offsets that break the contract give
+ * meaningless values in the rows concerned, never an access outside the tensors.  The group that owns
+ * a row tile is found by bisection (about log2 G loads per tile), so G up to 65536 costs nothing extra.
  */
 pike_status_t pike_grouped_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
                                            const pike_tensor_t *bias, const pike_tensor_t *residual,

@@ -15,175 +15,13 @@
 
 #include "handle.h"
 
+#include "validate.h"
+
+using namespace pike_api;
+
 namespace {
 
 constexpr unsigned long long DEFAULT_LIMIT_NS = 2000000000ull;
-
-// Brackets one kernel launch with CUDA events on the caller's stream while profiling is on.
-struct TimedLaunch {
-    pike_handle_t h;
-    pike_kernel_t kid;
-    cudaStream_t stream;
-    static cudaEvent_t get(pike_handle_t h)
-    {
-        cudaEvent_t e = nullptr;
-        if (!h->ev_pool.empty()) { e = h->ev_pool.back(); h->ev_pool.pop_back(); }
-        else if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); e = nullptr; }
-        return e;
-    }
-    TimedLaunch(pike_handle_t h_, pike_kernel_t kid_, cudaStream_t s) : h(h_), kid(kid_), stream(s)
-    {
-        if (!h->profiling) return;
-        cudaEvent_t e = get(h);
-        if (e != nullptr) { cudaEventRecord(e, stream); h->ev_start[kid].push_back(e); }
-    }
-    ~TimedLaunch()
-    {
-        if (!h->profiling || h->ev_start[kid].size() == h->ev_stop[kid].size()) return;
-        cudaEvent_t e = get(h);
-        if (e != nullptr) { cudaEventRecord(e, stream); h->ev_stop[kid].push_back(e); }
-        else { h->ev_pool.push_back(h->ev_start[kid].back()); h->ev_start[kid].pop_back(); }
-    }
-};
-
-size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
-size_t elem_size(pike_dtype_t t) { return t == PIKE_F32 ? 4 : 2; }
-
-bool valid_dtype(pike_dtype_t t) { return t == PIKE_F32 || t == PIKE_BF16 || t == PIKE_F16; }
-bool is_16bit(pike_dtype_t t) { return t == PIKE_BF16 || t == PIKE_F16; }
-// an optional side tensor of a 16-bit chain is fp32 or of the chain's own 16-bit type (bf16 and f16 never mix)
-bool side_ok(const pike_tensor_t *t, pike_dtype_t chain) { return t == nullptr || t->dtype == PIKE_F32 || t->dtype == chain; }
-CUtensorMapDataType map_dtype(pike_dtype_t t)
-{
-    return t == PIKE_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
-}
-
-// a dense-enough 2-D view: innermost stride 1, row pitch >= columns, 16-byte aligned base and pitch
-pike_status_t check_matrix(const pike_tensor_t *t, int64_t rows, int64_t cols, bool pitch16 = true)
-{
-    if (t == nullptr) return PIKE_ERR_NULL;
-    if (!valid_dtype(t->dtype)) return PIKE_ERR_DTYPE;
-    if (t->ndim != 2 || t->shape[0] != rows || t->shape[1] != cols) return PIKE_ERR_SHAPE;
-    if (rows == 0 || cols == 0) return PIKE_OK;  // an empty tensor may have no storage
-    if (t->data == nullptr) return PIKE_ERR_NULL;
-    if (t->stride[1] != 1 || t->stride[0] < cols) return PIKE_ERR_STRIDE;
-    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
-    if (pitch16 && (t->stride[0] * (int64_t)elem_size(t->dtype)) % 16 != 0) return PIKE_ERR_ALIGNMENT;
-    return PIKE_OK;
-}
-
-pike_status_t check_vector(const pike_tensor_t *t, int64_t n)
-{
-    if (t == nullptr) return PIKE_OK;  // optional
-    if (t->data == nullptr) return PIKE_ERR_NULL;
-    if (!valid_dtype(t->dtype)) return PIKE_ERR_DTYPE;
-    if (t->ndim != 1 || t->shape[0] != n) return PIKE_ERR_SHAPE;
-    if (t->stride[0] != 1) return PIKE_ERR_STRIDE;
-    if (reinterpret_cast<uintptr_t>(t->data) % 16 != 0) return PIKE_ERR_ALIGNMENT;
-    return PIKE_OK;
-}
-
-void byte_range(const pike_tensor_t *t, uintptr_t &lo, uintptr_t &hi)
-{
-    int64_t last = 0;
-    for (int i = 0; i < t->ndim; ++i) last += (t->shape[i] - 1) * t->stride[i];
-    lo = reinterpret_cast<uintptr_t>(t->data);
-    hi = lo + (uintptr_t)(last + 1) * elem_size(t->dtype);
-}
-
-bool overlaps(const pike_tensor_t *a, const pike_tensor_t *b)
-{
-    if (a == nullptr || b == nullptr || a->data == nullptr || b->data == nullptr) return false;
-    uintptr_t alo, ahi, blo, bhi;
-    byte_range(a, alo, ahi);
-    byte_range(b, blo, bhi);
-    return alo < bhi && blo < ahi;
-}
-
-pike_status_t check_epilogue(const pike_epilogue_t *e)
-{
-    if (e == nullptr) return PIKE_ERR_NULL;
-    if (e->struct_size != sizeof(pike_epilogue_t)) return PIKE_ERR_UNSUPPORTED;
-    if ((int)e->act < 0 || (int)e->act > 3 || (int)e->reduce < 0 || (int)e->reduce > 2) return PIKE_ERR_UNSUPPORTED;
-    if (!valid_dtype(e->out_dtype)) return PIKE_ERR_DTYPE;
-    if (!isfinite(e->scale)) return PIKE_ERR_UNSUPPORTED;
-    return PIKE_OK;
-}
-
-// 16-bit [rows, cols] row-major matrix -> tensor map with a (box_cols x box_rows) box, 128-byte swizzle
-pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t rows, uint64_t cols,
-                          uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
-{
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {pitch_elems * 2};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = h->encode(map, map_dtype(dt), 2, const_cast<void *>(ptr), dims, strides, box,
-                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
-}
-
-// 16-bit attention operand, element (b, h, s, d) at ptr + b*sb + h*sh + s*ss + d (strides in elements, multiples
-// of 8) -> 4-D map {D, S, H, B} with a (64 x 128 x 1 x 1) box
-pike_status_t make_map_bhsd(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t B, uint64_t H, uint64_t S,
-                            uint64_t D, uint64_t sb, uint64_t sh, uint64_t ss)
-{
-    const cuuint64_t dims[4] = {D, S, H, B};
-    const cuuint64_t strides[3] = {ss * 2, sh * 2, sb * 2};
-    const cuuint32_t box[4] = {64, 128, 1, 1};
-    const cuuint32_t estr[4] = {1, 1, 1, 1};
-    const CUresult r = h->encode(map, map_dtype(dt), 4, const_cast<void *>(ptr), dims, strides, box,
-                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
-}
-
-// 16-bit weights [groups, rows, cols] (dense matrices `group_pitch` elements apart; groups == 1 for a plain
-// GEMM) -> 3-D map with a (box_cols x box_rows x 1) box, 128-byte swizzle
-pike_status_t make_map_w(pike_handle_t h, CUtensorMap *map, pike_dtype_t dt, const void *ptr, uint64_t groups, uint64_t rows,
-                         uint64_t cols, uint64_t pitch_elems, uint64_t group_pitch, uint32_t box_cols, uint32_t box_rows)
-{
-    const cuuint64_t dims[3] = {cols, rows, groups};
-    const cuuint64_t strides[2] = {pitch_elems * 2, (groups > 1 ? group_pitch : rows * pitch_elems) * 2};
-    const cuuint32_t box[3] = {box_cols, box_rows, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    const CUresult r = h->encode(map, map_dtype(dt), 3, const_cast<void *>(ptr), dims, strides, box,
-                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? PIKE_OK : PIKE_ERR_CUDA;
-}
-
-struct LinearShape {
-    int64_t M, K, N;
-    bool w_is_nk;
-    bool fp32_path;
-};
-
-pike_status_t linear_shape(const pike_tensor_t *x, const pike_tensor_t *w, const pike_epilogue_t *epi, LinearShape &s)
-{
-    if (x == nullptr || w == nullptr) return PIKE_ERR_NULL;
-    if (pike_status_t st = check_epilogue(epi)) return st;
-    if (x->ndim != 2 || w->ndim != 2) return PIKE_ERR_SHAPE;
-    if (!valid_dtype(x->dtype) || x->dtype != w->dtype) return PIKE_ERR_DTYPE;
-    s.w_is_nk = (epi->flags & PIKE_FLAG_W_IS_NK) != 0;
-    s.M = x->shape[0];
-    s.K = x->shape[1];
-    s.N = s.w_is_nk ? w->shape[0] : w->shape[1];
-    if ((s.w_is_nk ? w->shape[1] : w->shape[0]) != s.K) return PIKE_ERR_SHAPE;
-    if (s.M < 0 || s.K < 1 || s.N < 1) return PIKE_ERR_SHAPE;
-    if (s.M > 0x7fffffff || s.K > 0x7fffffff || s.N > 0x7fffffff) return PIKE_ERR_UNSUPPORTED;
-    s.fp32_path = x->dtype == PIKE_F32;
-    if (s.fp32_path) {
-        if (s.N > 1024) return PIKE_ERR_UNSUPPORTED;
-        if (epi->out_dtype != PIKE_F32) return PIKE_ERR_DTYPE;
-    } else {
-        if (s.K % 8 != 0 || s.N % 8 != 0) return PIKE_ERR_UNSUPPORTED;
-        if (epi->out_dtype != PIKE_F32 && epi->out_dtype != x->dtype) return PIKE_ERR_DTYPE;
-        if (epi->reduce == PIKE_REDUCE_SOFTMAX && epi->out_dtype != PIKE_F32) return PIKE_ERR_UNSUPPORTED;
-    }
-    return PIKE_OK;
-}
 
 size_t softmax_partials_bytes(const LinearShape &s)
 {
@@ -191,11 +29,15 @@ size_t softmax_partials_bytes(const LinearShape &s)
     return align256((size_t)s.M * (size_t)num_n * sizeof(float2));
 }
 
+}  // namespace
+
+namespace pike_api {
+
 // Launch one 16-bit GEMM + epilogue; w's dtype (bf16 or f16) is the chain's.  All tensors validated by the caller.
 pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pike_tensor_t *w, bool w_is_nk, int64_t M,
                        int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
                        void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
-                       cudaStream_t stream, int partials_mode = 1, const int *group_offsets = nullptr, int num_groups = 0)
+                       cudaStream_t stream, int partials_mode, const int *group_offsets, int num_groups)
 {
     CUtensorMap tmA, tmB;
     if (pike_status_t st = make_map_2d(h, &tmA, w->dtype, a_ptr, (uint64_t)M, (uint64_t)K, (uint64_t)lda, pike::GEMM_BK, pike::GEMM_BM))
@@ -231,10 +73,20 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.test_withhold_loads = h->withhold_next ? 1 : 0;
     h->withhold_next = false;
     TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
-    return pike::launch_gemm_bf16(tmA, tmB, g, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+    return pike::launch_gemm_bf16(tmA, tmB, g, h->gemm_max_clusters, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
-}  // namespace
+// Second half of the split-row softmax: combine the per-tile pairs, normalise `out` in place.
+pike_status_t run_softmax_finish(pike_handle_t h, pike_tensor_t *out, const float2 *partials, int64_t M, int64_t N,
+                                 cudaStream_t stream)
+{
+    const int num_n = (int)((N + pike::GEMM_BN - 1) / pike::GEMM_BN);
+    TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
+    return pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)M, (int)N,
+                                       stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
+}  // namespace pike_api
 
 extern "C" {
 
@@ -279,8 +131,20 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
         return PIKE_ERR_CUDA;
     }
     h->encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
-    if (cudaMalloc(&h->status, 4 * sizeof(unsigned int)) != cudaSuccess ||
+    h->status = nullptr;
+    h->aux_stream = nullptr;
+    h->noalloc_partials = nullptr;
+    h->map_cache.reserve(pike_handle_s::MAP_CACHE_SIZE);
+    // per-device kernel set-up, once, here: shared-memory limits of every kernel on this device and the launch
+    // limits the launchers need, so that no launch pays for an attribute call or reads a process-wide variable
+    if (pike::setup_fp32_chain() != cudaSuccess || pike::setup_gemm_bf16(h->num_sms, &h->gemm_max_clusters) != cudaSuccess ||
+        pike::setup_row_kernels() != cudaSuccess || pike::setup_attention_bf16(&h->attention_regs_ok) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaMalloc(&h->status, 4 * sizeof(unsigned int)) != cudaSuccess ||
         cudaMemset(h->status, 0, 4 * sizeof(unsigned int)) != cudaSuccess) {
+        cudaGetLastError();
+        if (h->status != nullptr) cudaFree(h->status);
+        if (h->aux_stream != nullptr) cudaStreamDestroy(h->aux_stream);
         delete h;
         return PIKE_ERR_CUDA;
     }
@@ -292,6 +156,7 @@ pike_status_t pike_destroy(pike_handle_t h)
 {
     if (h == nullptr) return PIKE_ERR_NULL;
     cudaFree(h->status);
+    cudaStreamDestroy(h->aux_stream);
     for (int k = 0; k < PIKE_KERNEL_COUNT; ++k) {
         for (cudaEvent_t e : h->ev_start[k]) cudaEventDestroy(e);
         for (cudaEvent_t e : h->ev_stop[k]) cudaEventDestroy(e);
@@ -340,9 +205,14 @@ pike_status_t pike_get_last_device_status(pike_handle_t h, pike_status_t *status
 {
     if (h == nullptr || status == nullptr) return PIKE_ERR_NULL;
     unsigned int host[4] = {0, 0, 0, 0};
-    if (cudaDeviceSynchronize() != cudaSuccess) return PIKE_ERR_CUDA;
-    if (cudaMemcpy(host, h->status, sizeof(host), cudaMemcpyDeviceToHost) != cudaSuccess) return PIKE_ERR_CUDA;
-    if (host[0] != 0 && cudaMemset(h->status, 0, sizeof(host)) != cudaSuccess) return PIKE_ERR_CUDA;
+    // The read (and the clearing write) travel on the handle's own non-blocking stream: they wait for no
+    // kernel of the caller, who has synchronised the streams whose status is of interest beforehand.
+    if (cudaMemcpyAsync(host, h->status, sizeof(host), cudaMemcpyDeviceToHost, h->aux_stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->aux_stream) != cudaSuccess)
+        return PIKE_ERR_CUDA;
+    if (host[0] != 0 && (cudaMemsetAsync(h->status, 0, sizeof(host), h->aux_stream) != cudaSuccess ||
+                         cudaStreamSynchronize(h->aux_stream) != cudaSuccess))
+        return PIKE_ERR_CUDA;
     *status = host[0] != 0 ? PIKE_ERR_TIMEOUT : PIKE_OK;
     if (where != nullptr) *where = host[0];
     return PIKE_OK;
@@ -415,7 +285,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         a.act = (int)epi->act; a.reduce = (int)epi->reduce;
         a.scale = epi->scale; a.eps = epi->eps;
         TimedLaunch timed(h, PIKE_KERNEL_FP32_CHAIN, stream);
-        return pike::launch_fp32_chain(a, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+        return pike::launch_fp32_chain(a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
 
     for (const pike_tensor_t *t : {bias, residual, gamma, beta})
@@ -424,9 +294,8 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
     // workspace, a second kernel combines them and finishes the rows in place
     float2 *partials = nullptr;
     if (epi->reduce != PIKE_REDUCE_NONE) {
-        const size_t need = softmax_partials_bytes(s);
-        if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 || workspace_bytes < need)
-            return PIKE_ERR_WORKSPACE;
+        const pike_tensor_t *all[7] = {x, w, bias, residual, gamma, beta, out};
+        if (pike_status_t st = check_workspace(workspace, workspace_bytes, softmax_partials_bytes(s), all, 7)) return st;
         partials = static_cast<float2 *>(workspace);
     }
     const bool layernorm = epi->reduce == PIKE_REDUCE_LAYERNORM;
@@ -446,10 +315,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
                                               stream) != cudaSuccess)
                 return PIKE_ERR_CUDA;
         } else {
-            TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
-            if (pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)s.M,
-                                            (int)s.N, stream) != cudaSuccess)
-                return PIKE_ERR_CUDA;
+            return run_softmax_finish(h, out, partials, s.M, s.N, stream);
         }
     }
     return PIKE_OK;
@@ -492,9 +358,11 @@ pike_status_t pike_linear_softmax_shard_local(pike_handle_t h, const pike_tensor
     if (reinterpret_cast<uintptr_t>(row_stats) % 8 != 0) return PIKE_ERR_ALIGNMENT;
     for (const pike_tensor_t *t : {x, w, bias})
         if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
-    const size_t need = softmax_partials_bytes(s);
-    if (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 || workspace_bytes < need)
-        return PIKE_ERR_WORKSPACE;
+    {
+        const pike_tensor_t *all[4] = {x, w, bias, out};
+        if (pike_status_t st = check_workspace(workspace, workspace_bytes, softmax_partials_bytes(s), all, 4)) return st;
+        if (s.M > 0 && overlaps_bytes(out, row_stats, (size_t)s.M * 8)) return PIKE_ERR_UNSUPPORTED;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (s.M == 0) return PIKE_OK;
@@ -631,9 +499,10 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
     for (const pike_tensor_t *t : ins)
         if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
     const size_t z_bytes = align256((size_t)M * D * 2), h_bytes = align256((size_t)M * F * 2);
-    if (M > 0 && (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 ||
-                  workspace_bytes < z_bytes + h_bytes))
-        return PIKE_ERR_WORKSPACE;
+    if (M > 0) {
+        const pike_tensor_t *all[8] = {x, gamma, beta, w1, b1, w2, b2, out};
+        if (pike_status_t st = check_workspace(workspace, workspace_bytes, z_bytes + h_bytes, all, 8)) return st;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (M == 0) return PIKE_OK;
@@ -645,7 +514,7 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
         if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
                                         gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
                                         beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D,
-                                        x->dtype == PIKE_F16, h->status, h->limit_ns, stream) != cudaSuccess)
+                                        x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // h = act(z @ w1 + b1), rounded to the chain's 16-bit type
@@ -711,7 +580,8 @@ static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, cons
     a.status = h->status;
     a.limit_ns = h->limit_ns;
     TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
-    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+    return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, h->attention_regs_ok, stream) == cudaSuccess
+               ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 pike_status_t pike_attention_chain_workspace(pike_handle_t h, const pike_tensor_t *q, const pike_epilogue_t *epi,
@@ -812,9 +682,10 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
         if (overlaps(out, t)) return PIKE_ERR_UNSUPPORTED;
     const int64_t M = B * S, H = E / 128;
     const size_t z_bytes = align256((size_t)M * E * 2), qkv_bytes = align256((size_t)M * 3 * E * 2);
-    if (M > 0 && (workspace == nullptr || reinterpret_cast<uintptr_t>(workspace) % 256 != 0 ||
-                  workspace_bytes < 2 * z_bytes + qkv_bytes))
-        return PIKE_ERR_WORKSPACE;
+    if (M > 0) {
+        const pike_tensor_t *all[8] = {x, gamma, beta, w_qkv, b_qkv, w_o, b_o, out};
+        if (pike_status_t st = check_workspace(workspace, workspace_bytes, 2 * z_bytes + qkv_bytes, all, 8)) return st;
+    }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (cudaSetDevice(h->device) != cudaSuccess) return PIKE_ERR_CUDA;
     if (M == 0) return PIKE_OK;
@@ -825,7 +696,7 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
         TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
         if (pike::launch_layernorm_bf16(x->data, E, z, E, gamma ? gamma->data : nullptr, gamma && gamma->dtype == PIKE_F32,
                                         beta ? beta->data : nullptr, beta && beta->dtype == PIKE_F32, epi->eps, (int)M,
-                                        (int)E, x->dtype == PIKE_F16, h->status, h->limit_ns, stream) != cudaSuccess)
+                                        (int)E, x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // qkv = z @ w_qkv + b_qkv, laid out [B, S, 3, H, 128]

@@ -462,33 +462,45 @@ template <int D, bool F16>
 static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                                       const AttnArgs &a, int num_sms, cudaStream_t stream)
 {
-    // The in-kernel setmaxnreg split draws on threads x registers-at-launch; refuse to launch
-    // (rather than wait forever inside the kernel) if the compiled kernel was given fewer.
-    static int regs_ok = -1;
-    if (regs_ok < 0) {
-        cudaFuncAttributes attr;
-        cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel<D, F16>);
-        if (e != cudaSuccess) return e;
-        regs_ok = (attr.numRegs * THREADS >= 128 * REGS_WG0 + 256 * REGS_SOFTMAX) ? 1 : 0;
-    }
-    if (!regs_ok) return cudaErrorLaunchOutOfResources;
     const int num_q_tiles = (a.S + BQ - 1) / BQ;
     const int num_pairs = (num_q_tiles + 1) / 2;
     const long long num_items = (long long)((num_pairs + 1) / 2) * a.BH;   // slots: two items each
-    cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<D, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)SMEM_BYTES);
-    if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(num_items < num_sms ? num_items : num_sms);   // persistent: one CTA per SM
     attention_bf16_kernel<D, F16><<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError();
 }
 
+// shared-memory limit of one instantiation; regs_ok is cleared if it was compiled with fewer registers than
+// the in-kernel setmaxnreg split draws on (threads x registers-at-launch)
+template <int D, bool F16>
+static cudaError_t setup_attention_d(bool *regs_ok)
+{
+    cudaFuncAttributes attr;
+    cudaError_t e = cudaFuncGetAttributes(&attr, attention_bf16_kernel<D, F16>);
+    if (e != cudaSuccess) return e;
+    if (attr.numRegs * THREADS < 128 * REGS_WG0 + 256 * REGS_SOFTMAX) *regs_ok = false;
+    return cudaFuncSetAttribute(attention_bf16_kernel<D, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)SMEM_BYTES);
+}
+
 }  // namespace
 
+cudaError_t setup_attention_bf16(bool *regs_ok)
+{
+    *regs_ok = true;
+    cudaError_t e;
+    if ((e = setup_attention_d<64, false>(regs_ok)) != cudaSuccess) return e;
+    if ((e = setup_attention_d<64, true>(regs_ok)) != cudaSuccess) return e;
+    if ((e = setup_attention_d<128, false>(regs_ok)) != cudaSuccess) return e;
+    return setup_attention_d<128, true>(regs_ok);
+}
+
 cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
-                                  const AttnArgs &a, int num_sms, cudaStream_t stream)
+                                  const AttnArgs &a, int num_sms, bool regs_ok, cudaStream_t stream)
 {
     if (a.BH <= 0 || a.S <= 0 || a.Sk <= 0) return cudaSuccess;
+    // refuse to launch (rather than wait forever inside the kernel) if the register split cannot be satisfied
+    if (!regs_ok) return cudaErrorLaunchOutOfResources;
     if (a.D == 64)
         return a.f16 ? launch_attention_d<64, true>(tmQ, tmK, tmV, a, num_sms, stream)
                      : launch_attention_d<64, false>(tmQ, tmK, tmV, a, num_sms, stream);

@@ -90,28 +90,39 @@ __device__ __forceinline__ Work work_item(const WorkPlan &wp, int w)
 }
 
 // Rows covered by the pair-row-tile with linear index m_lin.  Plain mode: 256 consecutive rows of A.
-// Grouped mode: row tiles are counted group by group (a group's last tile may be partly empty), the
-// tile's rows stop at the end of its group, and `group` selects the weight matrix and bias row.
+// Grouped mode: group e (rows off[e] .. off[e+1]) owns the row-tile indices starting at
+//   T(e) = off[e] / 256 + e.
+// T grows by at least ceil(len_e / 256) from one group to the next, so the groups' index ranges never
+// overlap, the owner of an index is found by bisection over the offsets (O(log G) loads per tile, no
+// scratch memory, no pass over all groups) and off[G] / 256 + G indices cover everything.  An index whose
+// tile would start at or past its group's end is EMPTY: row0 == row_end, and every warp role skips the
+// item.  A tile's rows stop at the end of its group; `group` selects the weight matrix and bias row.
+// Offsets come from device memory the host cannot check, so each one is clamped to [0, M] (and an end
+// to at least its start): whatever a router wrote there, no row outside the tensors is touched.
 struct RowTile { int row0, row_end, group; };
+__device__ __forceinline__ int clamp_offset(const int *offsets, int i, int lo, int hi)
+{
+    return min(max(__ldg(offsets + i), lo), hi);
+}
 __device__ __forceinline__ RowTile row_tile(const GemmArgs &p, int m_lin)
 {
     if (p.group_offsets == nullptr) return RowTile{m_lin * 2 * BM, p.M, 0};
-    int first = 0;
-    for (int e = 0; e < p.num_groups; ++e) {
-        const int lo = __ldg(p.group_offsets + e), hi = __ldg(p.group_offsets + e + 1);
-        const int tiles = (hi - lo + 2 * BM - 1) / (2 * BM);
-        if (m_lin < first + tiles) return RowTile{lo + (m_lin - first) * 2 * BM, hi, e};
-        first += tiles;
+    int lo = 0, hi = p.num_groups - 1;      // the owner is the last group with T(e) <= m_lin
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (clamp_offset(p.group_offsets, mid, 0, p.M) / (2 * BM) + mid <= m_lin) lo = mid; else hi = mid - 1;
     }
-    return RowTile{p.M, p.M, 0};   // past the end: nothing to store
+    const int first = clamp_offset(p.group_offsets, lo, 0, p.M);
+    const int end = clamp_offset(p.group_offsets, lo + 1, first, p.M);
+    const long long local = (long long)m_lin - (first / (2 * BM) + lo);
+    const long long row0 = first + local * (2 * BM);
+    if (local < 0 || row0 >= end) return RowTile{p.M, p.M, 0};
+    return RowTile{(int)row0, end, lo};
 }
 __device__ __forceinline__ int count_row_tiles(const GemmArgs &p)
 {
     if (p.group_offsets == nullptr) return (p.M + 2 * BM - 1) / (2 * BM);
-    int n = 0;
-    for (int e = 0; e < p.num_groups; ++e)
-        n += (__ldg(p.group_offsets + e + 1) - __ldg(p.group_offsets + e) + 2 * BM - 1) / (2 * BM);
-    return n;
+    return clamp_offset(p.group_offsets, p.num_groups, 0, p.M) / (2 * BM) + p.num_groups;
 }
 
 template <int ACT>
@@ -160,6 +171,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 int m_blk, n_blk;
                 tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
                 const RowTile rt = row_tile(p, m_blk);
+                if (rt.row0 >= rt.row_end) continue;        // empty row tile (grouped mode): every role skips it
                 const int row0 = rt.row0 + (int)rank * BM;
                 // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
                 // (the bytes a stage waits for stay the same) and only their first 64 columns are used
@@ -199,8 +211,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             int it = 0;
-            for (int w = cluster_id; w < plan.items; w += num_clusters, ++it) {
-                const uint32_t idesc = work_item(plan, w).ncols == BN ? idesc_full : idesc_half;
+            for (int w = cluster_id; w < plan.items; w += num_clusters) {
+                const Work wk = work_item(plan, w);
+                if (p.group_offsets != nullptr) {
+                    int m_blk, n_blk;
+                    tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
+                    const RowTile rt = row_tile(p, m_blk);
+                    if (rt.row0 >= rt.row_end) continue;
+                }
+                const uint32_t idesc = wk.ncols == BN ? idesc_full : idesc_half;
                 const int acc = it & 1;
                 const uint32_t aph = (it >> 1) & 1;
                 mbar_wait_cluster(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
@@ -224,6 +243,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
                 if (leader) umma_commit_pair(&ctrl->tmem_full[acc], 0x3);
                 __syncwarp();
+                ++it;
             }
         }
     } else {
@@ -232,14 +252,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int et = threadIdx.x - 64;        // 0..127
         const bool f16 = p.f16 != 0;            // 16-bit tensors are IEEE half instead of bf16
         int it = 0;
-        for (int w = cluster_id; w < plan.items; w += num_clusters, ++it) {
+        for (int w = cluster_id; w < plan.items; w += num_clusters) {
             const Work wk = work_item(plan, w);
             int m_blk, n_blk;
             tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
+            const RowTile rt = row_tile(p, m_blk);
+            if (rt.row0 >= rt.row_end) continue;
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int n0 = n_blk * BN + wk.col_off;      // first output column of this item
-            const RowTile rt = row_tile(p, m_blk);
             const int row = rt.row0 + (int)rank * BM + q * 32 + lane;
             const bool row_ok = row < rt.row_end;
             const long long bias0 = (long long)rt.group * p.N + n0;    // bias is [num_groups, N] in grouped mode
@@ -391,6 +412,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctrl->tmem_empty[acc]), 0));
 
             if (p.row_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
+            ++it;
         }
     }
 
@@ -407,14 +429,48 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
 }  // namespace
 
-cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
+template <typename Kern>
+static cudaError_t setup_one(Kern kern, int num_sms, int *max_clusters)
+{
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    // how many CTA pairs the device can hold at once (one CTA per SM at this shared-memory size)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * (num_sms / 2));
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        n = num_sms / 2;
+    }
+    if (n < *max_clusters) *max_clusters = n;
+    return cudaSuccess;
+}
+
+cudaError_t setup_gemm_bf16(int num_sms, int *max_clusters)
+{
+    *max_clusters = num_sms / 2;
+    cudaError_t e;
+    if ((e = setup_one(gemm_bf16_kernel<ACT_NONE>, num_sms, max_clusters)) != cudaSuccess) return e;
+    if ((e = setup_one(gemm_bf16_kernel<ACT_GELU_ERF>, num_sms, max_clusters)) != cudaSuccess) return e;
+    if ((e = setup_one(gemm_bf16_kernel<ACT_GELU_TANH>, num_sms, max_clusters)) != cudaSuccess) return e;
+    return setup_one(gemm_bf16_kernel<ACT_SILU>, num_sms, max_clusters);
+}
+
+cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int max_clusters,
                              cudaStream_t stream)
 {
-    // grouped mode: the device counts the row tiles itself; this is the host's upper bound for sizing
-    const int num_m = (a.M + 2 * BM - 1) / (2 * BM) + (a.group_offsets != nullptr ? a.num_groups : 0);
+    // grouped mode: the device derives the row tiles from the offsets itself; this is the host's upper bound
+    const int num_m = a.group_offsets != nullptr ? a.M / (2 * BM) + a.num_groups : (a.M + 2 * BM - 1) / (2 * BM);
     const int num_n = (a.N + BN - 1) / BN;
-    const int num_tiles = num_m * num_n;
-    if (num_tiles <= 0 || a.M <= 0) return cudaSuccess;
+    const long long num_tiles = (long long)num_m * num_n;
+    if (num_tiles <= 0 || a.M <= 0 || max_clusters <= 0) return cudaSuccess;
     // Row blocks per rasterisation group.  Measured on B200 (DRAM bytes of the two MLP GEMMs): HBM reads
     // are lowest when the group's rows of A (group_m x 256 x K bf16) stay within about 32 MB - a quarter
     // of the 126 MB L2, which is split over two dies and shared with the streaming W and output traffic -
@@ -428,41 +484,18 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
         if (g > num_m) g = num_m;
         args.group_m = (int)g;
     }
-    auto go = [&](auto kern) -> cudaError_t {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        // how many CTA pairs the device can hold at once (one CTA per SM at this shared-memory size)
-        static int max_clusters = 0;
-        if (max_clusters == 0) {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(2 * (num_sms / 2));
-            cfg.blockDim = dim3(THREADS);
-            cfg.dynamicSmemBytes = SMEM_BYTES;
-            cudaLaunchAttribute attr;
-            attr.id = cudaLaunchAttributeClusterDimension;
-            attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-            cfg.attrs = &attr;
-            cfg.numAttrs = 1;
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
-                cudaGetLastError();
-                n = num_sms / 2;
-            }
-            max_clusters = n < num_sms / 2 ? n : num_sms / 2;
-        }
-        // up to two work items per tile (see work_plan): small problems get both halves of a tile onto
-        // different clusters
-        const int most = a.row_partials == 0 ? 2 * num_tiles : num_tiles;
-        const int clusters = most < max_clusters ? most : max_clusters;
-        kern<<<dim3(2 * clusters), dim3(THREADS), SMEM_BYTES, stream>>>(tmA, tmB, args);
-        return cudaGetLastError();
-    };
+    // up to two work items per tile (see work_plan): small problems get both halves of a tile onto
+    // different clusters
+    const long long most = a.row_partials == 0 ? 2 * num_tiles : num_tiles;
+    const int clusters = most < max_clusters ? (int)most : max_clusters;
+    const dim3 grid(2 * clusters), block(THREADS);
     switch (a.act) {
-    case ACT_GELU_ERF:  return go(gemm_bf16_kernel<ACT_GELU_ERF>);
-    case ACT_GELU_TANH: return go(gemm_bf16_kernel<ACT_GELU_TANH>);
-    case ACT_SILU:      return go(gemm_bf16_kernel<ACT_SILU>);
-    default:            return go(gemm_bf16_kernel<ACT_NONE>);
+    case ACT_GELU_ERF:  gemm_bf16_kernel<ACT_GELU_ERF><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
+    case ACT_GELU_TANH: gemm_bf16_kernel<ACT_GELU_TANH><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
+    case ACT_SILU:      gemm_bf16_kernel<ACT_SILU><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
+    default:            gemm_bf16_kernel<ACT_NONE><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
     }
+    return cudaGetLastError();
 }
 
 }  // namespace pike

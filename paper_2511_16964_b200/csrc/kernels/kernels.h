@@ -22,7 +22,15 @@ struct Fp32ChainArgs {
     int act, reduce;
     float scale, eps;
 };
-cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, cudaStream_t stream);
+cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, int num_sms, cudaStream_t stream);
+
+// ---- once per device (with that device current): function attributes and launch limits ------------
+// Each setup_* raises the dynamic shared-memory limit of its kernels on the current device, so that
+// the launchers make no attribute call per launch, and reports what the launchers need to know.
+cudaError_t setup_fp32_chain();
+cudaError_t setup_gemm_bf16(int num_sms, int *max_clusters);   // CTA pairs the device holds at once
+cudaError_t setup_row_kernels();
+cudaError_t setup_attention_bf16(bool *regs_ok);               // false: compiled with too few registers for the in-kernel split
 
 // ---- 16-bit (bf16 or f16) tcgen05 GEMM + epilogue --------------------------------
 struct GemmArgs {
@@ -50,7 +58,7 @@ struct GemmArgs {
 // the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
 // W as [K,N] {64, GEMM_BK}.
 constexpr int GEMM_BM = 128, GEMM_BN = 256, GEMM_BK = 64;
-cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int num_sms,
+cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int max_clusters,
                              cudaStream_t stream);
 
 // ---- row kernels -------------------------------------------------------------------
@@ -59,7 +67,7 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
 // (status / limit_ns: the device status word and the bound of the kernel's waits for its row copies)
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  unsigned int *status, unsigned long long limit_ns, cudaStream_t stream);
+                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream);
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
 // Pair t of row m sits at partials[m*pair_row_stride + t*pair_tile_stride] (pair_row_stride 0 = num_n_tiles,
 // the layout the GEMM epilogue writes; {1, M} reads pairs stored [t][m], as an all-gather over GPUs lays them).
@@ -87,6 +95,6 @@ struct AttnArgs {
     unsigned long long limit_ns;
 };
 cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
-                                  const AttnArgs &a, int num_sms, cudaStream_t stream);
+                                  const AttnArgs &a, int num_sms, bool regs_ok, cudaStream_t stream);
 
 }  // namespace pike

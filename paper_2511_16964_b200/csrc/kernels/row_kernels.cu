@@ -149,24 +149,14 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
     uint8_t *gamma_s = base + (size_t)LNW_WARPS * LNW_STAGES * LNW_STAGE_BYTES, *beta_s = gamma_s + LNW_PARAM_BYTES;
     const int nchunks = D / 8;
     const uint32_t row_bytes = (uint32_t)D * 2;
+    const long long stride = (long long)gridDim.x * LNW_WARPS;
+    const long long first = (long long)blockIdx.x * LNW_WARPS + warp;
     if (threadIdx.x == 0) abort_word = 0;
-    // gamma / beta -> shared memory, 16 bytes per thread and turn (D is a multiple of 8, so both sizes are of 16)
-    if constexpr (GK != 0)
-        for (int o = threadIdx.x * 16; o < D * (GK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
-            *reinterpret_cast<uint4 *>(gamma_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(gamma) + o));
-    if constexpr (BK != 0)
-        for (int o = threadIdx.x * 16; o < D * (BK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
-            *reinterpret_cast<uint4 *>(beta_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(beta) + o));
+    // each warp owns its barriers: it initialises them and puts its first rows in flight at once, before the
+    // CTA stages the parameters
     if (lane == 0) {
         for (int k = 0; k < LNW_STAGES; ++k) mbar_init(&full[warp][k], 1);
         fence_barrier_init();
-    }
-    __syncthreads();
-    const WaitCtx ctx{status, &abort_word, limit_ns, KID_LAYERNORM};
-    const long long stride = (long long)gridDim.x * LNW_WARPS;
-    const long long first = (long long)blockIdx.x * LNW_WARPS + warp;
-    // the first rows of this warp go into flight at once
-    if (lane == 0) {
         for (int k = 0; k < LNW_STAGES; ++k) {
             const long long r = first + k * stride;
             if (r < M) {
@@ -175,6 +165,15 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
             }
         }
     }
+    // gamma / beta -> shared memory, 16 bytes per thread and turn (D is a multiple of 8, so both sizes are of 16)
+    if constexpr (GK != 0)
+        for (int o = threadIdx.x * 16; o < D * (GK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
+            *reinterpret_cast<uint4 *>(gamma_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(gamma) + o));
+    if constexpr (BK != 0)
+        for (int o = threadIdx.x * 16; o < D * (BK == 2 ? 4 : 2); o += LNW_WARPS * 32 * 16)
+            *reinterpret_cast<uint4 *>(beta_s + o) = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint8_t *>(beta) + o));
+    __syncthreads();
+    const WaitCtx ctx{status, &abort_word, limit_ns, KID_LAYERNORM};
     int it = 0;
     for (long long row = first; row < M; row += stride, ++it) {
     const int stage = it % LNW_STAGES;
@@ -413,22 +412,33 @@ cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const f
     return cudaGetLastError();
 }
 
+cudaError_t setup_row_kernels()
+{
+#define PIKE_LN_SETUP(G, B)                                                                                         \
+    {                                                                                                               \
+        cudaError_t e = cudaFuncSetAttribute(layernorm_bf16_warp_kernel<G, B, true>,                                \
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LNW_SMEM_BYTES);     \
+        if (e != cudaSuccess) return e;                                                                             \
+        e = cudaFuncSetAttribute(layernorm_bf16_warp_kernel<G, B, false>,                                           \
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LNW_SMEM_BYTES);                 \
+        if (e != cudaSuccess) return e;                                                                             \
+    }
+    PIKE_LN_SETUP(0, 0) PIKE_LN_SETUP(0, 1) PIKE_LN_SETUP(0, 2) PIKE_LN_SETUP(1, 0) PIKE_LN_SETUP(1, 1)
+    PIKE_LN_SETUP(1, 2) PIKE_LN_SETUP(2, 0) PIKE_LN_SETUP(2, 1) PIKE_LN_SETUP(2, 2)
+#undef PIKE_LN_SETUP
+    return cudaSuccess;
+}
+
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  unsigned int *status, unsigned long long limit_ns, cudaStream_t stream)
+                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream)
 {
     if (M <= 0) return cudaSuccess;
     if (D % 8 != 0 || D > LN_THREADS * LN_MAX_CHUNKS * 8) return cudaErrorInvalidValue;
     if (D <= 32 * LNW_MAX_CHUNKS * 8) {
         const int gk = gamma == nullptr ? 0 : (gamma_f32 ? 2 : 1), bk = beta == nullptr ? 0 : (beta_f32 ? 2 : 1);
         // persistent: one CTA per SM (the ring takes most of its shared memory), fewer if there are few rows
-        static int num_sms = 0;
-        if (num_sms == 0) {
-            int dev = 0;
-            if (cudaGetDevice(&dev) != cudaSuccess ||
-                cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || num_sms <= 0)
-                num_sms = 1;
-        }
+        if (num_sms < 1) num_sms = 1;
         const int want = (M + LNW_WARPS - 1) / LNW_WARPS;
         const dim3 grid(want < num_sms ? want : num_sms), block(LNW_WARPS * 32);
         const uint16_t *xp = static_cast<const uint16_t *>(x);
@@ -436,8 +446,6 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
 #define PIKE_LN_CASE(G, B)                                                                                          \
     if (gk == G && bk == B) {                                                                                       \
         auto kern = f16 ? layernorm_bf16_warp_kernel<G, B, true> : layernorm_bf16_warp_kernel<G, B, false>;        \
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LNW_SMEM_BYTES); \
-        if (e != cudaSuccess) return e;                                                                             \
         kern<<<grid, block, LNW_SMEM_BYTES, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D, status, limit_ns);  \
     }
         PIKE_LN_CASE(0, 0) PIKE_LN_CASE(0, 1) PIKE_LN_CASE(0, 2) PIKE_LN_CASE(1, 0) PIKE_LN_CASE(1, 1)
