@@ -136,6 +136,20 @@ __device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, u
         ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w)
         : "memory");
 }
+// Asynchronous copies global -> shared issued by every thread (no tensor map, no barrier object): all of a
+// thread's copies are in flight at once and one wait covers them.  `valid` false writes zeros instead
+// (nothing is read, but src must still be an address inside the tensor).
+__device__ __forceinline__ void cp_async_16(void *dst, const void *src, bool valid)   // both 16-byte aligned
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(valid ? 16 : 0)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_4(void *dst, const void *src, bool valid)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(valid ? 4 : 0)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 // generic-proxy writes to shared memory -> visible to the async proxy (MMA/TMA)
 __device__ __forceinline__ void fence_proxy_async_smem()
 {
@@ -251,17 +265,34 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
-__device__ __forceinline__ void cluster_sync_all()  // every thread of both CTAs
+__device__ __forceinline__ uint32_t cluster_nctas()   // CTAs per cluster (x extent; clusters here are one-dimensional)
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctaid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()  // every thread of every CTA of the cluster
 {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of a cluster barrier on their own: a relaxed arrival orders no memory accesses (enough
+// when the barrier only has to say "I no longer read your shared memory") and lets work go on until the wait.
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.aligned;" ::: "memory"); }
 // shared::cta address of this CTA -> shared::cluster address of the same offset in CTA `rank`
 __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank)
 {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
+}
+// 8-byte load from any CTA's shared memory of the cluster (address from mapa_shared)
+__device__ __forceinline__ float2 ld_shared_cluster_f32x2(uint32_t cluster_addr)
+{
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(cluster_addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
