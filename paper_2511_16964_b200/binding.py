@@ -7,6 +7,7 @@ missing, loading raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes
 import os
 import threading
@@ -166,9 +167,19 @@ def _stream(stream) -> ctypes.c_void_p:
     return ctypes.c_void_p(s.cuda_stream)
 
 
-def _workspace(nbytes: int, device, workspace):
+def _on(stream):
+    """Allocations made for a call belong to the stream the kernels are enqueued on: torch's caching
+    allocator hands a freed block back to allocations of the SAME stream only, in stream order, so a
+    temporary dropped right after the call cannot be reused while the kernels still read or write it."""
+    return contextlib.nullcontext() if stream is None else torch.cuda.stream(stream)
+
+
+def _workspace(query, device, workspace, stream):
+    """(keep-alive, pointer, bytes) of the workspace: the caller's, or a temporary of the size `query()`
+    returns, allocated on `stream`.  A caller-supplied workspace is sized by the C side's own check."""
     if workspace is None:
-        workspace = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+        with _on(stream):
+            workspace = torch.empty(max(int(query()), 256), dtype=torch.uint8, device=device)
     return workspace, ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
 
 
@@ -189,7 +200,8 @@ def pike_test_withhold_loads(device=None) -> None:
 
 
 def pike_get_last_device_status(device=None) -> tuple[int, int]:
-    """(status, where) of the device status word; synchronises the device."""
+    """(status, where) of the device status word.  Does not wait for anybody's kernels: synchronise the
+    streams whose status is wanted first (torch.cuda.synchronize() or stream.synchronize())."""
     dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
     st, where = ctypes.c_int(0), ctypes.c_uint32(0)
     _check(load_library().pike_get_last_device_status(_handle(dev), ctypes.byref(st), ctypes.byref(where)),
@@ -228,11 +240,12 @@ def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, 
     out_dtype = (out.dtype if out is not None else x.dtype) if out_dtype is None else out_dtype
     N = w.shape[0] if w_is_nk else w.shape[1]
     if out is None:
-        out = torch.empty((x.shape[0], N), dtype=out_dtype, device=x.device)
+        with _on(stream):
+            out = torch.empty((x.shape[0], N), dtype=out_dtype, device=x.device)
     e = _epilogue(act, scale, reduce, eps, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
-    need = pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps,
-                                          out_dtype=out_dtype, w_is_nk=w_is_nk)
-    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    ws, ws_ptr, ws_bytes = _workspace(
+        lambda: pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps,
+                                               out_dtype=out_dtype, w_is_nk=w_is_nk), x.device, workspace, stream)
     _check(load_library().pike_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
                                                _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
                                                _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
@@ -254,16 +267,18 @@ def pike_linear_softmax_shard_local(x, w, bias=None, *, act="none", scale=1.0, w
     """First half of a softmax whose columns are split over GPUs: this GPU's un-normalised slice
     out [M,N_r] fp32 and row_stats [M,2] fp32 = (max, sum exp) of the slice; see include/pike.h."""
     N = w.shape[0] if w_is_nk else w.shape[1]
-    if out is None:
-        out = torch.empty((x.shape[0], N), dtype=torch.float32, device=x.device)
-    if row_stats is None:
-        row_stats = torch.empty((x.shape[0], 2), dtype=torch.float32, device=x.device)
+    with _on(stream):
+        if out is None:
+            out = torch.empty((x.shape[0], N), dtype=torch.float32, device=x.device)
+        if row_stats is None:
+            row_stats = torch.empty((x.shape[0], 2), dtype=torch.float32, device=x.device)
     if row_stats.dtype != torch.float32 or not row_stats.is_cuda or not row_stats.is_contiguous() \
             or row_stats.numel() != 2 * x.shape[0]:
         raise TypeError("row_stats must be a contiguous CUDA float32 tensor of M pairs")
     e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
-    need = pike_linear_softmax_shard_workspace(x, w, act=act, scale=scale, w_is_nk=w_is_nk)
-    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    ws, ws_ptr, ws_bytes = _workspace(
+        lambda: pike_linear_softmax_shard_workspace(x, w, act=act, scale=scale, w_is_nk=w_is_nk), x.device, workspace,
+        stream)
     _check(load_library().pike_linear_softmax_shard_local(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
                                                           ctypes.byref(e), _tensor(out),
                                                           ctypes.c_void_p(row_stats.data_ptr()), ws_ptr, ws_bytes,
@@ -314,10 +329,11 @@ def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5,
                    workspace=None, stream=None):
     """out = x + act(LayerNorm(x) @ w1 + b1) @ w2 + b2; see include/pike.h."""
     if out is None:
-        out = torch.empty_like(x)
+        with _on(stream):
+            out = torch.empty_like(x)
     e = _epilogue(act, 1.0, "none", eps, x.dtype, FLAG_W_IS_NK if w_is_nk else 0)
-    need = pike_mlp_block_workspace(x, w1, act=act, eps=eps, w_is_nk=w_is_nk)
-    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    ws, ws_ptr, ws_bytes = _workspace(lambda: pike_mlp_block_workspace(x, w1, act=act, eps=eps, w_is_nk=w_is_nk),
+                                      x.device, workspace, stream)
     _check(load_library().pike_mlp_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta), _tensor(w1),
                                          _tensor(b1), _tensor(w2), _tensor(b2), ctypes.byref(e), _tensor(out),
                                          ws_ptr, ws_bytes, _stream(stream)), "pike_mlp_block")
@@ -335,7 +351,8 @@ def pike_attention_chain_workspace(q, *, scale, causal=True) -> int:
 def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
     """out = softmax(scale * q k^T [+ causal mask]) v per (batch, head); see include/pike.h."""
     if out is None:
-        out = torch.empty_like(q)
+        with _on(stream):
+            out = torch.empty_like(q)
     e = _epilogue("none", scale, "none", 0.0, q.dtype, FLAG_CAUSAL if causal else 0)
     _check(load_library().pike_attention_chain(_handle(q.device), _tensor(q), _tensor(k), _tensor(v),
                                                ctypes.byref(e), _tensor(out), None, 0, _stream(stream)),
@@ -355,10 +372,12 @@ def pike_attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, scale, causa
                          out=None, workspace=None, stream=None):
     """out = x + attention(LayerNorm(x) @ w_qkv + b_qkv) @ w_o + b_o for x [B,S,E]; see include/pike.h."""
     if out is None:
-        out = torch.empty_like(x)
+        with _on(stream):
+            out = torch.empty_like(x)
     e = _epilogue("none", scale, "none", eps, x.dtype, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
-    need = pike_attention_block_workspace(x, scale=scale, causal=causal, eps=eps, w_is_nk=w_is_nk)
-    ws, ws_ptr, ws_bytes = _workspace(need, x.device, workspace)
+    ws, ws_ptr, ws_bytes = _workspace(
+        lambda: pike_attention_block_workspace(x, scale=scale, causal=causal, eps=eps, w_is_nk=w_is_nk), x.device,
+        workspace, stream)
     _check(load_library().pike_attention_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta),
                                                _tensor(w_qkv), _tensor(b_qkv), _tensor(w_o), _tensor(b_o),
                                                ctypes.byref(e), _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
@@ -375,7 +394,8 @@ def pike_grouped_linear_epilogue(x, w, bias, residual, group_offsets, *, act="no
     out_dtype = (out.dtype if out is not None else x.dtype) if out_dtype is None else out_dtype
     N = w.shape[1] if w_is_nk else w.shape[2]
     if out is None:
-        out = torch.zeros((x.shape[0], N), dtype=out_dtype, device=x.device)
+        with _on(stream):
+            out = torch.zeros((x.shape[0], N), dtype=out_dtype, device=x.device)
     e = _epilogue(act, scale, "none", 0.0, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
     _check(load_library().pike_grouped_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
                                                        _tensor(residual), ctypes.c_void_p(group_offsets.data_ptr()),

@@ -76,3 +76,37 @@ def test_two_streams_at_once():
         check_bf16(host64(o), want3, what="mlp block on stream 1")
     for o in outs5:
         check_bf16(host64(o), want5, what="attention on stream 2")
+
+
+def test_temporaries_belong_to_the_stream_the_kernels_run_on():
+    """The wrappers allocate missing outputs and workspaces for the stream given as `stream=`, even when another
+    stream is current: a block freed when the wrapper returns must not be handed to the current stream's next
+    allocation while the side stream's kernels still use it.  Here the default stream is current, the kernels are
+    queued on a busy side stream with workspace=None, and the default stream at once allocates and overwrites
+    tensors of the very sizes the temporaries had."""
+    import paper_2511_16964_b200 as P
+    side = torch.cuda.Stream()
+    c4 = G.config4(M=300, K=192, N=1000, seed=36)
+    c3 = G.config3(M=333, D=136, F=1032, seed=37, affine=True)
+    x4, w4 = dev(c4["x"], BF16), dev(c4["w"], BF16)
+    t3 = {k: dev(c3[k], BF16) for k in ("x", "gamma", "beta", "w1", "b1", "w2", "b2")}
+    need4 = P.pike_linear_epilogue_workspace(x4, w4, reduce="softmax", out_dtype=F32)
+    need3 = P.pike_mlp_block_workspace(t3["x"], t3["w1"])
+    torch.cuda.synchronize()
+    keep = _busy(side)                                       # the side stream's kernels will start late
+    got4 = P.pike_linear_epilogue(x4, w4, reduce="softmax", out_dtype=F32, stream=side)
+    got3 = P.pike_mlp_block(t3["x"], t3["gamma"], t3["beta"], t3["w1"], t3["b1"], t3["w2"], t3["b2"], eps=c3["eps"],
+                            stream=side)
+    junk = []
+    for _ in range(4):                                       # current (default) stream: same sizes, overwritten at once
+        junk.append(torch.full((max(need4, 256),), 0x7F, dtype=torch.uint8, device="cuda"))
+        junk.append(torch.full((max(need3, 256),), 0x7F, dtype=torch.uint8, device="cuda"))
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    want4 = O.linear_epilogue(c4["x"], c4["w"], reduce="softmax")
+    g4 = host64(got4)
+    assert (np.abs(g4 - want4) <= 1e-3 * want4 + 1e-9).all() and np.abs(g4.sum(1) - 1).max() <= 1e-5
+    check_bf16(host64(got3), O.mlp_block(c3["x"], c3["gamma"], c3["beta"], c3["w1"], c3["b1"], c3["w2"], c3["b2"],
+                                         eps=c3["eps"]), what="mlp block with a temporary workspace on a side stream")
+    del keep, junk
