@@ -114,8 +114,13 @@ def test_config5_full_size_sampled_rows():
     got = _run(c, True)
     rng = np.random.default_rng(11)
     worst = 0.0
-    for b, h in [(0, 0), (3, 17), (7, 31), (5, 8)]:
-        rows = np.unique(np.concatenate([[0, 127, 128, 2047], rng.integers(0, 2048, 12)]))
+    # every one of the 256 heads: two rows each, in query tiles that rotate with the head index, so every
+    # (head) and every one of the 16 query tiles (both tiles of every CTA's pair) is covered many times over
+    for i in range(256):
+        b, h = divmod(i, 32)
+        rows = np.array([(i % 16) * 128 + (29 * i) % 128, ((i + 7) % 16) * 128 + (53 * i + 11) % 128])
+        if i % 64 == 0:
+            rows = np.unique(np.concatenate([rows, [0, 127, 128, 2047], rng.integers(0, 2048, 12)]))
         want = O.attention_head(c["q"][b, h], c["k"][b, h], c["v"][b, h], scale=c["scale"], causal=True, rows=rows)
         worst = max(worst, check_bf16(got[b, h][rows], want, what=f"config 5 head ({b},{h})"))
     assert worst < 2e-2

@@ -5,6 +5,9 @@ import random
 import pytest
 import torch
 
+import pike_inputs as G
+from util import dev
+
 pytestmark = pytest.mark.gpu
 BF16 = torch.bfloat16
 
@@ -12,22 +15,20 @@ BF16 = torch.bfloat16
 def test_outputs_are_bitwise_reproducible():
     import paper_2511_16964_b200 as P
     rng = random.Random(0)
-    gen = torch.Generator(device="cuda").manual_seed(0)
-
-    def randn(*shape, scale=1.0):
-        return (torch.randn(*shape, device="cuda", generator=gen) * scale).to(BF16)
-
     cases = []
-    for M, K, N in [(1, 8, 8), (77, 64, 72), (300, 192, 328), (1000, 1024, 1000), (2560, 64, 2048)]:
-        x, w, b, r = randn(M, K), randn(K, N, scale=0.05), randn(N), randn(M, N)
+    for n, (M, K, N) in enumerate([(1, 8, 8), (77, 64, 72), (300, 192, 328), (1000, 1024, 1000), (2560, 64, 2048)]):
+        c = G.config2(M=M, K=K, N=N, seed=40 + n)
+        x, w, b, r = (dev(c[k], BF16) for k in "xwbr")
         cases.append(lambda x=x, w=w, b=b, r=r: P.pike_linear_epilogue(x, w, b, r, act="silu", scale=0.5))
         cases.append(lambda x=x, w=w: P.pike_linear_epilogue(x, w, reduce="softmax", out_dtype=torch.float32))
         cases.append(lambda x=x, w=w: P.pike_linear_epilogue(x, w, reduce="layernorm"))
-    for B, H, S, D in [(1, 1, 1, 128), (2, 3, 129, 64), (1, 3, 640, 128), (2, 1, 1500, 128)]:
-        q, k, v = randn(B, H, S, D), randn(B, H, S, D), randn(B, H, S, D)
+    for n, (B, H, S, D) in enumerate([(1, 1, 1, 128), (2, 3, 129, 64), (1, 3, 640, 128), (2, 1, 1500, 128)]):
+        c = G.config5(B=B, H=H, S=S, D=D, seed=50 + n)
+        q, k, v = (dev(c[name], BF16) for name in "qkv")
         cases.append(lambda q=q, k=k, v=v, D=D: P.pike_attention_chain(q, k, v, scale=D ** -0.5, causal=True))
-    x, w1, w2 = randn(333, 136), randn(136, 1032, scale=0.05), randn(1032, 136, scale=0.05)
-    cases.append(lambda: P.pike_mlp_block(x, None, None, w1, None, w2, None))
+    c3 = G.config3(M=333, D=136, F=1032, seed=60)
+    x3, w1, w2 = (dev(c3[name], BF16) for name in ("x", "w1", "w2"))
+    cases.append(lambda: P.pike_mlp_block(x3, None, None, w1, None, w2, None))
 
     ref = [c().clone() for c in cases]
     torch.cuda.synchronize()

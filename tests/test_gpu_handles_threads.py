@@ -1,0 +1,73 @@
+"""Two handles used from two host threads at once, through the raw C ABI (the header promises: one handle
+per host thread, no state shared between handles)."""
+import ctypes
+import threading
+
+import numpy as np
+import pytest
+import torch
+
+import pike_inputs as G
+from oracle import pike_oracle as O
+from util import check_bf16, check_f32, dev, host64
+
+pytestmark = pytest.mark.gpu
+BF16, F32 = torch.bfloat16, torch.float32
+
+
+def test_two_handles_on_two_threads():
+    from paper_2511_16964_b200 import binding as B
+    lib = B.load_library()
+    c2 = G.config2(M=600, K=256, N=520, seed=61)
+    c1 = G.config1(M=40, K=64, N=72, seed=62)
+    c5 = G.config5(B=1, H=2, S=300, seed=63)
+    x2, w2, b2, r2 = (dev(c2[k], BF16) for k in "xwbr")
+    x1, w1, b1 = (dev(c1[k], F32) for k in ("x", "w", "b"))
+    q, k, v = (dev(c5[n], BF16) for n in "qkv")
+    torch.cuda.synchronize()
+    results, errors = {}, []
+
+    def worker(tid):
+        try:
+            h = ctypes.c_void_p()
+            assert lib.pike_create(ctypes.byref(h), 0) == 0
+            stream = torch.cuda.Stream()
+            sp = ctypes.c_void_p(stream.cuda_stream)
+            outs = []
+            for rep in range(10):                      # both threads hammer the same kernels on their own handles
+                o2 = torch.empty((600, 520), dtype=BF16, device="cuda")
+                o1 = torch.empty((40, 72), dtype=F32, device="cuda")
+                o5 = torch.empty_like(q)
+                e2 = B._epilogue("silu", 0.5, "none", 0.0, BF16, 0)
+                e1 = B._epilogue("gelu_erf", 1.0, "layernorm", 1e-5, F32, 0)
+                e5 = B._epilogue("none", float(c5["scale"]), "none", 0.0, BF16, B.FLAG_CAUSAL)
+                rc = lib.pike_linear_epilogue(h, B._tensor(x2), B._tensor(w2), B._tensor(b2), B._tensor(r2), None, None,
+                                              ctypes.byref(e2), B._tensor(o2), None, 0, sp)
+                rc |= lib.pike_linear_epilogue(h, B._tensor(x1), B._tensor(w1), B._tensor(b1), None, None, None,
+                                               ctypes.byref(e1), B._tensor(o1), None, 0, sp)
+                rc |= lib.pike_attention_chain(h, B._tensor(q), B._tensor(k), B._tensor(v), ctypes.byref(e5),
+                                               B._tensor(o5), None, 0, sp)
+                assert rc == 0
+                outs.append((o2, o1, o5))
+            stream.synchronize()
+            st, where = ctypes.c_int(0), ctypes.c_uint32(0)
+            assert lib.pike_get_last_device_status(h, ctypes.byref(st), ctypes.byref(where)) == 0 and st.value == 0
+            assert lib.pike_destroy(h) == 0
+            results[tid] = outs
+        except BaseException as exc:                   # surfaced in the main thread
+            errors.append(exc)
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    want2 = O.linear_epilogue(c2["x"], c2["w"], c2["b"], c2["r"], act="silu", scale=0.5)
+    want1 = O.linear_epilogue(c1["x"], c1["w"], c1["b"], act="gelu_erf", reduce="layernorm")
+    want5 = O.attention(c5["q"], c5["k"], c5["v"], scale=c5["scale"], causal=True)
+    for tid in (0, 1):
+        for o2, o1, o5 in results[tid]:
+            check_bf16(host64(o2), want2, what=f"thread {tid} GEMM")
+            check_f32(host64(o1), want1, what=f"thread {tid} fp32 chain")
+            check_bf16(host64(o5), want5, what=f"thread {tid} attention")

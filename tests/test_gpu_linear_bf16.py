@@ -74,7 +74,8 @@ def _config2_full():
 
 def test_config2_full_size_sampled_rows():
     c = _config2_full()
-    rows = np.unique(np.concatenate([np.arange(0, 4096, 131), [127, 128, 4095]]))
+    # one row in every 128-row CTA block (32 blocks), at a different position in each, plus the corners
+    rows = np.unique(np.concatenate([[b * 128 + (37 * b + 5) % 128 for b in range(32)], [0, 127, 128, 4095]]))
     got, want = _gemm(c, act="silu", scale=0.5, rows=rows)
     check_bf16(got, want, what="config 2")
 
@@ -98,7 +99,8 @@ def test_split_row_softmax_small(M, K, N, w_is_nk):
 
 def test_config4_full_size_sampled_rows():
     c = G.config4()
-    rows = np.array([0, 1, 127, 128, 777, 1024, 2046, 2047])
+    # one row in every 128-row CTA block (16 blocks), at a different position in each, plus the corners
+    rows = np.unique(np.concatenate([[b * 128 + (37 * b + 5) % 128 for b in range(16)], [0, 127, 128, 2047]]))
     got, want = _gemm(c, bias=False, residual=False, out_dtype=F32, reduce="softmax", rows=rows)
     _softmax_gates(got, want, "config 4")
 
