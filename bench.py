@@ -13,10 +13,21 @@ With N > 1 launch under torchrun; every rank runs the same suite on its own GPU
 (rows / heads are independent, so the path shards without any collective: weak
 scaling) and rank 0 prints one JSON line.  `--impl reference` times the fp64 CPU
 oracle on a bounded row sample of the same workloads on the host cores.
+
+Beside the contract's keys the line carries:
+  sustained   the same step looped for at least two seconds with the clocks sampled: the
+              power-capped regime, with its own roofline against the sustained library figure
+  per_config  per chain: ms, TFLOP/s, fraction of the nominal 2250 TFLOP/s, eager time and
+              speed-up; X1..X3 (the further workloads, outside `value`) when N == 1
+  context     other ways to run the same chains on this GPU (fused library attention,
+              torch.compile): context rows, never a denominator
+  kernels     live device time per kernel of the library, with its own bound
+  host_call_us  what one call costs on the host (C ABI through prebuilt ctypes arguments)
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -33,10 +44,23 @@ if ROOT not in sys.path:
 METRIC = "fused_chain_tflops"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the four gemm_bf16_kernel launches of one step
-GEMM_DRAM_BYTES_PER_STEP = 2.793e9
 # x, W, residual and output once each: C2 134.2 MB, C3 GEMM1 469.8 MB, C3 GEMM2 469.8 MB, C4 541.1 MB
 GEMM_ALGORITHMIC_BYTES_PER_STEP = 1.615e9
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the four gemm_bf16_kernel launches of one step,
+# from the ncu captures summarised in profiles/gemm_bf16_kernel_dram_per_step.md: the value used, the spread
+# over repeated captures, and the SHA-256 (first 16 hex digits) of the kernel's sources at capture time.  The
+# line reports the traffic only while the sources still hash to that value.
+GEMM_DRAM_CAPTURE = {"bytes": None, "min": None, "max": None, "captures": 0, "sources_sha16": None}
+GEMM_SOURCES = ("paper_2511_16964_b200/csrc/kernels/gemm_bf16.cu", "paper_2511_16964_b200/csrc/device/ptx.cuh",
+                "paper_2511_16964_b200/csrc/device/act.cuh", "paper_2511_16964_b200/csrc/kernels/kernels.h")
+
+
+def sources_sha16(paths=GEMM_SOURCES) -> str:
+    h = hashlib.sha256()
+    for p in paths:
+        with open(os.path.join(ROOT, p), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
 
 
 # ----------------------------------------------------------------------------
@@ -59,6 +83,13 @@ def flops_per_config():
     }
 
 
+# flops of the launches of gemm_bf16_kernel inside each workload
+def gemm_kernel_flops():
+    f = flops_per_config()
+    return {"C2": f["C2"], "C3": f["C3"], "C4": f["C4"], "X1": 2.0 * 16384 * 4096 * (4 * 4096), "X2": f["X2"],
+            "X3": f["X3"]}
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -77,21 +108,31 @@ class ClockSampler:
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, period_ms: int = 20):
+        self.index, self.rows, self.proc, self.period_ms = index, [], None, period_ms
+        self.t_first = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms",
+                 str(self.period_ms), "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL,
+                text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
+            if self.t_first is None:
+                self.t_first = time.perf_counter()
             self.rows.append([c.strip() for c in line.split(",")])
+
+    def wait_first_sample(self, timeout=3.0):
+        """nvidia-smi needs a moment to start: a short region would otherwise end before the first sample."""
+        t0 = time.perf_counter()
+        while self.proc is not None and not self.rows and time.perf_counter() - t0 < timeout:
+            time.sleep(0.005)
 
     def stop(self):
         if self.proc is None:
@@ -113,8 +154,9 @@ class ClockSampler:
             for n, v in zip(names, r[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "power_w_max": max(power) if power else None,
+                "samples": len(sm), "period_ms": self.period_ms, "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------
@@ -124,28 +166,48 @@ ORACLE_SAMPLE = {"C1": 128, "C2": 4096, "C3": 288, "C4": 576, "C5_heads": 72}
 
 
 def oracle_sample_step(inputs):
-    """One pass of the oracle over the bounded sample; returns (flops, seconds)."""
+    """One pass of the oracle over the bounded sample; returns (flops, seconds, seconds per config)."""
     from oracle import pike_oracle as O
     f = flops_per_config()
     c1, c2, c3, c4, c5 = (inputs[k] for k in ("C1", "C2", "C3", "C4", "C5"))
     n = ORACLE_SAMPLE
-    flops = 0.0
-    t0 = time.perf_counter()
+    flops, per = 0.0, {}
+    t0 = t = time.perf_counter()
+
+    def lap(name):
+        nonlocal t
+        now = time.perf_counter()
+        per[name] = now - t
+        t = now
+
     O.linear_epilogue(c1["x"], c1["w"], c1["b"], None, c1["gamma"], c1["beta"], act="gelu_erf",
                       reduce="layernorm", eps=c1["eps"])
     flops += f["C1"]
+    lap("C1")
     O.linear_epilogue(c2["x"], c2["w"], c2["b"], c2["r"], act="silu", scale=0.5, rows=np.arange(n["C2"]))
     flops += f["C2"] * n["C2"] / 4096
+    lap("C2")
     O.mlp_block(c3["x"], c3["gamma"], c3["beta"], c3["w1"], c3["b1"], c3["w2"], c3["b2"], act="gelu_tanh",
                 eps=c3["eps"], rows=np.arange(n["C3"]))
     flops += f["C3"] * n["C3"] / 8192
+    lap("C3")
     O.linear_epilogue(c4["x"], c4["w"], reduce="softmax", rows=np.arange(n["C4"]))
     flops += f["C4"] * n["C4"] / 2048
+    lap("C4")
     for i in range(n["C5_heads"]):
         b, h = divmod(i, 32)
         O.attention_head(c5["q"][b, h], c5["k"][b, h], c5["v"][b, h], scale=c5["scale"], causal=True)
     flops += f["C5"] * n["C5_heads"] / 256
-    return flops, time.perf_counter() - t0
+    lap("C5")
+    return flops, time.perf_counter() - t0, per
+
+
+def oracle_full_size_seconds(per):
+    """Seconds the oracle would need for the whole step: every config's sample time scaled by rows (or heads)
+    total / sampled - rows and heads are independent, so the cost is linear in them."""
+    n = ORACLE_SAMPLE
+    scale = {"C1": 1.0, "C2": 4096 / n["C2"], "C3": 8192 / n["C3"], "C4": 2048 / n["C4"], "C5": 256 / n["C5_heads"]}
+    return {k: per[k] * scale[k] for k in per}
 
 
 def oracle_sample_text():
@@ -155,7 +217,7 @@ def oracle_sample_text():
 
 
 ALL = ("C1", "C2", "C3", "C4", "C5")          # the step
-EXTRA = ("X1", "X2", "X3")                   # further workloads, only with --only
+EXTRA = ("X1", "X2", "X3")                   # further workloads: with --only, or after the step when N == 1
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -174,6 +236,12 @@ def job_tflops(step_flops: float, world: int, ms_per_step: float) -> float:
     return world * step_flops / (ms_per_step * 1e-3) / 1e12
 
 
+def rank_env():
+    """(rank, world, local_rank) as torchrun exports them; a plain `python bench.py` is rank 0 of 1."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
 def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
@@ -184,7 +252,7 @@ def make_inputs(only=ALL):
 
 def run_reference(args):
     """--impl reference: the CPU oracle, as it stands, on the host cores."""
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = rank_env()
     if rank != 0:
         return 0
     from oracle import pike_oracle as O
@@ -192,12 +260,13 @@ def run_reference(args):
     inputs = make_inputs()
     for _ in range(max(0, args.ref_warmup)):
         oracle_sample_step(inputs)
-    total_f, total_t = 0.0, 0.0
+    total_f, total_t, per = 0.0, 0.0, {}
     for _ in range(args.ref_steps):
-        fl, dt = oracle_sample_step(inputs)
+        fl, dt, per = oracle_sample_step(inputs)
         total_f += fl
         total_t += dt
     value = total_f / total_t / 1e12
+    full = oracle_full_size_seconds(per)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.ref_steps, "warmup": args.ref_warmup, "ms_per_step": 1e3 * total_t / args.ref_steps,
@@ -205,7 +274,8 @@ def run_reference(args):
         "config": {"workload": "C1-C5 chain suite", "note": "fp64 CPU oracle on a bounded row sample per step; "
                    "the requested --steps/--warmup are mapped to %d/%d oracle passes" % (args.ref_steps, args.ref_warmup)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-                         "sample": oracle_sample_text()},
+                         "sample": oracle_sample_text(), "full_size_seconds_extrapolated": sum(full.values()),
+                         "full_size_seconds_per_config": full},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -215,15 +285,133 @@ def run_reference(args):
 # ----------------------------------------------------------------------------
 # the CUDA path
 # ----------------------------------------------------------------------------
+class Suite:
+    """Device tensors, outputs, workspaces and the chain calls of a set of workloads."""
+
+    def __init__(self, P, torch, device, only, rank=0, world=1):
+        BF16, F32 = torch.bfloat16, torch.float32
+        self.only = tuple(only)
+        self.inputs = inputs = make_inputs(self.only)
+
+        def pin(a, dtype):
+            return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dtype).pin_memory()
+
+        c1, c2, c3, c4, c5 = (inputs.get(k) for k in ALL)
+        x1, x2, x3 = (inputs.get(k) for k in EXTRA)
+        host_act, wts = {}, {}   # activations are copied host -> device every e2e step; weights stay resident in HBM
+        if c1:
+            host_act.update(c1x=pin(c1["x"], F32))
+            wts.update(c1w=pin(c1["w"], F32), c1b=pin(c1["b"], F32), c1g=pin(c1["gamma"], F32), c1be=pin(c1["beta"], F32))
+        if c2:
+            host_act.update(c2x=pin(c2["x"], BF16), c2r=pin(c2["r"], BF16))
+            wts.update(c2w=pin(c2["w"], BF16), c2b=pin(c2["b"], BF16))
+        if c3:
+            host_act.update(c3x=pin(c3["x"], BF16))
+            wts.update(c3w1=pin(c3["w1"], BF16), c3b1=pin(c3["b1"], BF16), c3w2=pin(c3["w2"], BF16),
+                       c3b2=pin(c3["b2"], BF16), c3g=pin(c3["gamma"], BF16), c3be=pin(c3["beta"], BF16))
+        if c4:
+            host_act.update(c4x=pin(c4["x"], BF16))
+            wts.update(c4w=pin(c4["w"], BF16))
+        if c5:
+            host_act.update(c5q=pin(c5["q"], BF16), c5k=pin(c5["k"], BF16), c5v=pin(c5["v"], BF16))
+        if x1:
+            host_act.update(x1x=pin(x1["x"], BF16))
+            wts.update(x1wq=pin(x1["w_qkv"], BF16), x1bq=pin(x1["b_qkv"], BF16), x1wo=pin(x1["w_o"], BF16),
+                       x1bo=pin(x1["b_o"], BF16), x1g=pin(x1["gamma"], BF16), x1be=pin(x1["beta"], BF16))
+        if x2:
+            host_act.update(x2x=pin(x2["x"], BF16))
+            wts.update(x2w=pin(x2["w"], BF16), x2b=pin(x2["b"], BF16))
+        x3_cols = (0, 0)
+        if x3:
+            x3_cols = P.vocab_shard_range(32000, rank, world)
+            host_act.update(x3x=pin(x3["x"], BF16))
+            wts.update(x3w=pin(x3["w"][:, x3_cols[0]:x3_cols[1]], BF16))
+        self.host_act = host_act
+        self.d = d = {k: v.to(device) for k, v in host_act.items()}
+        d.update({k: v.to(device) for k, v in wts.items()})
+        shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
+                  "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16),
+                  "X2": ((16384, 4096), BF16), "X3": ((2048, x3_cols[1] - x3_cols[0]), F32)}
+        self.out = out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in self.only}
+        self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
+        ws0 = torch.empty(256, dtype=torch.uint8, device=device)
+        ws3 = ws4 = wsx = wsx3 = ws0
+        if x3:
+            wsx3 = torch.empty(P.pike_linear_softmax_shard_workspace(d["x3x"], d["x3w"]), dtype=torch.uint8, device=device)
+        if x1:
+            wsx = torch.empty(P.pike_attention_block_workspace(d["x1x"], scale=float(x1["scale"])), dtype=torch.uint8,
+                              device=device)
+        if c3:
+            ws3 = torch.empty(P.pike_mlp_block_workspace(d["c3x"], d["c3w1"]), dtype=torch.uint8, device=device)
+        if c4:
+            ws4 = torch.empty(P.pike_linear_epilogue_workspace(d["c4x"], d["c4w"], reduce="softmax", out_dtype=F32),
+                              dtype=torch.uint8, device=device)
+        x2off = torch.from_numpy(x2["offsets"]).to(device) if x2 else None
+        if x2:
+            d["x2off_host"] = [int(o) for o in x2["offsets"]]
+        chains = {
+            "C1": lambda: P.pike_linear_epilogue(d["c1x"], d["c1w"], d["c1b"], None, d["c1g"], d["c1be"], act="gelu_erf",
+                                                 reduce="layernorm", eps=c1["eps"], out=out["C1"], workspace=ws0),
+            "C2": lambda: P.pike_linear_epilogue(d["c2x"], d["c2w"], d["c2b"], d["c2r"], act="silu", scale=0.5,
+                                                 out=out["C2"], workspace=ws0),
+            "C3": lambda: P.pike_mlp_block(d["c3x"], d["c3g"], d["c3be"], d["c3w1"], d["c3b1"], d["c3w2"], d["c3b2"],
+                                           act="gelu_tanh", eps=c3["eps"], out=out["C3"], workspace=ws3),
+            "C4": lambda: P.pike_linear_epilogue(d["c4x"], d["c4w"], reduce="softmax", out_dtype=F32, out=out["C4"],
+                                                 workspace=ws4),
+            "C5": lambda: P.pike_attention_chain(d["c5q"], d["c5k"], d["c5v"], scale=float(c5["scale"]), causal=True,
+                                                 out=out["C5"]),
+            "X1": lambda: P.pike_attention_block(d["x1x"], d["x1g"], d["x1be"], d["x1wq"], d["x1bq"], d["x1wo"], d["x1bo"],
+                                                 scale=float(x1["scale"]), causal=True, eps=x1["eps"], out=out["X1"],
+                                                 workspace=wsx),
+            "X2": lambda: P.pike_grouped_linear_epilogue(d["x2x"], d["x2w"], d["x2b"], None, x2off, act="silu",
+                                                         out=out["X2"]),
+            # the exchange between the two library calls is an all-gather of 16 KiB per rank over the default group
+            "X3": lambda: P.linear_softmax_vocab_sharded(d["x3x"], d["x3w"], out=out["X3"], workspace=wsx3),
+        }
+        self.chains = {n: chains[n] for n in chains if n in self.only}
+        self.names = list(self.chains)
+        self.attn_scale = float((c5 or x1 or {"scale": 1.0})["scale"])
+
+    def step(self, torch, events=None):
+        for n in self.names:
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            self.chains[n]()
+            if events is not None:
+                e1.record()
+                events[n].append((e0, e1))
+
+
+def timed_steps(P, torch, suite, steps, barrier, sampler=None):
+    """`steps` steps bracketed by a barrier + synchronise on both sides, timed with CUDA events on the launching
+    stream; returns (total ms, mean ms per chain, per-kernel profile, clocks)."""
+    events = {n: [] for n in suite.names}
+    if sampler is not None:
+        sampler.start()
+        sampler.wait_first_sample()
+    P.pike_profile_begin()
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        suite.step(torch, events)
+    t1.record()
+    barrier()
+    total_ms = t0.elapsed_time(t1)
+    prof = P.pike_profile_end()
+    clocks = sampler.stop() if sampler is not None else None
+    per_cfg = {n: float(np.mean([a.elapsed_time(b) for a, b in events[n]])) for n in suite.names}
+    return total_ms, per_cfg, prof, clocks
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
 
     import paper_2511_16964_b200 as P
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local_rank = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
@@ -232,101 +420,12 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=device)
     P.load_library()
 
-    BF16, F32 = torch.bfloat16, torch.float32
     only = args.only
-    inputs = make_inputs(only)
+    suite = Suite(P, torch, device, only, rank, world)
+    names = suite.names
     f = {k: v for k, v in flops_per_config().items() if k in only}
     if "X3" in f:
         f["X3"] /= world          # strong scaling: job_tflops multiplies the per-rank flops by world again
-
-    # ---- host (pinned) and device copies --------------------------------------------
-    def pin(a, dtype):
-        t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dtype)
-        return t.pin_memory()
-
-    c1, c2, c3, c4, c5 = (inputs.get(k) for k in ALL)
-    host_act, wts = {}, {}   # activations are copied host -> device every e2e step; weights stay resident in HBM
-    if c1:
-        host_act.update(c1x=pin(c1["x"], F32))
-        wts.update(c1w=pin(c1["w"], F32), c1b=pin(c1["b"], F32), c1g=pin(c1["gamma"], F32), c1be=pin(c1["beta"], F32))
-    if c2:
-        host_act.update(c2x=pin(c2["x"], BF16), c2r=pin(c2["r"], BF16))
-        wts.update(c2w=pin(c2["w"], BF16), c2b=pin(c2["b"], BF16))
-    if c3:
-        host_act.update(c3x=pin(c3["x"], BF16))
-        wts.update(c3w1=pin(c3["w1"], BF16), c3b1=pin(c3["b1"], BF16), c3w2=pin(c3["w2"], BF16),
-                   c3b2=pin(c3["b2"], BF16), c3g=pin(c3["gamma"], BF16), c3be=pin(c3["beta"], BF16))
-    if c4:
-        host_act.update(c4x=pin(c4["x"], BF16))
-        wts.update(c4w=pin(c4["w"], BF16))
-    if c5:
-        host_act.update(c5q=pin(c5["q"], BF16), c5k=pin(c5["k"], BF16), c5v=pin(c5["v"], BF16))
-    x1 = inputs.get("X1")
-    if x1:
-        host_act.update(x1x=pin(x1["x"], BF16))
-        wts.update(x1wq=pin(x1["w_qkv"], BF16), x1bq=pin(x1["b_qkv"], BF16), x1wo=pin(x1["w_o"], BF16),
-                   x1bo=pin(x1["b_o"], BF16), x1g=pin(x1["gamma"], BF16), x1be=pin(x1["beta"], BF16))
-    x2 = inputs.get("X2")
-    if x2:
-        host_act.update(x2x=pin(x2["x"], BF16))
-        wts.update(x2w=pin(x2["w"], BF16), x2b=pin(x2["b"], BF16))
-    x3 = inputs.get("X3")
-    x3_cols = (0, 0)
-    if x3:
-        x3_cols = P.vocab_shard_range(32000, rank, world)
-        host_act.update(x3x=pin(x3["x"], BF16))
-        wts.update(x3w=pin(x3["w"][:, x3_cols[0]:x3_cols[1]], BF16))
-    d = {k: v.to(device) for k, v in host_act.items()}
-    d.update({k: v.to(device) for k, v in wts.items()})
-    shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
-              "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16), "X2": ((16384, 4096), BF16),
-              "X3": ((2048, x3_cols[1] - x3_cols[0]), F32)}
-    out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in only}
-    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
-    ws0 = torch.empty(256, dtype=torch.uint8, device=device)
-    ws3 = ws4 = wsx = wsx3 = ws0
-    if x3:
-        wsx3 = torch.empty(P.pike_linear_softmax_shard_workspace(d["x3x"], d["x3w"]), dtype=torch.uint8, device=device)
-    if x1:
-        wsx = torch.empty(P.pike_attention_block_workspace(d["x1x"], scale=float(x1["scale"])), dtype=torch.uint8,
-                          device=device)
-    if c3:
-        ws3 = torch.empty(P.pike_mlp_block_workspace(d["c3x"], d["c3w1"]), dtype=torch.uint8, device=device)
-    if c4:
-        ws4 = torch.empty(P.pike_linear_epilogue_workspace(d["c4x"], d["c4w"], reduce="softmax", out_dtype=F32),
-                          dtype=torch.uint8, device=device)
-
-    x2off = torch.from_numpy(x2["offsets"]).to(device) if x2 else None
-    chains = {
-        "C1": lambda: P.pike_linear_epilogue(d["c1x"], d["c1w"], d["c1b"], None, d["c1g"], d["c1be"], act="gelu_erf",
-                                             reduce="layernorm", eps=c1["eps"], out=out["C1"], workspace=ws0),
-        "C2": lambda: P.pike_linear_epilogue(d["c2x"], d["c2w"], d["c2b"], d["c2r"], act="silu", scale=0.5,
-                                             out=out["C2"], workspace=ws0),
-        "C3": lambda: P.pike_mlp_block(d["c3x"], d["c3g"], d["c3be"], d["c3w1"], d["c3b1"], d["c3w2"], d["c3b2"],
-                                       act="gelu_tanh", eps=c3["eps"], out=out["C3"], workspace=ws3),
-        "C4": lambda: P.pike_linear_epilogue(d["c4x"], d["c4w"], reduce="softmax", out_dtype=F32, out=out["C4"],
-                                             workspace=ws4),
-        "C5": lambda: P.pike_attention_chain(d["c5q"], d["c5k"], d["c5v"], scale=float(c5["scale"]), causal=True,
-                                             out=out["C5"]),
-        "X1": lambda: P.pike_attention_block(d["x1x"], d["x1g"], d["x1be"], d["x1wq"], d["x1bq"], d["x1wo"], d["x1bo"],
-                                             scale=float(x1["scale"]), causal=True, eps=x1["eps"], out=out["X1"],
-                                             workspace=wsx),
-        "X2": lambda: P.pike_grouped_linear_epilogue(d["x2x"], d["x2w"], d["x2b"], None, x2off, act="silu",
-                                                     out=out["X2"]),
-        # the exchange between the two library calls is an all-gather of 16 KiB per rank over the default group
-        "X3": lambda: P.linear_softmax_vocab_sharded(d["x3x"], d["x3w"], out=out["X3"], workspace=wsx3),
-    }
-    names = [n for n in chains if n in only]
-
-    def step(events=None):
-        for n in names:
-            if events is not None:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-            chains[n]()
-            if events is not None:
-                e1.record()
-                events[n].append((e0, e1))
 
     def barrier():
         if world > 1:
@@ -335,35 +434,22 @@ def run_ours(args):
 
     # ---- warm-up, then the timed region ------------------------------------------------
     for _ in range(args.warmup):
-        step()
+        suite.step(torch)
     barrier()
     st, where = P.pike_get_last_device_status()
     if st != 0:
         raise SystemExit(f"device status {st} at {where:#x} during warm-up")
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    events = {n: [] for n in names}
-    P.pike_profile_begin()
-    barrier()
-    t_start, t_stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t_start.record()
-    for _ in range(args.steps):
-        step(events)
-    t_stop.record()
-    barrier()
-    total_ms = t_start.elapsed_time(t_stop)
-    prof = P.pike_profile_end()
-    clocks = sampler.stop() if rank == 0 else None
+    total_ms, per_cfg_ms, prof, clocks = timed_steps(P, torch, suite, args.steps, barrier,
+                                                     ClockSampler(local_rank) if rank == 0 else None)
     total_ms = max_over_ranks(total_ms, world, device)
     ms_per_step = total_ms / args.steps
     step_flops = sum(f.values())
     value = job_tflops(step_flops, world, ms_per_step)
-    per_cfg_ms = {n: float(np.mean([a.elapsed_time(b) for a, b in events[n]])) for n in names}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ---
     e2e_steps = max(1, min(args.steps, 5))
+    host_act, host_out, d, out, chains = suite.host_act, suite.host_out, suite.d, suite.out, suite.chains
     h2d = sum(v.numel() * v.element_size() for v in host_act.values())
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
 
@@ -426,74 +512,118 @@ def run_ours(args):
         torch.cuda.synchronize()
         warm_ms[n] = w0.elapsed_time(w1) / 20
 
+    # ---- sustained: the same step looped for seconds, clocks sampled: the power-capped regime ------------
+    sustained = None
+    peaks = load_peaks()
+    if args.sustained_seconds > 0 and tuple(only) == ALL:
+        n_steps = max(args.steps, int(args.sustained_seconds * 1e3 / ms_per_step) + 1)
+        s_ms, s_cfg, s_prof, s_clocks = timed_steps(P, torch, suite, n_steps, barrier,
+                                                    ClockSampler(local_rank, 50) if rank == 0 else None)
+        s_ms = max_over_ranks(s_ms, world, device)
+        gl, gms = s_prof["gemm_bf16"]
+        gtf = sum(gemm_kernel_flops()[k] for k in ("C2", "C3", "C4")) * n_steps / (gms * 1e-3) / 1e12
+        sustained = {
+            "steps": n_steps, "seconds": s_ms * 1e-3, "ms_per_step": s_ms / n_steps,
+            "value": job_tflops(step_flops, world, s_ms / n_steps), "unit": UNIT, "clocks": s_clocks,
+            "per_config": {n: {"ms": s_cfg[n], "tflops": f[n] / (s_cfg[n] * 1e-3) / 1e12,
+                               "frac_of_nominal_2250": f[n] / (s_cfg[n] * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
+                               "meets_60pct_of_nominal": bool(f[n] / (s_cfg[n] * 1e-3) / 1e12 >= 0.6 * NOMINAL_BF16_TFLOPS)}
+                           for n in names},
+            "roofline": {"kernel": "gemm_bf16_kernel", "bound": "tensor", "achieved": gtf,
+                         "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": gtf / peaks["bf16_tflops_sustained"],
+                         "peak_source": f"{peaks['source']} cuBLAS bf16, sustained figure",
+                         "frac_of_nominal_2250": gtf / NOMINAL_BF16_TFLOPS, "launches": gl},
+            "kernels": {k: {"launches": v[0], "ms_per_step": v[1] / n_steps} for k, v in s_prof.items()},
+        }
+
     if rank != 0:
         if world > 1:
             dist.barrier()
             dist.destroy_process_group()
         return 0
 
-    # ---- rank 0 only: eager comparison, parity spot check, CPU baseline, JSON ------------
-    peaks = load_peaks()
+    # ---- rank 0 only: eager comparison, context rows, further workloads, parity, CPU baseline, JSON -------
     gemm_launches, gemm_ms = prof["gemm_bf16"]
-    gemm_flops = sum(f.get(k, 0.0) for k in ("C2", "C3", "C4"))      # the launches of the bf16 GEMM kernel
-    if "X1" in f:
-        gemm_flops += 2.0 * 16384 * 4096 * (4 * 4096)
-    gemm_flops += f.get("X2", 0.0) + f.get("X3", 0.0)
+    gkf = gemm_kernel_flops()
+    gemm_flops = sum(gkf[k] / (world if k == "X3" else 1) for k in gkf if k in f)
     gemm_tflops = gemm_flops * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
     # a long timed region runs under the power cap: compare with the sustained library figure
-    sustained = total_ms > 500.0 or "sw_power_cap" in (clocks or {}).get("reasons", [])
-    peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    capped = total_ms > 500.0 or "sw_power_cap" in (clocks or {}).get("reasons", [])
+    peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
+    cap = GEMM_DRAM_CAPTURE
+    traffic_valid = tuple(only) == ALL and cap["bytes"] is not None and cap["sources_sha16"] == sources_sha16()
     roofline = {
         "kernel": "gemm_bf16_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": peak, "unit": "TFLOP/s",
-        "frac": (gemm_tflops / peak) if gemm_tflops else None, "peak_source": f"{peaks['source']} cuBLAS bf16, {'sustained' if sustained else 'burst'} figure",
+        "frac": (gemm_tflops / peak) if gemm_tflops else None,
+        "peak_source": f"{peaks['source']} cuBLAS bf16, {'sustained' if capped else 'burst'} figure",
         "frac_of_nominal_2250": (gemm_tflops / NOMINAL_BF16_TFLOPS) if gemm_tflops else None,
         "launches": gemm_launches,
-        # DRAM bytes of the kernel's four launches of one step, from the ncu capture summarised under profiles/
-        # (per-step DRAM bytes of this kernel); null for partial suites, and to be reset to null whenever the
-        # kernel changes after that capture
-        "traffic": GEMM_DRAM_BYTES_PER_STEP if tuple(only) == ALL else None,
+        # DRAM bytes of the kernel's four launches of one step from the ncu captures summarised under profiles/;
+        # null for partial suites and whenever the kernel's sources no longer hash to the captured build
+        "traffic": cap["bytes"] if traffic_valid else None,
+        "traffic_min_max": [cap["min"], cap["max"]] if traffic_valid else None,
+        "traffic_captures": cap["captures"] if traffic_valid else None,
+        "traffic_sources_sha16": cap["sources_sha16"], "sources_sha16_now": sources_sha16(),
         "traffic_unit": "bytes per step (4 launches)", "algorithmic_bytes": GEMM_ALGORITHMIC_BYTES_PER_STEP,
     }
 
-    if x2:
-        d["x2off_host"] = [int(o) for o in x2["offsets"]]
-    if x3 and not args.no_eager:   # the eager comparison is the unsharded chain on one GPU
-        d["x3w_full"] = pin(x3["w"], BF16).to(device)
-    eager_ms = {} if args.no_eager else eager_baseline(torch, d, c1, c3, c5 or x1, names)
-    library_gemm = None if args.no_eager else library_gemm_context(torch, device, sampler.__class__(local_rank))
+    if "X3" in only and not args.no_eager:   # the eager comparison is the unsharded chain on one GPU
+        d["x3w_full"] = torch.from_numpy(np.ascontiguousarray(suite.inputs["X3"]["w"], np.float32)).to(torch.bfloat16).to(device)
+    eager_ms = {} if args.no_eager else eager_baseline(torch, d, suite.attn_scale, names)
+    context = None if (args.no_eager or args.no_context) else context_rows(torch, d, suite.attn_scale, names)
+    library_gemm = None if args.no_eager else library_gemm_context(torch, device, ClockSampler(local_rank, 50))
     if tuple(only) != ALL:
-        args.no_parity = args.no_cpu_baseline = True                 # partial suites are profiling runs
-    per_config = {}
-    for n in names:
-        per_config[n] = {"ms": per_cfg_ms[n], "tflops": f[n] / (per_cfg_ms[n] * 1e-3) / 1e12,
-                         "frac_of_nominal_2250": f[n] / (per_cfg_ms[n] * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
-        per_config[n]["warm_ms"] = warm_ms[n]
-        if n in eager_ms:
-            per_config[n]["eager_ms"] = eager_ms[n]
-            per_config[n]["speedup_vs_eager"] = eager_ms[n] / per_cfg_ms[n]
+        args.no_parity = args.no_cpu_baseline = args.no_extras = True      # partial suites are profiling runs
+
+    def config_row(n, ms, fl, warm=None, eager=None):
+        row = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_nominal_2250": fl / (ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+        row["meets_60pct_of_nominal"] = bool(row["frac_of_nominal_2250"] >= 0.6)
+        if warm is not None:
+            row["warm_ms"] = warm
+        if eager is not None:
+            row["eager_ms"] = eager
+            row["speedup_vs_eager"] = eager / ms
+        return row
+
+    per_config = {n: config_row(n, per_cfg_ms[n], f[n], warm_ms[n], eager_ms.get(n)) for n in names}
     kernels = {k: {"launches": v[0], "ms_per_step": v[1] / args.steps} for k, v in prof.items()}
     # the other kernels of the default step against their own bounds (algorithmic bytes / flops per launch)
     if tuple(only) == ALL:
-        def _bw(name, nbytes):
-            ms = kernels[name]["ms_per_step"]
+        def _bw(name, nbytes, into=kernels):
+            ms = into[name]["ms_per_step"]
             gbs = nbytes / (ms * 1e-3) / 1e9 if ms > 0 else None
-            kernels[name].update(bound="hbm", achieved=gbs, unit="GB/s", peak=peaks["hbm_gbs"],
-                                 frac=(gbs / peaks["hbm_gbs"]) if gbs else None)
-        _bw("layernorm_bf16", 2.0 * 8192 * 4096 * 2)                      # C3 prologue: x in, z out
-        _bw("softmax_finish", 2.0 * 2048 * 32000 * 4 + 2048 * 125 * 8)    # C4: logits in, probabilities out, pairs
-        ms = kernels["attention_bf16"]["ms_per_step"]
-        tf = f["C5"] / (ms * 1e-3) / 1e12 if ms > 0 else None
-        kernels["attention_bf16"].update(bound="tensor + sfu", achieved=tf, unit="TFLOP/s", peak=peak,
-                                         frac=(tf / peak) if tf else None)
+            into[name].update(bound="hbm", achieved=gbs, unit="GB/s", peak=peaks["hbm_gbs"],
+                              frac=(gbs / peaks["hbm_gbs"]) if gbs else None)
+        for block, pk in ((kernels, peak), (sustained["kernels"] if sustained else None, peaks["bf16_tflops_sustained"])):
+            if block is None:
+                continue
+            _bw("layernorm_bf16", 2.0 * 8192 * 4096 * 2, block)                      # C3 prologue: x in, z out
+            _bw("softmax_finish", 2.0 * 2048 * 32000 * 4 + 2048 * 125 * 8, block)    # C4: logits in, probabilities out, pairs
+            ms = block["attention_bf16"]["ms_per_step"]
+            tf = f["C5"] / (ms * 1e-3) / 1e12 if ms > 0 else None
+            block["attention_bf16"].update(bound="tensor + sfu", achieved=tf, unit="TFLOP/s", peak=pk,
+                                           frac=(tf / pk) if tf else None,
+                                           frac_of_nominal_2250=(tf / NOMINAL_BF16_TFLOPS) if tf else None)
 
-    parity = None if args.no_parity else parity_spot_check(inputs, out)
+    parity = None if args.no_parity else parity_spot_check(suite.inputs, out)
+    host_call_us = None if tuple(only) != ALL else host_call_overhead(P, torch, suite)
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
         from oracle import pike_oracle as O
-        fl, dt = oracle_sample_step(inputs)
+        fl, dt, per = oracle_sample_step(suite.inputs)
+        full = oracle_full_size_seconds(per)
         cpu_baseline = {"value": fl / dt / 1e12, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-                        "sample": oracle_sample_text(), "seconds": dt}
+                        "sample": oracle_sample_text(), "seconds": dt,
+                        "full_size_seconds_extrapolated": sum(full.values()), "full_size_seconds_per_config": full}
+
+    # ---- the further workloads (outside `value`): one at a time, each with its own tensors ---------------
+    if world == 1 and not args.no_extras:
+        del suite, d, out, chains, host_act, host_out
+        torch.cuda.empty_cache()
+        for x in EXTRA:
+            per_config[x] = extra_workload(P, torch, device, x, not args.no_eager)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -508,6 +638,8 @@ def run_ours(args):
                          "so every chain starts with its inputs evicted",
                    "warm_ms": "per_config.warm_ms = the same chain 20 times back to back without per-kernel events "
                               "(short bursts run at higher clocks; for C1 it is the host's call rate)",
+                   "extras": "per_config X1..X3 are further workloads timed after the step (10 runs each, tensors "
+                             "larger than L2), not part of value",
                    "weights": "resident in HBM", "flops": "GEMM multiply-adds x2; attention counts the causal half"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
@@ -516,7 +648,8 @@ def run_ours(args):
         "gpu_launches": int(sum(v[0] for v in prof.values())),
         "roofline": roofline, "cpu_baseline": cpu_baseline,
         "frac_of_nominal_2250": value / world / NOMINAL_BF16_TFLOPS,
-        "per_config": per_config, "kernels": kernels, "parity": parity, "library_gemm_same_box": library_gemm,
+        "sustained": sustained, "per_config": per_config, "context": context, "kernels": kernels, "parity": parity,
+        "host_call_us": host_call_us, "library_gemm_same_box": library_gemm,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -525,12 +658,99 @@ def run_ours(args):
     return 0
 
 
-def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
-    """The same ops as separate PyTorch calls (TF32 off); ms per config."""
+def extra_workload(P, torch, device, name, with_eager, iters=10):
+    """One of X1..X3 on its own: 3 warm-up runs, then `iters` runs timed one by one with CUDA events."""
+    s = Suite(P, torch, device, (name,))
+    fl = flops_per_config()[name]
+    for _ in range(3):
+        s.chains[name]()
+    torch.cuda.synchronize()
+    ts = []
+    P.pike_profile_begin()
+    for _ in range(iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        s.chains[name]()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    prof = P.pike_profile_end()
+    ms = float(np.mean(ts))
+    row = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12, "frac_of_nominal_2250": fl / (ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
+           "min_ms": float(min(ts)), "runs": iters, "in_value": False,
+           "kernels": {k: {"launches": v[0] // iters, "ms": v[1] / iters} for k, v in prof.items() if v[0]}}
+    gms = prof["gemm_bf16"][1] / iters
+    if gms > 0:
+        row["gemm_kernel_tflops"] = gemm_kernel_flops()[name] / (gms * 1e-3) / 1e12
+    if with_eager:
+        if name == "X3":
+            s.d["x3w_full"] = s.d["x3w"]
+        e = eager_baseline(torch, s.d, s.attn_scale, [name])
+        row["eager_ms"] = e[name]
+        row["speedup_vs_eager"] = e[name] / ms
+    st, where = P.pike_get_last_device_status()
+    row["device_status"] = st
+    del s
+    torch.cuda.empty_cache()
+    return row
+
+
+def host_call_overhead(P, torch, suite, calls=400):
+    """Microseconds of host time one library call costs, without the Python wrappers: the C entry point is
+    called through ctypes with argument structs built once, and only the enqueue loop is timed (the queue is
+    drained before and after, and `calls` stays below the depth at which launches start to block)."""
+    import ctypes
+    from paper_2511_16964_b200 import binding as B
+    lib, d, out = B.load_library(), suite.d, suite.out
+    h = B._handle(out["C1"].device)
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    res = {}
+    e1 = B._epilogue("gelu_erf", 1.0, "layernorm", 1e-5, torch.float32, 0)
+    a1 = [B._tensor(d[k]) for k in ("c1x", "c1w", "c1b")] + [None] + [B._tensor(d[k]) for k in ("c1g", "c1be")]
+    o1 = B._tensor(out["C1"])
+    e2 = B._epilogue("silu", 0.5, "none", 0.0, torch.bfloat16, 0)
+    a2 = [B._tensor(d[k]) for k in ("c2x", "c2w", "c2b", "c2r")] + [None, None]
+    o2 = B._tensor(out["C2"])
+    for name, args_, e, o, n in (("pike_linear_epilogue_fp32_128x256x256", a1, e1, o1, calls),
+                                 ("pike_linear_epilogue_bf16_4096^3", a2, e2, o2, 60)):
+        for _ in range(3):
+            lib.pike_linear_epilogue(h, *args_, ctypes.byref(e), o, None, 0, stream)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n):
+            lib.pike_linear_epilogue(h, *args_, ctypes.byref(e), o, None, 0, stream)
+        t1 = time.perf_counter()
+        torch.cuda.synchronize()
+        res[name] = (t1 - t0) / n * 1e6
+    # the same fp32 call through the Python wrapper, for comparison
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        suite.chains["C1"]()
+    t1 = time.perf_counter()
+    torch.cuda.synchronize()
+    res["python_wrapper_fp32_128x256x256"] = (t1 - t0) / calls * 1e6
+    return res
+
+
+def _timed_cold(torch, fn, flush, iters=3):
+    fn()
+    fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return float(np.mean(ts))
+
+
+def eager_ops(torch, d, scale):
     F = torch.nn.functional
-    torch.backends.cuda.matmul.allow_tf32 = False
-    torch.backends.cudnn.allow_tf32 = False
-    scale = float(c5["scale"]) if c5 else 1.0
 
     def attn():
         q, k, v = d["c5q"], d["c5k"], d["c5v"]
@@ -539,18 +759,6 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         mask = torch.ones((S, S), dtype=torch.bool, device=q.device).tril()
         s = s.masked_fill(~mask, float("-inf"))
         return torch.softmax(s, dim=-1) @ v
-
-    ops = {
-        "C1": lambda: F.layer_norm(F.gelu(d["c1x"] @ d["c1w"] + d["c1b"]), (256,), d["c1g"], d["c1be"], 1e-5),
-        "C2": lambda: 0.5 * F.silu(d["c2x"] @ d["c2w"] + d["c2b"]) + d["c2r"],
-        "C3": lambda: d["c3x"] + F.gelu(F.layer_norm(d["c3x"], (4096,), d["c3g"], d["c3be"], 1e-5) @ d["c3w1"]
-                                        + d["c3b1"], approximate="tanh") @ d["c3w2"] + d["c3b2"],
-        "C4": lambda: torch.softmax(d["c4x"] @ d["c4w"], dim=-1, dtype=torch.float32),
-        "C5": attn,
-        "X1": lambda: x1_eager(),
-        "X2": lambda: x2_eager(),
-        "X3": lambda: torch.softmax(d["x3x"] @ d["x3w_full"], dim=-1, dtype=torch.float32),
-    }
 
     def x2_eager():     # the per-expert loop the grouped kernel replaces
         off = d["x2off_host"]
@@ -569,23 +777,60 @@ def eager_baseline(torch, d, c1, c3, c5, names, iters=3):
         mask = torch.ones((S, S), dtype=torch.bool, device=x.device).tril()
         a = (torch.softmax(sc.masked_fill(~mask, float("-inf")), dim=-1) @ v).permute(0, 2, 1, 3).reshape(B, S, E)
         return x + a @ d["x1wo"] + d["x1bo"]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=next(v for v in d.values() if hasattr(v, "device")).device)
-    res = {}
-    for n in names:
-        ops[n]()
-        ops[n]()
-        torch.cuda.synchronize()
-        ts = []
-        for _ in range(iters):
-            flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            ops[n]()
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        res[n] = float(np.mean(ts))
-    return res
+
+    return {
+        "C1": lambda: F.layer_norm(F.gelu(d["c1x"] @ d["c1w"] + d["c1b"]), (256,), d["c1g"], d["c1be"], 1e-5),
+        "C2": lambda: 0.5 * F.silu(d["c2x"] @ d["c2w"] + d["c2b"]) + d["c2r"],
+        "C3": lambda: d["c3x"] + F.gelu(F.layer_norm(d["c3x"], (4096,), d["c3g"], d["c3be"], 1e-5) @ d["c3w1"]
+                                        + d["c3b1"], approximate="tanh") @ d["c3w2"] + d["c3b2"],
+        "C4": lambda: torch.softmax(d["c4x"] @ d["c4w"], dim=-1, dtype=torch.float32),
+        "C5": attn,
+        "X1": x1_eager,
+        "X2": x2_eager,
+        "X3": lambda: torch.softmax(d["x3x"] @ d["x3w_full"], dim=-1, dtype=torch.float32),
+    }
+
+
+def eager_baseline(torch, d, scale, names, iters=3):
+    """The same ops as separate PyTorch calls (TF32 off); ms per config, L2 flushed before every timed run."""
+    torch.backends.cuda.matmul.allow_tf32 = False
+    torch.backends.cudnn.allow_tf32 = False
+    ops = eager_ops(torch, d, scale)
+    device = next(v for v in d.values() if hasattr(v, "device")).device
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    return {n: _timed_cold(torch, ops[n], flush, iters) for n in names}
+
+
+def context_rows(torch, d, scale, names, budget_s=150.0):
+    """Context only, never a denominator: the same chains through the library's fused attention
+    (scaled_dot_product_attention) and through torch.compile (default mode), timed like the eager baseline.
+    A row that fails or would exceed the time budget is reported as null with the reason."""
+    F = torch.nn.functional
+    device = next(v for v in d.values() if hasattr(v, "device")).device
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    rows, t_start = {}, time.perf_counter()
+    if "C5" in names:
+        try:
+            rows["C5_sdpa_ms"] = _timed_cold(
+                torch, lambda: F.scaled_dot_product_attention(d["c5q"], d["c5k"], d["c5v"], is_causal=True, scale=scale),
+                flush)
+        except Exception as exc:       # noqa: BLE001 - a context row must never break the benchmark
+            rows["C5_sdpa_ms"], rows["C5_sdpa_error"] = None, repr(exc)[:200]
+    ops = eager_ops(torch, d, scale)
+    for n in ("C2", "C3", "C5"):
+        if n not in names:
+            continue
+        if time.perf_counter() - t_start > budget_s:
+            rows[f"{n}_compile_ms"], rows[f"{n}_compile_error"] = None, "time budget for context rows used up"
+            continue
+        try:
+            fn = torch.compile(ops[n])
+            rows[f"{n}_compile_ms"] = _timed_cold(torch, fn, flush)
+        except Exception as exc:       # noqa: BLE001
+            rows[f"{n}_compile_ms"], rows[f"{n}_compile_error"] = None, repr(exc)[:200]
+    rows["seconds_spent"] = time.perf_counter() - t_start
+    rows["note"] = "C5_sdpa = torch scaled_dot_product_attention (is_causal); *_compile = torch.compile(default) of the eager composition"
+    return rows
 
 
 def library_gemm_context(torch, device, sampler, seconds=0.6):
@@ -650,7 +895,7 @@ def parity_spot_check(inputs, out):
     return res
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
@@ -658,15 +903,24 @@ def main():
     ap.add_argument("--only", type=lambda v: tuple(x for x in ALL + EXTRA if x in v.split(",")), default=ALL,
                     help="comma-separated subset of C1..C5 and X1..X3 (profiling runs; the default is the whole suite C1..C5)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="length of the sustained loop reported beside the K timed steps (0 = skip)")
     ap.add_argument("--no-eager", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the scaled_dot_product_attention / torch.compile rows")
+    ap.add_argument("--no-extras", action="store_true", help="skip the further workloads X1..X3")
     ap.add_argument("--no-parity", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     # the oracle pass is ~10-30 s of CPU work: bound the number of passes
     args.ref_steps = max(1, min(args.steps, 3))
     args.ref_warmup = 1 if args.warmup > 0 else 0
+    return args
+
+
+def main(argv=None):
+    args = parse_args(argv)
     return run_reference(args) if args.impl == "reference" else run_ours(args)
 
 
