@@ -52,19 +52,22 @@ constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_
 
 enum : uint32_t { BAR_EMPTY = 1, BAR_FULL = 2, BAR_TMEM_EMPTY = 3, BAR_TMEM_FULL = 4 };
 
-// Rasterisation: tiles are walked in groups of group_m pair-row-blocks, all column blocks of a group
-// before the next group, row-block fastest.  The clusters that run together therefore share a few row
-// blocks and a few column blocks (their k-slices meet in L2), and the group's rows of A stay in L2 for
-// the whole column sweep, so W is streamed from HBM once per group.
-__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int group_m, int &m_blk, int &n_blk)
+// Rasterisation: tiles are walked in groups of `group` blocks of one dimension (the PANEL dimension), all blocks
+// of the other dimension before the next group, panel block fastest.  The clusters that run together therefore
+// share a few row blocks and a few column blocks (their k-slices meet in L2), and the group's panel - group x 256
+// rows of A, or group x 256 columns of W - stays in L2 for the whole sweep while the other operand streams through
+// once per group.  along_n == 0: the panel is a group of row blocks of A; 1: a group of column blocks of W.
+__device__ __forceinline__ void tile_coords(int t, int num_m, int num_n, int group, int along_n, int &m_blk, int &n_blk)
 {
-    const int per_group = group_m * num_n;
+    const int num_p = along_n ? num_n : num_m, num_s = along_n ? num_m : num_n;
+    const int per_group = group * num_s;
     const int g = t / per_group;
-    const int first_m = g * group_m;
-    const int gsz = min(group_m, num_m - first_m);
+    const int first_p = g * group;
+    const int gsz = min(group, num_p - first_p);
     const int r = t - g * per_group;
-    m_blk = first_m + r % gsz;
-    n_blk = r / gsz;
+    const int p_blk = first_p + r % gsz, s_blk = r / gsz;
+    m_blk = along_n ? s_blk : p_blk;
+    n_blk = along_n ? p_blk : s_blk;
 }
 
 // Work items.  The tiles are dealt round-robin to the persistent clusters, so the last, partial round leaves
@@ -169,7 +172,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int w = cluster_id; w < plan.items && !p.test_withhold_loads; w += num_clusters) {
                 const Work wk = work_item(plan, w);
                 int m_blk, n_blk;
-                tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
+                tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
                 const RowTile rt = row_tile(p, m_blk);
                 if (rt.row0 >= rt.row_end) continue;        // empty row tile (grouped mode): every role skips it
                 const int row0 = rt.row0 + (int)rank * BM;
@@ -215,7 +218,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const Work wk = work_item(plan, w);
                 if (p.group_offsets != nullptr) {
                     int m_blk, n_blk;
-                    tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
+                    tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
                     const RowTile rt = row_tile(p, m_blk);
                     if (rt.row0 >= rt.row_end) continue;
                 }
@@ -255,7 +258,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int w = cluster_id; w < plan.items; w += num_clusters) {
             const Work wk = work_item(plan, w);
             int m_blk, n_blk;
-            tile_coords(wk.tile, num_m, num_n, p.group_m, m_blk, n_blk);
+            tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
             const RowTile rt = row_tile(p, m_blk);
             if (rt.row0 >= rt.row_end) continue;
             const int acc = it & 1;
@@ -471,18 +474,30 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
     const int num_n = (a.N + BN - 1) / BN;
     const long long num_tiles = (long long)num_m * num_n;
     if (num_tiles <= 0 || a.M <= 0 || max_clusters <= 0) return cudaSuccess;
-    // Row blocks per rasterisation group.  Measured on B200 (DRAM bytes of the two MLP GEMMs): HBM reads
-    // are lowest when the group's rows of A (group_m x 256 x K bf16) stay within about 32 MB - a quarter
-    // of the 126 MB L2, which is split over two dies and shared with the streaming W and output traffic -
-    // and never below 8 groups rows, where the clusters running together (74 = about 8 x 9 tiles) share
-    // the fewest distinct k-slices: 1169 -> 402 MB for 8192x4096x16384, 1501 -> 1322 MB for 8192x16384x4096.
+    // Rasterisation.  Both operands come in slabs of 256 x K 16-bit values (a pair-row-block of A, a column block
+    // of W).  One of them is the PANEL: a group of its slabs is walked against all slabs of the other operand, so
+    // the panel is fetched once and the other operand once per group:
+    //   traffic(panel = A) = bytes(A) + bytes(W) * groups_of_A,   traffic(panel = W) = bytes(W) + bytes(A) * groups_of_W
+    // and the cheaper one is taken (the MLP's second GEMM, K = 16384, reads 11 % less with W as the panel).  A group
+    // holds as many slabs as fit in PANEL_BYTES, at least 8 (with fewer the clusters that run together - 74 = about
+    // 8 x 9 tiles - span too many slabs of the streaming operand).  Measured on B200 (DRAM bytes of the two MLP
+    // GEMMs): a panel is only kept below about 32 MB - a quarter of the 126 MB L2, which is split over two dies and
+    // shared with the streaming operand and the output: 1169 -> 402 MB for 8192x4096x16384.  L2 eviction priorities
+    // on the loads (evict_last for the panel, evict_first or normal for the stream) were measured too and made the
+    // reads worse by 40 to 110 %: a streamed slab is shared by the eight or nine clusters that run side by side, and
+    // lowering its priority evicts it between their reads.
     GemmArgs args = a;
     {
-        const long long row_block_bytes = 2ll * BM * a.K * 2;
-        long long g = (33ll << 20) / (row_block_bytes > 0 ? row_block_bytes : 1);
+        constexpr long long PANEL_BYTES = 33ll << 20;
+        const long long slab = 2ll * BM * a.K * 2;
+        long long g = PANEL_BYTES / (slab > 0 ? slab : 1);
         if (g < 8) g = 8;
-        if (g > num_m) g = num_m;
-        args.group_m = (int)g;
+        const long long gm = g < num_m ? g : num_m, gn = g < num_n ? g : num_n;
+        const long long groups_m = (num_m + gm - 1) / gm, groups_n = (num_n + gn - 1) / gn;
+        const double bytes_a = 2.0 * a.M * a.K, bytes_w = 2.0 * a.K * a.N;
+        const bool along_n = a.group_offsets == nullptr && bytes_w + bytes_a * groups_n < bytes_a + bytes_w * groups_m;
+        args.group_along_n = along_n ? 1 : 0;
+        args.group_m = (int)(along_n ? gn : gm);
     }
     // up to two work items per tile (see work_plan): small problems get both halves of a tile onto
     // different clusters

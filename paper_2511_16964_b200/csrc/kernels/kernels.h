@@ -51,7 +51,9 @@ struct GemmArgs {
     // matrix e (third coordinate of the W tensor map) and bias row e; M is the total row count
     const int *group_offsets;  // device, num_groups + 1 ints
     int num_groups;
-    int group_m;              // set by the launcher: pair-row-blocks per rasterisation group
+    // set by the launcher: the rasterisation (see tile_coords)
+    int group_m;              // blocks per rasterisation group (row blocks, or column blocks if group_along_n)
+    int group_along_n;        // 0: groups of row blocks, W streams; 1: groups of column blocks, A streams
     int test_withhold_loads;  // test hook: the producers issue no loads, so the first "full" wait runs out
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
