@@ -242,6 +242,16 @@ def rank_env():
             int(os.environ.get("LOCAL_RANK", "0")))
 
 
+def per_rank_flops(only, world: int) -> dict:
+    """GEMM flops ONE rank processes per step, per workload.  C1..C5, X1, X2 are replicated (every rank runs the
+    whole workload on its own rows or heads: weak scaling, job_tflops multiplies by world); X3 splits the columns of
+    one problem over the ranks (strong scaling), so a rank does 1/world of it."""
+    f = {k: v for k, v in flops_per_config().items() if k in only}
+    if "X3" in f:
+        f["X3"] /= world
+    return f
+
+
 def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
@@ -423,9 +433,7 @@ def run_ours(args):
     only = args.only
     suite = Suite(P, torch, device, only, rank, world)
     names = suite.names
-    f = {k: v for k, v in flops_per_config().items() if k in only}
-    if "X3" in f:
-        f["X3"] /= world          # strong scaling: job_tflops multiplies the per-rank flops by world again
+    f = per_rank_flops(only, world)
 
     def barrier():
         if world > 1:
