@@ -18,7 +18,7 @@ Beside the contract's keys the line carries:
   sustained   the same step looped for at least two seconds with the clocks sampled: the
               power-capped regime, with its own roofline against the sustained library figure
   per_config  per chain: ms, TFLOP/s, fraction of the nominal 2250 TFLOP/s, eager time and
-              speed-up; X1..X3 (the further workloads, outside `value`) when N == 1
+              speed-up; X1..X4 (the further workloads, outside `value`) when N == 1
   context     other ways to run the same chains on this GPU (fused library attention,
               torch.compile): context rows, never a denominator
   kernels     live device time per kernel of the library, with its own bound
@@ -80,6 +80,8 @@ def flops_per_config():
         # X3 (not part of the default step): C4's logits + softmax with the 32000 columns split over the ranks
         # (whole-job flops; every rank does 1/world of them)
         "X3": 2.0 * 2048 * 4096 * 32000,
+        # X4 (not part of the default step): C4's logits + softmax as ONE kernel (PIKE_FLAG_ONE_PASS)
+        "X4": 2.0 * 2048 * 4096 * 32000,
     }
 
 
@@ -87,7 +89,7 @@ def flops_per_config():
 def gemm_kernel_flops():
     f = flops_per_config()
     return {"C2": f["C2"], "C3": f["C3"], "C4": f["C4"], "X1": 2.0 * 16384 * 4096 * (4 * 4096), "X2": f["X2"],
-            "X3": f["X3"]}
+            "X3": f["X3"], "X4": f["X4"]}
 
 
 def load_peaks():
@@ -217,7 +219,7 @@ def oracle_sample_text():
 
 
 ALL = ("C1", "C2", "C3", "C4", "C5")          # the step
-EXTRA = ("X1", "X2", "X3")                   # further workloads: with --only, or after the step when N == 1
+EXTRA = ("X1", "X2", "X3", "X4")             # further workloads: with --only, or after the step when N == 1
 
 
 def max_over_ranks(ms: float, world: int, device=None) -> float:
@@ -256,7 +258,7 @@ def make_inputs(only=ALL):
     import pike_inputs as G
     gen = {"C1": G.config1, "C2": G.config2, "C3": G.config3, "C4": G.config4, "C5": G.config5,
            "X1": lambda: G.attention_block(B=8, S=2048, E=4096), "X2": G.grouped_linear,
-           "X3": G.config4}
+           "X3": G.config4, "X4": G.config4}
     return {k: gen[k]() for k in only}
 
 
@@ -307,7 +309,7 @@ class Suite:
             return torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).to(dtype).pin_memory()
 
         c1, c2, c3, c4, c5 = (inputs.get(k) for k in ALL)
-        x1, x2, x3 = (inputs.get(k) for k in EXTRA)
+        x1, x2, x3, x4 = (inputs.get(k) for k in EXTRA)
         host_act, wts = {}, {}   # activations are copied host -> device every e2e step; weights stay resident in HBM
         if c1:
             host_act.update(c1x=pin(c1["x"], F32))
@@ -336,16 +338,22 @@ class Suite:
             x3_cols = P.vocab_shard_range(32000, rank, world)
             host_act.update(x3x=pin(x3["x"], BF16))
             wts.update(x3w=pin(x3["w"][:, x3_cols[0]:x3_cols[1]], BF16))
+        if x4:
+            host_act.update(x4x=pin(x4["x"], BF16))
+            wts.update(x4w=pin(x4["w"], BF16))
         self.host_act = host_act
         self.d = d = {k: v.to(device) for k, v in host_act.items()}
         d.update({k: v.to(device) for k, v in wts.items()})
         shapes = {"C1": ((128, 256), F32), "C2": ((4096, 4096), BF16), "C3": ((8192, 4096), BF16),
                   "C4": ((2048, 32000), F32), "C5": ((8, 32, 2048, 128), BF16), "X1": ((8, 2048, 4096), BF16),
-                  "X2": ((16384, 4096), BF16), "X3": ((2048, x3_cols[1] - x3_cols[0]), F32)}
+                  "X2": ((16384, 4096), BF16), "X3": ((2048, x3_cols[1] - x3_cols[0]), F32), "X4": ((2048, 32000), F32)}
         self.out = out = {k: torch.empty(shapes[k][0], dtype=shapes[k][1], device=device) for k in self.only}
         self.host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in out.items()}
         ws0 = torch.empty(256, dtype=torch.uint8, device=device)
-        ws3 = ws4 = wsx = wsx3 = ws0
+        ws3 = ws4 = wsx = wsx3 = wsx4 = ws0
+        if x4:
+            wsx4 = torch.empty(P.pike_linear_epilogue_workspace(d["x4x"], d["x4w"], reduce="softmax", out_dtype=F32,
+                                                                one_pass=True), dtype=torch.uint8, device=device)
         if x3:
             wsx3 = torch.empty(P.pike_linear_softmax_shard_workspace(d["x3x"], d["x3w"]), dtype=torch.uint8, device=device)
         if x1:
@@ -377,6 +385,8 @@ class Suite:
                                                          out=out["X2"]),
             # the exchange between the two library calls is an all-gather of 16 KiB per rank over the default group
             "X3": lambda: P.linear_softmax_vocab_sharded(d["x3x"], d["x3w"], out=out["X3"], workspace=wsx3),
+            "X4": lambda: P.pike_linear_epilogue(d["x4x"], d["x4w"], reduce="softmax", out_dtype=F32, one_pass=True,
+                                                 out=out["X4"], workspace=wsx4),
         }
         self.chains = {n: chains[n] for n in chains if n in self.only}
         self.names = list(self.chains)
@@ -646,8 +656,8 @@ def run_ours(args):
                          "so every chain starts with its inputs evicted",
                    "warm_ms": "per_config.warm_ms = the same chain 20 times back to back without per-kernel events "
                               "(short bursts run at higher clocks; for C1 it is the host's call rate)",
-                   "extras": "per_config X1..X3 are further workloads timed after the step (10 runs each, tensors "
-                             "larger than L2), not part of value",
+                   "extras": "per_config X1..X4 are further workloads timed after the step (10 runs each, tensors "
+                             "larger than L2), not part of value; X4 = C4 as one kernel (PIKE_FLAG_ONE_PASS)",
                    "weights": "resident in HBM", "flops": "GEMM multiply-adds x2; attention counts the causal half"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
@@ -667,7 +677,7 @@ def run_ours(args):
 
 
 def extra_workload(P, torch, device, name, with_eager, iters=10):
-    """One of X1..X3 on its own: 3 warm-up runs, then `iters` runs timed one by one with CUDA events."""
+    """One of X1..X4 on its own: 3 warm-up runs, then `iters` runs timed one by one with CUDA events."""
     s = Suite(P, torch, device, (name,))
     fl = flops_per_config()[name]
     for _ in range(3):
@@ -796,6 +806,7 @@ def eager_ops(torch, d, scale):
         "X1": x1_eager,
         "X2": x2_eager,
         "X3": lambda: torch.softmax(d["x3x"] @ d["x3w_full"], dim=-1, dtype=torch.float32),
+        "X4": lambda: torch.softmax(d["x4x"] @ d["x4w"], dim=-1, dtype=torch.float32),
     }
 
 
@@ -909,13 +920,13 @@ def parse_args(argv=None):
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--only", type=lambda v: tuple(x for x in ALL + EXTRA if x in v.split(",")), default=ALL,
-                    help="comma-separated subset of C1..C5 and X1..X3 (profiling runs; the default is the whole suite C1..C5)")
+                    help="comma-separated subset of C1..C5 and X1..X4 (profiling runs; the default is the whole suite C1..C5)")
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--sustained-seconds", type=float, default=2.0,
                     help="length of the sustained loop reported beside the K timed steps (0 = skip)")
     ap.add_argument("--no-eager", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the scaled_dot_product_attention / torch.compile rows")
-    ap.add_argument("--no-extras", action="store_true", help="skip the further workloads X1..X3")
+    ap.add_argument("--no-extras", action="store_true", help="skip the further workloads X1..X4")
     ap.add_argument("--no-parity", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args(argv)

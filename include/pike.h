@@ -74,6 +74,8 @@ typedef enum { PIKE_REDUCE_NONE = 0, PIKE_REDUCE_LAYERNORM = 1, PIKE_REDUCE_SOFT
 
 #define PIKE_FLAG_W_IS_NK 0x1u /* weight tensors are [N,K] ("out,in") instead of [K,N]   */
 #define PIKE_FLAG_CAUSAL  0x2u /* attention: key j takes part for query i only if j <= i */
+#define PIKE_FLAG_ONE_PASS 0x4u /* pike_linear_epilogue, 16-bit path, reduce == SOFTMAX: one kernel, every      */
+                               /* probability written exactly once (see pike_linear_epilogue)                 */
 
 /* Epilogue descriptor: what follows the GEMM inside the same kernel. */
 typedef struct {
@@ -123,6 +125,13 @@ pike_status_t pike_set_wait_limit_ns(pike_handle_t handle, uint64_t ns);
  * the handle stay usable.  Use with a small pike_set_wait_limit_ns. */
 pike_status_t pike_test_withhold_loads(pike_handle_t handle);
 
+/* Test hook for the cross-CTA wait of the one-pass softmax (PIKE_FLAG_ONE_PASS; no counterpart in the paper): in the
+ * NEXT such launch through this handle one CTA never counts itself in on the stripe counters, so its peers' waits run
+ * out after the wait limit, the kernel records where, runs to its end (the output is garbage) and
+ * pike_get_last_device_status reports PIKE_ERR_TIMEOUT.  Nothing faults, traps or hangs.  Use with a small
+ * pike_set_wait_limit_ns. */
+pike_status_t pike_test_withhold_partials(pike_handle_t handle);
+
 /*
  * Per-kernel device timing, following the paper's timing protocol (Section 4.6:
  * timed runs bracketed on the device, synchronisation inside the timed region).
@@ -164,6 +173,15 @@ pike_status_t pike_profile_end(pike_handle_t handle, pike_kernel_profile_t *out)
  *   deviations) for LAYERNORM - and a second kernel combines the pairs and
  *   finishes the rows in place.  SOFTMAX needs out F32; LAYERNORM takes 16-bit or F32
  *   (with a 16-bit out the un-reduced values are rounded once before normalisation).
+ *   With PIKE_FLAG_ONE_PASS a SOFTMAX on this path runs as ONE kernel that never writes an un-normalised value
+ *   (Section 5.3: "eliminating intermediate memory writes"): a 256-row stripe of logits stays in tensor memory
+ *   across all CTA pairs of the device until its per-tile (max, sum exp) pairs have been exchanged through the
+ *   workspace, then every probability is written once.  The kernel's CTAs wait for one another, so it is
+ *   launched cooperatively (it needs the whole device; the wait is bounded like every other and reports
+ *   PIKE_ERR_TIMEOUT through the status word).  Needs ceil(N/256) <= 2 x (CTA pairs the device holds), i.e.
+ *   N <= 37888 on a 148-SM part, else PIKE_ERR_UNSUPPORTED; the workspace also holds one counter per stripe.
+ *   On the benchmark's logits chain it is SLOWER than the two-kernel form (measured; see profiles/), which is
+ *   why it is an option and not the default.
  * out must not alias any input (PIKE_ERR_UNSUPPORTED if the ranges overlap).
  *
  * Workspace: pike_linear_epilogue_workspace returns the bytes needed (0 unless a

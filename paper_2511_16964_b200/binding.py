@@ -20,11 +20,11 @@ _LIB_PATH = os.path.join(_HERE, "libpike.so")
 PIKE_F32, PIKE_BF16, PIKE_F16 = 0, 1, 2
 ACT = {"none": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 REDUCE = {"none": 0, "layernorm": 1, "softmax": 2}
-FLAG_W_IS_NK, FLAG_CAUSAL = 0x1, 0x2
+FLAG_W_IS_NK, FLAG_CAUSAL, FLAG_ONE_PASS = 0x1, 0x2, 0x4
 
 EXPORTS = (
     "pike_create", "pike_destroy", "pike_status_string", "pike_get_last_device_status",
-    "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
+    "pike_set_wait_limit_ns", "pike_test_withhold_loads", "pike_test_withhold_partials", "pike_profile_begin", "pike_profile_end", "pike_linear_epilogue_workspace", "pike_linear_epilogue",
     "pike_mlp_block_workspace", "pike_mlp_block", "pike_attention_chain_workspace",
     "pike_attention_chain", "pike_linear_softmax_noalloc", "pike_attention_block_workspace", "pike_attention_block",
     "pike_grouped_linear_epilogue", "pike_linear_softmax_shard_workspace", "pike_linear_softmax_shard_local",
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
             lib.pike_get_last_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_uint32)]
             lib.pike_set_wait_limit_ns.argtypes = [vp, ctypes.c_uint64]
             lib.pike_test_withhold_loads.argtypes = [vp]
+            lib.pike_test_withhold_partials.argtypes = [vp]
             lib.pike_profile_begin.argtypes = [vp]
             lib.pike_profile_end.argtypes = [vp, ctypes.POINTER(pike_kernel_profile_t)]
             lib.pike_linear_epilogue_workspace.argtypes = [vp, T, T, E, ctypes.POINTER(sz)]
@@ -199,6 +200,12 @@ def pike_test_withhold_loads(device=None) -> None:
     _check(load_library().pike_test_withhold_loads(_handle(dev)), "pike_test_withhold_loads")
 
 
+def pike_test_withhold_partials(device=None) -> None:
+    """Test hook: in the next one-pass softmax one CTA never counts itself in, so the stripe waits run out."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    _check(load_library().pike_test_withhold_partials(_handle(dev)), "pike_test_withhold_partials")
+
+
 def pike_get_last_device_status(device=None) -> tuple[int, int]:
     """(status, where) of the device status word.  Does not wait for anybody's kernels: synchronise the
     streams whose status is wanted first (torch.cuda.synchronize() or stream.synchronize())."""
@@ -223,9 +230,9 @@ def pike_profile_end(device=None) -> dict:
 
 
 def pike_linear_epilogue_workspace(x, w, *, act="none", scale=1.0, reduce="none", eps=1e-5,
-                                   out_dtype=None, w_is_nk=False) -> int:
+                                   out_dtype=None, w_is_nk=False, one_pass=False) -> int:
     out_dtype = x.dtype if out_dtype is None else out_dtype
-    e = _epilogue(act, scale, reduce, eps, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
+    e = _epilogue(act, scale, reduce, eps, out_dtype, (FLAG_W_IS_NK if w_is_nk else 0) | (FLAG_ONE_PASS if one_pass else 0))
     n = ctypes.c_size_t(0)
     _check(load_library().pike_linear_epilogue_workspace(_handle(x.device), _tensor(x), _tensor(w),
                                                          ctypes.byref(e), ctypes.byref(n)),
@@ -234,18 +241,18 @@ def pike_linear_epilogue_workspace(x, w, *, act="none", scale=1.0, reduce="none"
 
 
 def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, *, act="none", scale=1.0,
-                         reduce="none", eps=1e-5, out_dtype=None, w_is_nk=False, out=None, workspace=None,
-                         stream=None):
-    """out = reduce(scale*act(x @ w + bias) + residual); see include/pike.h."""
+                         reduce="none", eps=1e-5, out_dtype=None, w_is_nk=False, one_pass=False, out=None,
+                         workspace=None, stream=None):
+    """out = reduce(scale*act(x @ w + bias) + residual); one_pass selects PIKE_FLAG_ONE_PASS; see include/pike.h."""
     out_dtype = (out.dtype if out is not None else x.dtype) if out_dtype is None else out_dtype
     N = w.shape[0] if w_is_nk else w.shape[1]
     if out is None:
         with _on(stream):
             out = torch.empty((x.shape[0], N), dtype=out_dtype, device=x.device)
-    e = _epilogue(act, scale, reduce, eps, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
+    e = _epilogue(act, scale, reduce, eps, out_dtype, (FLAG_W_IS_NK if w_is_nk else 0) | (FLAG_ONE_PASS if one_pass else 0))
     ws, ws_ptr, ws_bytes = _workspace(
-        lambda: pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps,
-                                               out_dtype=out_dtype, w_is_nk=w_is_nk), x.device, workspace, stream)
+        lambda: pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps, out_dtype=out_dtype,
+                                               w_is_nk=w_is_nk, one_pass=one_pass), x.device, workspace, stream)
     _check(load_library().pike_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
                                                _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
                                                _tensor(out), ws_ptr, ws_bytes, _stream(stream)),

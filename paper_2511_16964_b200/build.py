@@ -16,6 +16,7 @@ SOURCES = [
     "api/pike_noalloc.cu",
     "kernels/fp32_chain.cu",
     "kernels/gemm_bf16.cu",
+    "kernels/gemm_softmax_onepass.cu",
     "kernels/row_kernels.cu",
     "kernels/attention_bf16.cu",
 ]

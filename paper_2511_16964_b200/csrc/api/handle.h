@@ -30,6 +30,7 @@ struct pike_handle_s {
     unsigned int *status;  // device, 4 words
     unsigned long long limit_ns;
     bool withhold_next;    // pike_test_withhold_loads: applies to the next bf16 GEMM launch only
+    bool withhold_partials_next;   // pike_test_withhold_partials: applies to the next one-pass softmax launch only
     PFN_cuTensorMapEncodeTiled_v12000 encode;
     cudaStream_t aux_stream;      // non-blocking; carries the status-word reads so that they wait for nobody's kernels
     // launch limits, filled by pike_create with the handle's device current
@@ -157,6 +158,12 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
                        int64_t K, int64_t N, const pike_tensor_t *bias, const void *res_ptr, bool res_f32, int64_t ldr,
                        void *out_ptr, bool out_f32, int64_t ldo, int act, float scale, float2 *partials,
                        cudaStream_t stream, int partials_mode = 1, const int *group_offsets = nullptr, int num_groups = 0);
+// The one-pass logits + softmax kernel (PIKE_FLAG_ONE_PASS); `workspace` holds the pairs, then the stripe counters.
+size_t onepass_workspace_bytes(int64_t M, int64_t N);
+pike_status_t run_gemm_softmax_onepass(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w, bool w_is_nk,
+                                       int64_t M, int64_t K, int64_t N, const pike_tensor_t *bias,
+                                       const pike_tensor_t *residual, pike_tensor_t *out, int act, float scale,
+                                       void *workspace, cudaStream_t stream);
 pike_status_t run_softmax_finish(pike_handle_t h, pike_tensor_t *out, const float2 *partials, int64_t M, int64_t N,
                                  cudaStream_t stream);
 

@@ -76,6 +76,54 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     return pike::launch_gemm_bf16(tmA, tmB, g, h->gemm_max_clusters, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
+size_t onepass_workspace_bytes(int64_t M, int64_t N)
+{
+    const int64_t num_n = (N + pike::GEMM_BN - 1) / pike::GEMM_BN, stripes = (M + 2 * pike::GEMM_BM - 1) / (2 * pike::GEMM_BM);
+    return align256((size_t)M * (size_t)num_n * sizeof(float2)) + align256((size_t)stripes * sizeof(unsigned int));
+}
+
+pike_status_t run_gemm_softmax_onepass(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w, bool w_is_nk,
+                                       int64_t M, int64_t K, int64_t N, const pike_tensor_t *bias,
+                                       const pike_tensor_t *residual, pike_tensor_t *out, int act, float scale,
+                                       void *workspace, cudaStream_t stream)
+{
+    CUtensorMap tmA, tmB;
+    if (pike_status_t st = make_map_2d(h, &tmA, w->dtype, x->data, (uint64_t)M, (uint64_t)K, (uint64_t)x->stride[0],
+                                       pike::GEMM_BK, pike::GEMM_BM))
+        return st;
+    if (pike_status_t st = w_is_nk ? make_map_w(h, &tmB, w->dtype, w->data, 1, (uint64_t)N, (uint64_t)K, (uint64_t)w->stride[0],
+                                                0, pike::GEMM_BK, pike::GEMM_BN / 2)
+                                   : make_map_w(h, &tmB, w->dtype, w->data, 1, (uint64_t)K, (uint64_t)N, (uint64_t)w->stride[0],
+                                                0, 64, pike::GEMM_BK))
+        return st;
+    const int64_t num_n = (N + pike::GEMM_BN - 1) / pike::GEMM_BN, stripes = (M + 2 * pike::GEMM_BM - 1) / (2 * pike::GEMM_BM);
+    pike::GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = (int)M; g.N = (int)N; g.K = (int)K;
+    g.w_is_nk = w_is_nk ? 1 : 0;
+    g.f16 = w->dtype == PIKE_F16 ? 1 : 0;
+    g.bias = bias ? bias->data : nullptr;
+    g.bias_f32 = bias && bias->dtype == PIKE_F32;
+    g.residual = residual ? residual->data : nullptr;
+    g.residual_f32 = residual && residual->dtype == PIKE_F32;
+    g.ldr = residual ? residual->stride[0] : 0;
+    g.out = out->data; g.out_f32 = 1; g.ldo = out->stride[0];
+    g.act = act; g.scale = scale;
+    g.row_partials = 1;
+    g.partials = static_cast<float2 *>(workspace);
+    g.stripe_counters = reinterpret_cast<unsigned int *>(static_cast<uint8_t *>(workspace) +
+                                                         align256((size_t)M * (size_t)num_n * sizeof(float2)));
+    g.status = h->status;
+    g.limit_ns = h->limit_ns;
+    g.test_withhold_loads = h->withhold_next ? 1 : 0;
+    g.test_withhold_partials = h->withhold_partials_next ? 1 : 0;
+    h->withhold_next = h->withhold_partials_next = false;
+    // the counters start at zero for every launch (a memset node on the caller's stream, no allocation)
+    if (cudaMemsetAsync(g.stripe_counters, 0, (size_t)stripes * sizeof(unsigned int), stream) != cudaSuccess) return PIKE_ERR_CUDA;
+    TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
+    return pike::launch_gemm_softmax_onepass(tmA, tmB, g, h->gemm_max_clusters, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+}
+
 // Second half of the split-row softmax: combine the per-tile pairs, normalise `out` in place.
 pike_status_t run_softmax_finish(pike_handle_t h, pike_tensor_t *out, const float2 *partials, int64_t M, int64_t N,
                                  cudaStream_t stream)
@@ -123,6 +171,7 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     h->limit_ns = DEFAULT_LIMIT_NS;
     h->profiling = false;
     h->withhold_next = false;
+    h->withhold_partials_next = false;
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -138,6 +187,7 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     // per-device kernel set-up, once, here: shared-memory limits of every kernel on this device and the launch
     // limits the launchers need, so that no launch pays for an attribute call or reads a process-wide variable
     if (pike::setup_fp32_chain() != cudaSuccess || pike::setup_gemm_bf16(h->num_sms, &h->gemm_max_clusters) != cudaSuccess ||
+        pike::setup_gemm_softmax_onepass() != cudaSuccess ||
         pike::setup_row_kernels() != cudaSuccess || pike::setup_attention_bf16(&h->attention_regs_ok) != cudaSuccess ||
         cudaStreamCreateWithFlags(&h->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
         cudaMalloc(&h->status, 4 * sizeof(unsigned int)) != cudaSuccess ||
@@ -232,12 +282,26 @@ pike_status_t pike_test_withhold_loads(pike_handle_t h)
     return PIKE_OK;
 }
 
+pike_status_t pike_test_withhold_partials(pike_handle_t h)
+{
+    if (h == nullptr) return PIKE_ERR_NULL;
+    h->withhold_partials_next = true;
+    return PIKE_OK;
+}
+
 pike_status_t pike_linear_epilogue_workspace(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
                                              const pike_epilogue_t *epi, size_t *bytes)
 {
     if (h == nullptr || bytes == nullptr) return PIKE_ERR_NULL;
     LinearShape s;
     if (pike_status_t st = linear_shape(x, w, epi, s)) return st;
+    const bool one_pass = (epi->flags & PIKE_FLAG_ONE_PASS) != 0;
+    if (one_pass) {
+        if (s.fp32_path || epi->reduce != PIKE_REDUCE_SOFTMAX) return PIKE_ERR_UNSUPPORTED;
+        if (!pike::gemm_softmax_onepass_fits((int)s.N, h->gemm_max_clusters)) return PIKE_ERR_UNSUPPORTED;
+        *bytes = onepass_workspace_bytes(s.M, s.N);
+        return PIKE_OK;
+    }
     *bytes = (!s.fp32_path && epi->reduce != PIKE_REDUCE_NONE) ? softmax_partials_bytes(s) : 0;
     return PIKE_OK;
 }
@@ -290,6 +354,15 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
 
     for (const pike_tensor_t *t : {bias, residual, gamma, beta})
         if (!side_ok(t, x->dtype)) return PIKE_ERR_DTYPE;
+    if (epi->flags & PIKE_FLAG_ONE_PASS) {
+        // the softmax in one kernel: a stripe's logits stay in tensor memory until its statistics are known
+        if (epi->reduce != PIKE_REDUCE_SOFTMAX) return PIKE_ERR_UNSUPPORTED;
+        if (!pike::gemm_softmax_onepass_fits((int)s.N, h->gemm_max_clusters)) return PIKE_ERR_UNSUPPORTED;
+        const pike_tensor_t *all[5] = {x, w, bias, residual, out};
+        if (pike_status_t st = check_workspace(workspace, workspace_bytes, onepass_workspace_bytes(s.M, s.N), all, 5)) return st;
+        return run_gemm_softmax_onepass(h, x, w, s.w_is_nk, s.M, s.K, s.N, bias, residual, out, (int)epi->act, epi->scale,
+                                        workspace, stream);
+    }
     // a row reduction on this path is split across the GEMM's column tiles: per-(row, tile) pairs go to the
     // workspace, a second kernel combines them and finishes the rows in place
     float2 *partials = nullptr;

@@ -93,6 +93,36 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
     return true;
 }
 
+// Wait until a counter in global memory that other CTAs increment has reached `target` (acquire at device scope).
+// Bounded like mbar_wait: after ctx.limit_ns, or when another thread of the CTA gave up, it records where it
+// stopped, raises the CTA's abort word and returns false.  Only for kernels whose CTAs are all resident.
+__device__ __forceinline__ bool counter_wait(const unsigned int *counter, unsigned int target, const WaitCtx &ctx,
+                                             uint32_t barrier_id)
+{
+    uint32_t spins = 0;
+    unsigned long long t0 = 0;
+    for (;;) {
+        unsigned int seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+        if (seen >= target) return true;
+        if ((++spins & 0xF) == 0) {
+            if (*ctx.abort) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > ctx.limit_ns) {
+                *ctx.abort = 1;
+                if (ctx.status != nullptr) {
+                    if (atomicCAS(ctx.status, 0u, (ctx.kernel_id << 16) | barrier_id) == 0u)
+                        ctx.status[1] = blockIdx.x;
+                }
+                return false;
+            }
+        }
+        __nanosleep(100);
+    }
+}
+
 // Give copies that may still be in flight time to land before the CTA exits on
 // the abort path (about one millisecond, bounded).
 __device__ __forceinline__ void abort_drain()

@@ -4,53 +4,18 @@
 //   out[m,n] = scale * act( sum_k A[m,k] * W[k,n] + bias[n] ) + residual[m,n]
 //
 // Persistent clusters of two CTAs (cta_group::2), one cluster per SM pair, each cluster
-// walking over 256 x 256 output tiles.  Per CTA (192 threads):
-//   warp 0      TMA producer: this CTA's 128 rows of A and its 128 of the tile's 256 W
-//               columns, 64 k at a time, into a 6-stage 128-byte-swizzled ring (32 KiB per
-//               stage).  Both CTAs' loads complete on the LEADER's "full" barrier.
-//   warp 1      allocates 512 tensor-memory columns (two 128x256 fp32 accumulator stages
-//               per CTA); in the leader CTA one thread issues tcgen05.mma.cta_group::2
-//               (256x256x16) for the pair and commits to mbarriers in both CTAs
-//   warps 2..5  epilogue: tcgen05.ld this CTA's accumulator rows (thread = row, 32
-//               columns at a time), bias/activation/scale/residual in registers, 16-byte
-//               stores; optionally per-row partials - (max, sum exp) or (mean, sum of squared
-//               deviations) - for a softmax / LayerNorm split across N tiles.  Runs under the
-//               next tile's K loop.
+// walking over 256 x 256 output tiles; warp roles and the shared building blocks are in
+// gemm_tile.cuh.  The epilogue warps apply bias/activation/scale/residual in registers and
+// store; optionally they emit per-row partials - (max, sum exp) or (mean, sum of squared
+// deviations) - for a softmax / LayerNorm split across N tiles.  The epilogue of one tile runs
+// under the next tile's K loop (two accumulator stages).
 // The pair halves the W traffic each SM's shared memory sees compared with a 128x256
-// single-CTA tile, which was shared-memory-bandwidth bound.  No TMA multicast is used.
-// Every mbarrier wait is bounded (see mbar_wait).
-#include "../device/act.cuh"
-#include "../device/ptx.cuh"
-#include "kernels.h"
+// single-CTA tile, which was shared-memory-bandwidth bound.
+#include "gemm_tile.cuh"
 
 namespace pike {
+using namespace gemm;
 namespace {
-
-constexpr int BM = GEMM_BM;                     // rows per CTA (the pair covers 2*BM)
-constexpr int BN = GEMM_BN, BK = GEMM_BK;
-constexpr int BN_HALF = BN / 2;                 // W columns staged by each CTA
-constexpr int STAGES = 6;
-constexpr int A_BYTES = BM * BK * 2;            // 16 KiB
-constexpr int B_BYTES = BN_HALF * BK * 2;       // 16 KiB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // 32 KiB per CTA
-constexpr int NUM_ACC = 2;
-constexpr int TMEM_COLS = NUM_ACC * BN;         // 512
-constexpr int THREADS = 192;
-constexpr int EPI_THREADS = 128;
-constexpr int EPI_WARPS = 4;
-
-struct __align__(8) Ctrl {
-    uint64_t full[STAGES];        // used in the leader: both CTAs' TMA bytes land here
-    uint64_t empty[STAGES];       // in each CTA: stage consumed (multicast commit)
-    uint64_t tmem_full[NUM_ACC];  // in each CTA: accumulator ready (multicast commit)
-    uint64_t tmem_empty[NUM_ACC]; // used in the leader: 4 epilogue warps x 2 CTAs drained it
-    uint32_t tmem_base;
-    uint32_t abort;
-    float bias[BN];
-};
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + sizeof(Ctrl);
-
-enum : uint32_t { BAR_EMPTY = 1, BAR_FULL = 2, BAR_TMEM_EMPTY = 3, BAR_TMEM_FULL = 4 };
 
 // Rasterisation: tiles are walked in groups of `group` blocks of one dimension (the PANEL dimension), all blocks
 // of the other dimension before the next group, panel block fastest.  The clusters that run together therefore
@@ -144,61 +109,23 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int num_kb = (p.K + BK - 1) / BK;
     const WorkPlan plan = work_plan(num_tiles, num_clusters, p.row_partials == 0);
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&ctrl->full[s], 1); mbar_init(&ctrl->empty[s], 1); }
-        for (int a = 0; a < NUM_ACC; ++a) { mbar_init(&ctrl->tmem_full[a], 1); mbar_init(&ctrl->tmem_empty[a], 2 * EPI_WARPS); }
-        ctrl->abort = 0;
-        fence_barrier_init();
-        tma_prefetch_desc(&tmA);
-        tma_prefetch_desc(&tmB);
-    }
-    if (warp == 1) {
-        tmem_alloc_pair(&ctrl->tmem_base, TMEM_COLS);
-        tmem_relinquish_pair();
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();          // the peer's barriers are initialised before anything signals them
-    tc_fence_after();
-    const uint32_t tmem_base = ctrl->tmem_base;
+    const uint32_t tmem_base = pair_setup(ctrl, &tmA, &tmB, warp);
     const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
 
     if (warp == 0) {
         // -------------------- TMA producer (warp-uniform loop, one elected lane issues)
-        {
-            const bool leader = elect_one();
-            int s = 0;
-            uint32_t ph = 0;
-            for (int w = cluster_id; w < plan.items && !p.test_withhold_loads; w += num_clusters) {
-                const Work wk = work_item(plan, w);
-                int m_blk, n_blk;
-                tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
-                const RowTile rt = row_tile(p, m_blk);
-                if (rt.row0 >= rt.row_end) continue;        // empty row tile (grouped mode): every role skips it
-                const int row0 = rt.row0 + (int)rank * BM;
-                // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
-                // (the bytes a stage waits for stay the same) and only their first 64 columns are used
-                const int col0 = n_blk * BN + wk.col_off + (int)rank * (wk.ncols / 2);
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    mbar_wait(&ctrl->empty[s], ph ^ 1, ctx, BAR_EMPTY);
-                    uint8_t *a_s = tiles + (size_t)s * STAGE_BYTES;
-                    uint8_t *b_s = a_s + A_BYTES;
-                    const uint32_t full_leader = mapa_shared(smem_u32(&ctrl->full[s]), 0);
-                    if (leader) {
-                        if (rank == 0) mbar_arrive_expect_tx(&ctrl->full[s], 2 * STAGE_BYTES);
-                        tma_load_2d_pair(a_s, &tmA, full_leader, kb * BK, row0);
-                        if (p.w_is_nk) {
-                            tma_load_3d_pair(b_s, &tmB, full_leader, kb * BK, col0, rt.group);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < BN_HALF / 64; ++i)
-                                tma_load_3d_pair(b_s + i * (64 * BK * 2), &tmB, full_leader, col0 + i * 64, kb * BK, rt.group);
-                        }
-                    }
-                    __syncwarp();
-                    if (++s == STAGES) { s = 0; ph ^= 1; }
-                }
-            }
+        const bool leader = elect_one();
+        RingPos rp{0, 0};
+        for (int w = cluster_id; w < plan.items && !p.test_withhold_loads; w += num_clusters) {
+            const Work wk = work_item(plan, w);
+            int m_blk, n_blk;
+            tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
+            const RowTile rt = row_tile(p, m_blk);
+            if (rt.row0 >= rt.row_end) continue;        // empty row tile (grouped mode): every role skips it
+            // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
+            // (the bytes a stage waits for stay the same) and only their first 64 columns are used
+            produce_tile(tiles, ctrl, &tmA, &tmB, rp, num_kb, rt.row0 + (int)rank * BM,
+                         n_blk * BN + wk.col_off + (int)rank * (wk.ncols / 2), rt.group, p.w_is_nk != 0, rank, leader, ctx);
         }
     } else if (warp == 1) {
         // ---------- MMA issuer (leader CTA only; warp-uniform loop, one elected lane issues)
@@ -206,13 +133,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool leader = elect_one();
             const uint32_t idesc_full = make_idesc_bf16(2 * BM, BN, false, !p.w_is_nk, p.f16 != 0);
             const uint32_t idesc_half = make_idesc_bf16(2 * BM, BN / 2, false, !p.w_is_nk, p.f16 != 0);
-            const uint32_t a_addr0 = smem_u32(tiles), b_addr0 = a_addr0 + A_BYTES;
-            const uint64_t adesc0 = make_smem_desc_sw128(a_addr0, 0, 1024);
-            const uint64_t bdesc0 = p.w_is_nk ? make_smem_desc_sw128(b_addr0, 0, 1024)
-                                              : make_smem_desc_sw128(b_addr0, 64 * BK * 2, 1024);
-            const uint32_t b_kstep = p.w_is_nk ? 32u : 2048u;     // bytes per 16-k step inside a stage
-            int s = 0;
-            uint32_t ph = 0;
+            const MmaDescs md = make_mma_descs(tiles, p.w_is_nk != 0);
+            RingPos rp{0, 0};
             int it = 0;
             for (int w = cluster_id; w < plan.items; w += num_clusters) {
                 const Work wk = work_item(plan, w);
@@ -222,30 +144,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const RowTile rt = row_tile(p, m_blk);
                     if (rt.row0 >= rt.row_end) continue;
                 }
-                const uint32_t idesc = wk.ncols == BN ? idesc_full : idesc_half;
                 const int acc = it & 1;
                 const uint32_t aph = (it >> 1) & 1;
                 mbar_wait_cluster(&ctrl->tmem_empty[acc], aph ^ 1, ctx, BAR_TMEM_EMPTY);
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    mbar_wait_cluster(&ctrl->full[s], ph, ctx, BAR_FULL);
-                    tc_fence_after();
-                    // stage 0's descriptors were built once; a stage is a constant number of bytes further
-                    const uint64_t adesc = desc_advance(adesc0, (uint32_t)s * STAGE_BYTES);
-                    const uint64_t bdesc = desc_advance(bdesc0, (uint32_t)s * STAGE_BYTES);
-                    if (leader) {
-#pragma unroll
-                        for (int k = 0; k < BK / 16; ++k)
-                            umma_ss_pair(d_tmem, desc_advance(adesc, k * 32), desc_advance(bdesc, k * b_kstep), idesc,
-                                         (kb | k) != 0 ? 1u : 0u);
-                        umma_commit_pair(&ctrl->empty[s], 0x3);
-                    }
-                    __syncwarp();
-                    if (++s == STAGES) { s = 0; ph ^= 1; }
-                }
-                if (leader) umma_commit_pair(&ctrl->tmem_full[acc], 0x3);
-                __syncwarp();
+                mma_tile(ctrl, md, rp, num_kb, tmem_base + acc * BN, wk.ncols == BN ? idesc_full : idesc_half,
+                         &ctrl->tmem_full[acc], leader, ctx);
                 ++it;
             }
         }
@@ -266,19 +170,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int n0 = n_blk * BN + wk.col_off;      // first output column of this item
             const int row = rt.row0 + (int)rank * BM + q * 32 + lane;
             const bool row_ok = row < rt.row_end;
-            const long long bias0 = (long long)rt.group * p.N + n0;    // bias is [num_groups, N] in grouped mode
 
-            // stage the tile's bias as fp32
-            named_bar_sync(1, EPI_THREADS);
-            for (int i = et; i < BN; i += EPI_THREADS) {
-                float b = 0.0f;
-                if (p.bias != nullptr && n0 + i < p.N)
-                    b = p.bias_f32 ? static_cast<const float *>(p.bias)[bias0 + i]
-                                   : h16_at(p.bias, bias0 + i, p.f16 != 0);
-                ctrl->bias[i] = b;
-            }
-            named_bar_sync(1, EPI_THREADS);
-
+            stage_bias(p, ctrl, n0, rt.group, et);
             mbar_wait(&ctrl->tmem_full[acc], aph, ctx, BAR_TMEM_FULL);
             tc_fence_after();
 
@@ -288,59 +181,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int c = 0; c < wk.ncols / 32; ++c) {
                 const int nc = n0 + c * 32;
                 if (nc >= p.N) break;
-                uint32_t r[32];
-                tmem_ld32(tmem_base + acc * BN + c * 32 + (static_cast<uint32_t>(q * 32) << 16), r);
-
-                // residual prefetch (thread = row, 32 consecutive columns)
-                uint4 res16[4];
-                float4 res32[8];
-                const bool has_res = p.residual != nullptr && row_ok;
-                if (has_res) {
-                    if (p.residual_f32) {
-                        const float *rp = static_cast<const float *>(p.residual) + (long long)row * p.ldr + nc;
-#pragma unroll
-                        for (int g = 0; g < 8; ++g)
-                            res32[g] = (nc + g * 4 < p.N) ? *reinterpret_cast<const float4 *>(rp + g * 4)
-                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
-                    } else {
-                        const uint16_t *rp = static_cast<const uint16_t *>(p.residual) + (long long)row * p.ldr + nc;
-                        if (nc + 32 <= p.N && (reinterpret_cast<uintptr_t>(rp) & 31) == 0) {
-                            // whole, 32-byte aligned chunk: two 32-byte loads (thread = row: one sector per row each)
-                            ld_global_32B(rp, reinterpret_cast<uint32_t *>(&res16[0]));
-                            ld_global_32B(rp + 16, reinterpret_cast<uint32_t *>(&res16[2]));
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g)
-                                res16[g] = (nc + g * 8 < p.N) ? *reinterpret_cast<const uint4 *>(rp + g * 8)
-                                                              : make_uint4(0u, 0u, 0u, 0u);
-                        }
-                    }
-                }
-                tmem_ld_wait();
-
                 float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    v[j] = p.scale * act_fast<ACT>(__uint_as_float(r[j]) + ctrl->bias[c * 32 + j]);
-                if (has_res) {
-                    if (p.residual_f32) {
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            v[g * 4 + 0] += res32[g].x; v[g * 4 + 1] += res32[g].y;
-                            v[g * 4 + 2] += res32[g].z; v[g * 4 + 3] += res32[g].w;
-                        }
-                    } else {
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            const uint32_t w4[4] = {res16[g].x, res16[g].y, res16[g].z, res16[g].w};
-#pragma unroll
-                            for (int h = 0; h < 4; ++h) {
-                                v[g * 8 + 2 * h] += h16_lo(w4[h], f16);
-                                v[g * 8 + 2 * h + 1] += h16_hi(w4[h], f16);
-                            }
-                        }
-                    }
-                }
+                chunk_values<ACT>(p, ctrl, tmem_base + acc * BN + c * 32 + (static_cast<uint32_t>(q * 32) << 16), row,
+                                  row_ok, nc, c, f16, v);
 
                 if (p.row_partials == 2) {
                     // LayerNorm partials: this chunk's (count, mean, sum of squared deviations), merged into
@@ -360,74 +203,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     run_m += delta * ((float)cnt / n_new);             // run_m: running mean
                     run_l += cm2 + delta * delta * (n_old * (float)cnt / n_new);   // run_l: running M2
                 } else if (p.row_partials) {
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (nc + j < p.N) cm = fmaxf(cm, v[j]);
-                    const float nm = fmaxf(run_m, cm);
-                    float s = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (nc + j < p.N) s += __expf(v[j] - nm);
-                    run_l = run_l * __expf(run_m - nm) + s;
-                    run_m = nm;
+                    softmax_fold(v, nc, p.N, run_m, run_l);
                 }
-
-                // Thread = row, so one store instruction of a warp touches 32 different rows: where the chunk
-                // lies fully inside N and starts on a 32-byte boundary it is written with 32-byte stores (whole
-                // sectors, half as many instructions), else with 16-byte ones.
-                if (row_ok) {
-                    const bool whole = nc + 32 <= p.N;
-                    if (p.out_f32) {
-                        float *op = static_cast<float *>(p.out) + (long long)row * p.ldo + nc;
-                        if (whole && (reinterpret_cast<uintptr_t>(op) & 31) == 0) {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g)
-                                st_global_32B(op + g * 8, reinterpret_cast<const uint32_t *>(&v[g * 8]));
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < 8; ++g)
-                                if (nc + g * 4 < p.N)
-                                    *reinterpret_cast<float4 *>(op + g * 4) =
-                                        make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
-                        }
-                    } else {
-                        uint16_t *op = static_cast<uint16_t *>(p.out) + (long long)row * p.ldo + nc;
-                        uint32_t w[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) w[i] = pack_h16x2(v[2 * i], v[2 * i + 1], f16);
-                        if (whole && (reinterpret_cast<uintptr_t>(op) & 31) == 0) {
-                            st_global_32B(op, &w[0]);
-                            st_global_32B(op + 16, &w[8]);
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g)
-                                if (nc + g * 8 < p.N)
-                                    *reinterpret_cast<uint4 *>(op + g * 8) =
-                                        make_uint4(w[g * 4], w[g * 4 + 1], w[g * 4 + 2], w[g * 4 + 3]);
-                        }
-                    }
-                }
+                if (row_ok) store_chunk(p, row, nc, f16, v);
             }
             // accumulator drained: one arrival per epilogue warp on the LEADER's barrier
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_shared(smem_u32(&ctrl->tmem_empty[acc]), 0));
+            release_accumulator(ctrl, acc, lane);
 
             if (p.row_partials && row_ok) p.partials[(long long)row * num_n + n_blk] = make_float2(run_m, run_l);
             ++it;
         }
     }
 
-    // ------------------------------------------------------------------ teardown
-    tc_fence_before();
-    __syncthreads();
-    if (ctrl->abort) abort_drain();
-    cluster_sync_all();          // neither CTA frees tensor memory while the pair may still use it
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc_pair(tmem_base, TMEM_COLS);
-    }
+    pair_teardown(ctrl, tmem_base, warp);
 }
 
 }  // namespace

@@ -55,6 +55,9 @@ struct GemmArgs {
     int group_m;              // blocks per rasterisation group (row blocks, or column blocks if group_along_n)
     int group_along_n;        // 0: groups of row blocks, W streams; 1: groups of column blocks, A streams
     int test_withhold_loads;  // test hook: the producers issue no loads, so the first "full" wait runs out
+    // one-pass logits + softmax kernel only
+    unsigned int *stripe_counters;   // device, one per 256-row stripe, zero at launch
+    int test_withhold_partials;      // test hook: block 0 never counts itself in, so every stripe wait runs out
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
 // the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
@@ -62,6 +65,14 @@ struct GemmArgs {
 constexpr int GEMM_BM = 128, GEMM_BN = 256, GEMM_BK = 64;
 cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a, int max_clusters,
                              cudaStream_t stream);
+
+// One-pass logits + softmax (gemm_softmax_onepass.cu): a.partials holds M * ceil(N/256) pairs, a.stripe_counters
+// ceil(M/256) zeroed words; out is fp32.  Needs ceil(N/256) <= 2 * max_clusters (a stripe's tiles fit the chip's
+// tensor memory); launched cooperatively with exactly max_clusters CTA pairs.
+cudaError_t setup_gemm_softmax_onepass();
+bool gemm_softmax_onepass_fits(int N, int max_clusters);
+cudaError_t launch_gemm_softmax_onepass(const CUtensorMap &tmA, const CUtensorMap &tmB, const GemmArgs &a,
+                                        int max_clusters, cudaStream_t stream);
 
 // ---- row kernels -------------------------------------------------------------------
 // z = LayerNorm(x) rows, 16-bit in/out (f16 != 0: IEEE half, else bf16), fp32 statistics; gamma/beta of
