@@ -284,7 +284,8 @@ pike_status_t pike_linear_softmax_noalloc(pike_handle_t handle, const pike_tenso
  * [0, group_offsets[G]) are not written.  The host cannot check the offsets, so the kernel clamps each
  * one to [0, T] and each group's end to at least its start: offsets that break the contract give
  * meaningless values in the rows concerned, never an access outside the tensors.  The group that owns
- * a row tile is found by bisection (about log2 G loads per tile), so G up to 65536 costs nothing extra.
+ * a row tile is found by bisection over prefix sums each CTA builds once in shared memory (up to 4096
+ * groups; beyond that over the offsets themselves), so G up to 65536 costs no scan per tile.
  */
 pike_status_t pike_grouped_linear_epilogue(pike_handle_t handle, const pike_tensor_t *x, const pike_tensor_t *w,
                                            const pike_tensor_t *bias, const pike_tensor_t *residual,

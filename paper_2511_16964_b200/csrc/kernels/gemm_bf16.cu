@@ -58,38 +58,72 @@ __device__ __forceinline__ Work work_item(const WorkPlan &wp, int w)
 }
 
 // Rows covered by the pair-row-tile with linear index m_lin.  Plain mode: 256 consecutive rows of A.
-// Grouped mode: group e (rows off[e] .. off[e+1]) owns the row-tile indices starting at
-//   T(e) = off[e] / 256 + e.
-// T grows by at least ceil(len_e / 256) from one group to the next, so the groups' index ranges never
-// overlap, the owner of an index is found by bisection over the offsets (O(log G) loads per tile, no
-// scratch memory, no pass over all groups) and off[G] / 256 + G indices cover everything.  An index whose
-// tile would start at or past its group's end is EMPTY: row0 == row_end, and every warp role skips the
-// item.  A tile's rows stop at the end of its group; `group` selects the weight matrix and bias row.
+// Grouped mode: row tiles are counted group by group - group e (rows off[e] .. off[e+1]) has
+// ceil(len_e / 256) of them - a tile's rows stop at the end of its group, and `group` selects the weight matrix
+// and bias row.  The exclusive prefix sums first[e] of the tile counts are built once per CTA in shared memory
+// (build_group_table) and the owner of an index is found by bisection over them: O(log G) shared-memory reads per
+// tile, and no index is wasted, so the tiles of one group and column block stay neighbours in the round-robin deal
+// (they share a slab of W through L2).  With more groups than the table holds the owner is found by bisection
+// over the offsets themselves, with group e owning the indices from off[e]/256 + e - ranges that never overlap
+// but leave some indices EMPTY (row0 == row_end): every warp role skips such an item.
 // Offsets come from device memory the host cannot check, so each one is clamped to [0, M] (and an end
 // to at least its start): whatever a router wrote there, no row outside the tensors is touched.
+constexpr int MAX_TABLE_GROUPS = 4096;
+constexpr size_t SMEM_BYTES_GEMM = SMEM_BYTES + (MAX_TABLE_GROUPS + 1) * sizeof(int);
+
 struct RowTile { int row0, row_end, group; };
 __device__ __forceinline__ int clamp_offset(const int *offsets, int i, int lo, int hi)
 {
     return min(max(__ldg(offsets + i), lo), hi);
 }
-__device__ __forceinline__ RowTile row_tile(const GemmArgs &p, int m_lin)
+__device__ __forceinline__ int group_tiles(const GemmArgs &p, int e)
+{
+    const int first = clamp_offset(p.group_offsets, e, 0, p.M);
+    return (clamp_offset(p.group_offsets, e + 1, first, p.M) - first + 2 * BM - 1) / (2 * BM);
+}
+// first[0 .. G]: exclusive prefix sums of the groups' tile counts (all threads of the CTA call this; warp 0 scans)
+__device__ __forceinline__ void build_group_table(const GemmArgs &p, int *first)
+{
+    if (p.group_offsets == nullptr || p.num_groups > MAX_TABLE_GROUPS) return;
+    if (threadIdx.x < 32) {
+        int carry = 0;
+        for (int e0 = 0; e0 < p.num_groups; e0 += 32) {
+            const int e = e0 + (int)threadIdx.x;
+            const int n = e < p.num_groups ? group_tiles(p, e) : 0;
+            int incl = n;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if ((int)threadIdx.x >= o) incl += up;
+            }
+            if (e < p.num_groups) first[e] = carry + incl - n;
+            carry += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (threadIdx.x == 0) first[p.num_groups] = carry;
+    }
+    __syncthreads();
+}
+__device__ __forceinline__ RowTile row_tile(const GemmArgs &p, const int *first_tile, int m_lin)
 {
     if (p.group_offsets == nullptr) return RowTile{m_lin * 2 * BM, p.M, 0};
-    int lo = 0, hi = p.num_groups - 1;      // the owner is the last group with T(e) <= m_lin
+    const bool table = p.num_groups <= MAX_TABLE_GROUPS;
+    int lo = 0, hi = p.num_groups - 1;      // the owner is the last group whose first index is <= m_lin
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
-        if (clamp_offset(p.group_offsets, mid, 0, p.M) / (2 * BM) + mid <= m_lin) lo = mid; else hi = mid - 1;
+        const int t_mid = table ? first_tile[mid] : clamp_offset(p.group_offsets, mid, 0, p.M) / (2 * BM) + mid;
+        if (t_mid <= m_lin) lo = mid; else hi = mid - 1;
     }
     const int first = clamp_offset(p.group_offsets, lo, 0, p.M);
     const int end = clamp_offset(p.group_offsets, lo + 1, first, p.M);
-    const long long local = (long long)m_lin - (first / (2 * BM) + lo);
+    const long long local = (long long)m_lin - (table ? first_tile[lo] : first / (2 * BM) + lo);
     const long long row0 = first + local * (2 * BM);
     if (local < 0 || row0 >= end) return RowTile{p.M, p.M, 0};
     return RowTile{(int)row0, end, lo};
 }
-__device__ __forceinline__ int count_row_tiles(const GemmArgs &p)
+__device__ __forceinline__ int count_row_tiles(const GemmArgs &p, const int *first_tile)
 {
     if (p.group_offsets == nullptr) return (p.M + 2 * BM - 1) / (2 * BM);
+    if (p.num_groups <= MAX_TABLE_GROUPS) return first_tile[p.num_groups];
     return clamp_offset(p.group_offsets, p.num_groups, 0, p.M) / (2 * BM) + p.num_groups;
 }
 
@@ -101,10 +135,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     Ctrl *ctrl = reinterpret_cast<Ctrl *>(tiles + (size_t)STAGES * STAGE_BYTES);
 
+    int *first_tile = reinterpret_cast<int *>(ctrl + 1);      // grouped mode: prefix sums of the groups' row tiles
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();           // 0 = leader
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
-    const int num_m = count_row_tiles(p), num_n = (p.N + BN - 1) / BN;
+    build_group_table(p, first_tile);
+    const int num_m = count_row_tiles(p, first_tile), num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
     const WorkPlan plan = work_plan(num_tiles, num_clusters, p.row_partials == 0);
@@ -120,7 +157,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const Work wk = work_item(plan, w);
             int m_blk, n_blk;
             tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
-            const RowTile rt = row_tile(p, m_blk);
+            const RowTile rt = row_tile(p, first_tile, m_blk);
             if (rt.row0 >= rt.row_end) continue;        // empty row tile (grouped mode): every role skips it
             // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
             // (the bytes a stage waits for stay the same) and only their first 64 columns are used
@@ -141,7 +178,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (p.group_offsets != nullptr) {
                     int m_blk, n_blk;
                     tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
-                    const RowTile rt = row_tile(p, m_blk);
+                    const RowTile rt = row_tile(p, first_tile, m_blk);
                     if (rt.row0 >= rt.row_end) continue;
                 }
                 const int acc = it & 1;
@@ -163,7 +200,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const Work wk = work_item(plan, w);
             int m_blk, n_blk;
             tile_coords(wk.tile, num_m, num_n, p.group_m, p.group_along_n, m_blk, n_blk);
-            const RowTile rt = row_tile(p, m_blk);
+            const RowTile rt = row_tile(p, first_tile, m_blk);
             if (rt.row0 >= rt.row_end) continue;
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
@@ -223,13 +260,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 template <typename Kern>
 static cudaError_t setup_one(Kern kern, int num_sms, int *max_clusters)
 {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES_GEMM);
     if (e != cudaSuccess) return e;
     // how many CTA pairs the device can hold at once (one CTA per SM at this shared-memory size)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * (num_sms / 2));
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM_BYTES_GEMM;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
@@ -258,6 +295,7 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
                              cudaStream_t stream)
 {
     // grouped mode: the device derives the row tiles from the offsets itself; this is the host's upper bound
+    // (every group can add one partly filled tile)
     const int num_m = a.group_offsets != nullptr ? a.M / (2 * BM) + a.num_groups : (a.M + 2 * BM - 1) / (2 * BM);
     const int num_n = (a.N + BN - 1) / BN;
     const long long num_tiles = (long long)num_m * num_n;
@@ -293,10 +331,10 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
     const int clusters = most < max_clusters ? (int)most : max_clusters;
     const dim3 grid(2 * clusters), block(THREADS);
     switch (a.act) {
-    case ACT_GELU_ERF:  gemm_bf16_kernel<ACT_GELU_ERF><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
-    case ACT_GELU_TANH: gemm_bf16_kernel<ACT_GELU_TANH><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
-    case ACT_SILU:      gemm_bf16_kernel<ACT_SILU><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
-    default:            gemm_bf16_kernel<ACT_NONE><<<grid, block, SMEM_BYTES, stream>>>(tmA, tmB, args); break;
+    case ACT_GELU_ERF:  gemm_bf16_kernel<ACT_GELU_ERF><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
+    case ACT_GELU_TANH: gemm_bf16_kernel<ACT_GELU_TANH><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
+    case ACT_SILU:      gemm_bf16_kernel<ACT_SILU><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
+    default:            gemm_bf16_kernel<ACT_NONE><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
     }
     return cudaGetLastError();
 }

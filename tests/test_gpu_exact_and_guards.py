@@ -114,6 +114,23 @@ def test_grouped_many_small_groups_are_exact():
     assert np.array_equal(host64(out.t), O.grouped_linear_epilogue(x, w, b, None, off))
 
 
+def test_grouped_more_groups_than_the_shared_memory_table_holds():
+    """5000 groups of 0..4 rows: past 4096 groups the kernel finds a row tile's group by bisection over the offsets
+    themselves (most row-tile indices are then empty and skipped)."""
+    import paper_2511_16964_b200 as P
+    rng = np.random.default_rng(18)
+    sizes = rng.integers(0, 5, 5000)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    T, K, N, Gn = int(off[-1]), 64, 64, len(sizes)
+    x, w, b = ints(rng, (T, K)), ints(rng, (Gn, K, N), -2, 2), ints(rng, (Gn, N), -8, 8)
+    out = Guarded((T, N), F32)
+    P.pike_grouped_linear_epilogue(dev(x, BF16), dev(w, BF16), dev(b, BF16), None, torch.from_numpy(off).cuda(),
+                                   out_dtype=F32, out=out.t)
+    _status_ok()
+    out.check("5000 groups")
+    assert np.array_equal(host64(out.t), O.grouped_linear_epilogue(x, w, b, None, off))
+
+
 @pytest.mark.parametrize("bad", ["past_the_end", "decreasing", "negative"])
 def test_grouped_offsets_that_break_the_contract_touch_nothing_outside(bad):
     """The kernel reads the offsets from device memory the host cannot check: whatever is there, stores stay inside
