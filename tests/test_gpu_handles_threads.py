@@ -71,3 +71,19 @@ def test_two_handles_on_two_threads():
             check_bf16(host64(o2), want2, what=f"thread {tid} GEMM")
             check_f32(host64(o1), want1, what=f"thread {tid} fp32 chain")
             check_bf16(host64(o5), want5, what=f"thread {tid} attention")
+
+
+def test_more_distinct_buffers_than_the_tensor_map_cache_holds():
+    """The handle keeps the 48 most recently used tensor maps; calls on 70 different activation buffers (and then on
+    the first ones again, whose maps have been evicted meanwhile) must all come out right."""
+    import paper_2511_16964_b200 as P
+    c = G.config2(M=130, K=64, N=264, seed=64)
+    w, b = dev(c["w"], BF16), dev(c["b"], BF16)
+    want = O.linear_epilogue(c["x"], c["w"], c["b"], act="gelu_tanh")
+    xs = [dev(c["x"], BF16).clone() for _ in range(70)]
+    outs = [P.pike_linear_epilogue(x, w, b, act="gelu_tanh") for x in xs]
+    outs += [P.pike_linear_epilogue(x, w, b, act="gelu_tanh") for x in xs[:5]]
+    torch.cuda.synchronize()
+    assert P.pike_get_last_device_status() == (0, 0)
+    for o in outs:
+        check_bf16(host64(o), want, what="tensor-map cache")
