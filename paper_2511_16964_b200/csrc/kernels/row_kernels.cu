@@ -92,14 +92,14 @@ layernorm_bf16_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *_
     }
 }
 
-// One WARP per row for rows of at most 4096 elements, in a persistent grid (one CTA per SM, ten warps).
+// One WARP per row for rows of at most 4096 elements, in a persistent grid (one CTA per SM, twelve warps).
 // Each warp streams its rows through a private two-stage ring in shared memory filled by bulk copies
 // (one elected lane issues them, an mbarrier per stage counts the bytes): while a row is being reduced and
 // normalised in registers, the next two are already in flight, so loads, arithmetic and stores of different
 // rows overlap inside every warp instead of all warps of an SM loading, computing and storing in phase.
 // The row sits in 16 x 16-byte registers per lane and both reductions are pure shuffles.  gamma and beta are
 // copied to shared memory once per CTA (every warp needs all of them for every row).
-constexpr int LNW_WARPS = 10;
+constexpr int LNW_WARPS = 12;
 constexpr int LNW_STAGES = 2;
 constexpr int LNW_MAX_CHUNKS = 16;  // D <= 32 * 16 * 8 = 4096
 constexpr int LNW_STAGE_BYTES = LNW_MAX_CHUNKS * 32 * 16;   // 8 KiB: one row of 4096 16-bit elements
@@ -196,32 +196,37 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
         }
     }
     // all arithmetic on fp32 pairs (one 16-bit word = two elements): the kernel moves 4 bytes per element and is
-    // otherwise bound by how many instructions per element the warp has to issue
-    uint64_t sum2[2] = {0ull, 0ull};
+    // otherwise bound by how many instructions per element the warp has to issue.  Mean and variance come from ONE
+    // pass over values shifted by the row's first element (sums of d and d^2 with d = v - v0; the shift removes the
+    // cancellation a plain sum of squares would suffer when the mean dwarfs the spread).
+    const float v0 = __shfl_sync(0xffffffffu, h16_lo(c[0].x, F16), 0);
+    const uint64_t neg_v0 = pack_f32x2(-v0, -v0);
+    uint64_t s1[2] = {0ull, 0ull}, s2[2] = {0ull, 0ull};
 #pragma unroll
     for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
-        const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
-#pragma unroll
-        for (int h = 0; h < 4; ++h) sum2[h & 1] = add_f32x2(sum2[h & 1], h16x2_to_f32x2(w[h], F16));   // padding chunks are zero
-    }
-    float s0, s1;
-    unpack_f32x2(add_f32x2(sum2[0], sum2[1]), s0, s1);
-    const float mean = warp_sum(s0 + s1) / (float)D;
-    const uint64_t neg_mean2 = pack_f32x2(-mean, -mean);
-    uint64_t ss2[2] = {0ull, 0ull};
-#pragma unroll
-    for (int i = 0; i < LNW_MAX_CHUNKS; ++i) {
-        if (lane + i * 32 < nchunks) {
+        if (lane + i * 32 < nchunks) {              // padding chunks hold no elements
             const uint32_t w[4] = {c[i].x, c[i].y, c[i].z, c[i].w};
 #pragma unroll
             for (int h = 0; h < 4; ++h) {
-                const uint64_t d2 = add_f32x2(h16x2_to_f32x2(w[h], F16), neg_mean2);
-                ss2[h & 1] = fma_f32x2(d2, d2, ss2[h & 1]);
+                const uint64_t d2 = add_f32x2(h16x2_to_f32x2(w[h], F16), neg_v0);
+                s1[h & 1] = add_f32x2(s1[h & 1], d2);
+                s2[h & 1] = fma_f32x2(d2, d2, s2[h & 1]);
             }
         }
     }
-    unpack_f32x2(add_f32x2(ss2[0], ss2[1]), s0, s1);
-    const float rstd = rsqrtf(warp_sum(s0 + s1) / (float)D + eps);
+    float a0, a1, b0, b1;
+    unpack_f32x2(add_f32x2(s1[0], s1[1]), a0, a1);
+    unpack_f32x2(add_f32x2(s2[0], s2[1]), b0, b1);
+    float sd = a0 + a1, sq = b0 + b1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {              // the two reductions interleaved
+        sd += __shfl_xor_sync(0xffffffffu, sd, o);
+        sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    }
+    const float inv_d = 1.0f / (float)D;
+    const float md = sd * inv_d;                    // mean of d
+    const float rstd = rsqrtf(fmaxf(sq * inv_d - md * md, 0.0f) + eps);
+    const float mean = v0 + md;
     const uint64_t rstd2 = pack_f32x2(rstd, rstd), shift2 = pack_f32x2(-mean * rstd, -mean * rstd);
     uint4 *zr = reinterpret_cast<uint4 *>(z + row * ldz);
 #pragma unroll
