@@ -100,7 +100,9 @@ typedef struct pike_handle_s *pike_handle_t;
  * cache of encoded TMA tensor maps keyed by (pointer, extents, pitches, box), so
  * repeated calls on the same buffers skip the encoding.  A handle is not
  * thread-safe; use one per host thread.  PIKE_ERR_ARCH if the device is not
- * compute capability 10.x. */
+ * compute capability 10.x.  With PIKE_LOG=1 in the environment when the handle is
+ * created, every kernel selection made through it is written to stderr as one line
+ * (kernel, shapes, layout, epilogue): host-side only, nothing changes on the device. */
 pike_status_t pike_create(pike_handle_t *handle, int device);
 pike_status_t pike_destroy(pike_handle_t handle);
 

@@ -7,6 +7,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cudaTypedefs.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <vector>
@@ -37,6 +39,7 @@ struct pike_handle_s {
     int gemm_max_clusters;        // CTA pairs of the GEMM kernel the device holds at once
     bool attention_regs_ok;       // the attention kernels were compiled with the registers their setmaxnreg split needs
     float2 *noalloc_partials;     // device address of the built-in scratch of pike_linear_softmax_noalloc (set on its first call)
+    bool log;                     // PIKE_LOG=1 in the environment at pike_create: one stderr line per kernel selection
     // encoded tensor maps, most recent use first (a model calls the same few GEMMs on the same buffers over and over)
     static constexpr size_t MAP_CACHE_SIZE = 48;
     struct CachedMap { TensorMapKey key; CUtensorMap map; };
@@ -49,6 +52,15 @@ struct pike_handle_s {
 };
 
 namespace pike_api {
+
+// Host-side kernel-selection log (PIKE_LOG=1): what was launched, on which shapes.  Never on unless asked for.
+#define PIKE_LOGF(h, ...)                                  \
+    do {                                                   \
+        if ((h)->log) {                                    \
+            fprintf(stderr, "[pike] " __VA_ARGS__);        \
+            fputc('\n', stderr);                           \
+        }                                                  \
+    } while (0)
 
 // Brackets one kernel launch with CUDA events on the caller's stream while profiling is on.
 struct TimedLaunch {

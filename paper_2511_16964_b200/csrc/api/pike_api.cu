@@ -72,6 +72,10 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     g.limit_ns = h->limit_ns;
     g.test_withhold_loads = h->withhold_next ? 1 : 0;
     h->withhold_next = false;
+    PIKE_LOGF(h, "gemm_bf16_kernel M=%lld K=%lld N=%lld %s w=%s act=%d out=%s%s%s partials=%d groups=%d clusters<=%d",
+              (long long)M, (long long)K, (long long)N, g.f16 ? "f16" : "bf16", w_is_nk ? "[N,K]" : "[K,N]", act,
+              out_f32 ? "f32" : "16-bit", bias ? " +bias" : "", res_ptr ? " +residual" : "", g.row_partials, num_groups,
+              h->gemm_max_clusters);
     TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
     return pike::launch_gemm_bf16(tmA, tmB, g, h->gemm_max_clusters, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
@@ -120,6 +124,8 @@ pike_status_t run_gemm_softmax_onepass(pike_handle_t h, const pike_tensor_t *x, 
     h->withhold_next = h->withhold_partials_next = false;
     // the counters start at zero for every launch (a memset node on the caller's stream, no allocation)
     if (cudaMemsetAsync(g.stripe_counters, 0, (size_t)stripes * sizeof(unsigned int), stream) != cudaSuccess) return PIKE_ERR_CUDA;
+    PIKE_LOGF(h, "gemm_softmax_onepass_kernel M=%lld K=%lld N=%lld stripes=%lld tiles_per_stripe=%lld clusters=%d (cooperative)",
+              (long long)M, (long long)K, (long long)N, (long long)stripes, (long long)num_n, h->gemm_max_clusters);
     TimedLaunch timed(h, PIKE_KERNEL_GEMM_BF16, stream);
     return pike::launch_gemm_softmax_onepass(tmA, tmB, g, h->gemm_max_clusters, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
@@ -129,6 +135,7 @@ pike_status_t run_softmax_finish(pike_handle_t h, pike_tensor_t *out, const floa
                                  cudaStream_t stream)
 {
     const int num_n = (int)((N + pike::GEMM_BN - 1) / pike::GEMM_BN);
+    PIKE_LOGF(h, "softmax_finish_kernel M=%lld N=%lld pairs_per_row=%d", (long long)M, (long long)N, num_n);
     TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
     return pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)M, (int)N,
                                        stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
@@ -172,6 +179,10 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     h->profiling = false;
     h->withhold_next = false;
     h->withhold_partials_next = false;
+    {
+        const char *env = getenv("PIKE_LOG");
+        h->log = env != nullptr && env[0] != '\0' && env[0] != '0';
+    }
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
@@ -348,6 +359,8 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         a.w_is_nk = s.w_is_nk;
         a.act = (int)epi->act; a.reduce = (int)epi->reduce;
         a.scale = epi->scale; a.eps = epi->eps;
+        PIKE_LOGF(h, "fp32_chain_kernel M=%d K=%d N=%d act=%d reduce=%d w=%s", a.M, a.K, a.N, a.act, a.reduce,
+                  a.w_is_nk ? "[N,K]" : "[K,N]");
         TimedLaunch timed(h, PIKE_KERNEL_FP32_CHAIN, stream);
         return pike::launch_fp32_chain(a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
@@ -652,6 +665,8 @@ static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, cons
     a.out_b = (long long)eff_stride(out, 0); a.out_h = (long long)eff_stride(out, 1); a.out_s = (long long)eff_stride(out, 2);
     a.status = h->status;
     a.limit_ns = h->limit_ns;
+    PIKE_LOGF(h, "attention_bf16_kernel B*H=%d S=%d Sk=%d D=%d %s%s scale=%g", a.BH, a.S, a.Sk, a.D, a.f16 ? "f16" : "bf16",
+              causal ? " causal" : "", (double)scale);
     TimedLaunch timed(h, PIKE_KERNEL_ATTENTION_BF16, stream);
     return pike::launch_attention_bf16(tmQ, tmK, tmV, a, h->num_sms, h->attention_regs_ok, stream) == cudaSuccess
                ? PIKE_OK : PIKE_ERR_CUDA;

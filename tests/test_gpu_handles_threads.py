@@ -87,3 +87,22 @@ def test_more_distinct_buffers_than_the_tensor_map_cache_holds():
     assert P.pike_get_last_device_status() == (0, 0)
     for o in outs:
         check_bf16(host64(o), want, what="tensor-map cache")
+
+
+def test_kernel_selection_log_goes_to_stderr_when_asked_for():
+    """PIKE_LOG=1 at handle creation: one stderr line per kernel selection; nothing without it."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import torch, paper_2511_16964_b200 as P\n"
+            "x = torch.zeros((64, 64), device='cuda', dtype=torch.bfloat16); w = torch.zeros((64, 256), device='cuda', dtype=torch.bfloat16)\n"
+            "P.pike_linear_epilogue(x, w, reduce='softmax', out_dtype=torch.float32); torch.cuda.synchronize()\n")
+    for flag, expect in (("1", True), ("0", False)):
+        res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, cwd=root,
+                             env=dict(os.environ, PIKE_LOG=flag), timeout=300)
+        assert res.returncode == 0, res.stderr[-1000:]
+        lines = [l for l in res.stderr.splitlines() if l.startswith("[pike] ")]
+        assert (len(lines) == 2) == expect, res.stderr[-1000:]
+        if expect:
+            assert "gemm_bf16_kernel M=64 K=64 N=256" in lines[0] and "softmax_finish_kernel" in lines[1]
