@@ -62,6 +62,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
+// The bookkeeping of a bounded wait, out of line: a wait is inlined at dozens of places and only its polling
+// loop has to be there; this part runs once per 32 failed polls.  It looks at the CTA's abort word, reads the clock
+// every 1024 polls (a slow system register) and, once limit_ns have passed since the first reading, records where
+// the wait stopped and raises the abort word.  Returns the (possibly updated) time of the first reading, or
+// WAIT_GAVE_UP when the caller must stop waiting.
+constexpr unsigned long long WAIT_GAVE_UP = ~0ull;
+static __device__ __noinline__ unsigned long long wait_bookkeeping(unsigned int *status, volatile uint32_t *abort,
+                                                            unsigned long long limit_ns, uint32_t status_word,
+                                                            uint32_t spins, unsigned long long t0)
+{
+    if (*abort) return WAIT_GAVE_UP;            // another thread of the CTA gave up
+    if ((spins & 0x3FF) != 0) return t0;
+    const unsigned long long now = globaltimer_ns();
+    if (t0 == 0) return now;
+    if (now - t0 <= limit_ns) return t0;
+    *abort = 1;
+    if (status != nullptr) {
+        if (atomicCAS(status, 0u, status_word) == 0u) status[1] = blockIdx.x;
+    }
+    return WAIT_GAVE_UP;
+}
+
 // Wait for the phase with the given parity to complete.  Never spins forever:
 // after ctx.limit_ns (or as soon as another thread of the CTA gave up) it records
 // where it stopped, raises the CTA's abort word and returns false.  Callers keep
@@ -69,25 +91,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 // releases tensor memory and returns; the host sees PIKE_ERR_TIMEOUT.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const WaitCtx &ctx, uint32_t barrier_id)
 {
-    // Fast path: poll.  The abort word is looked at every 32 failed polls and the clock (a slow system
-    // register) every 1024, so an ordinary hand-off never pays for them.
     if (mbar_try_wait(bar, parity)) return true;
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x1F) == 0 && *ctx.abort) return false;   // another thread of the CTA gave up
-        if ((spins & 0x3FF) == 0) {
-            const unsigned long long now = globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > ctx.limit_ns) {
-                *ctx.abort = 1;
-                if (ctx.status != nullptr) {
-                    if (atomicCAS(ctx.status, 0u, (ctx.kernel_id << 16) | barrier_id) == 0u)
-                        ctx.status[1] = blockIdx.x;
-                }
-                return false;
-            }
+        if ((++spins & 0x1F) == 0) {
+            t0 = wait_bookkeeping(ctx.status, ctx.abort, ctx.limit_ns, (ctx.kernel_id << 16) | barrier_id, spins, t0);
+            if (t0 == WAIT_GAVE_UP) return false;
         }
     }
     return true;
@@ -127,6 +137,7 @@ __device__ __forceinline__ bool counter_wait(const unsigned int *counter, unsign
 // the abort path (about one millisecond, bounded).
 __device__ __forceinline__ void abort_drain()
 {
+#pragma unroll 1
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
 }
 
@@ -401,19 +412,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
     uint32_t spins = 0;
     unsigned long long t0 = 0;
     while (!mbar_try_wait_cluster(bar, parity)) {
-        if ((++spins & 0x1F) == 0 && *ctx.abort) return false;   // another thread of the CTA gave up
-        if ((spins & 0x3FF) == 0) {
-            const unsigned long long now = globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > ctx.limit_ns) {
-                *ctx.abort = 1;
-                if (ctx.status != nullptr) {
-                    if (atomicCAS(ctx.status, 0u, (ctx.kernel_id << 16) | barrier_id) == 0u)
-                        ctx.status[1] = blockIdx.x;
-                }
-                return false;
-            }
+        if ((++spins & 0x1F) == 0) {
+            t0 = wait_bookkeeping(ctx.status, ctx.abort, ctx.limit_ns, (ctx.kernel_id << 16) | barrier_id, spins, t0);
+            if (t0 == WAIT_GAVE_UP) return false;
         }
     }
     return true;

@@ -332,24 +332,22 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                     const int nv_max = min(kv_left, p.causal ? warp_row0 - k0 + 32 : BKV);
 #pragma unroll
                     for (int cc = 0; cc < BKV / 32; ++cc) {
-                        if ((cc + 1) * 32 <= nv_min) {
+                        if (cc * 32 >= nv_max) {
+                            live &= ~(1u << cc);
+                        } else if ((cc + 1) * 32 > nv_min) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i)
-                                pm[i & 7] = fmaxf(pm[i & 7], __uint_as_float(s[cc * 32 + i]));
-                        } else if (cc * 32 >= nv_max) {
-                            live &= ~(1u << cc);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const float v = (cc * 32 + i < n_valid) ? __uint_as_float(s[cc * 32 + i]) : -INFINITY;
-                                s[cc * 32 + i] = __float_as_uint(v);
-                                pm[i & 7] = fmaxf(pm[i & 7], v);
-                            }
+                                if (cc * 32 + i >= n_valid) s[cc * 32 + i] = __float_as_uint(-INFINITY);
                         }
                     }
-                } else {
+                }
+                // (skipped chunks still hold scores: harmless in the maximum only if they are excluded)
 #pragma unroll
-                    for (int i = 0; i < BKV; ++i) pm[i & 7] = fmaxf(pm[i & 7], __uint_as_float(s[i]));
+                for (int cc = 0; cc < BKV / 32; ++cc) {
+                    if (live & (1u << cc)) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) pm[i & 7] = fmaxf(pm[i & 7], __uint_as_float(s[cc * 32 + i]));
+                    }
                 }
                 const float tmax = fmaxf(fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3])),
                                          fmaxf(fmaxf(pm[4], pm[5]), fmaxf(pm[6], pm[7])));
