@@ -102,7 +102,12 @@ typedef struct pike_handle_s *pike_handle_t;
  * thread-safe; use one per host thread.  PIKE_ERR_ARCH if the device is not
  * compute capability 10.x.  With PIKE_LOG=1 in the environment when the handle is
  * created, every kernel selection made through it is written to stderr as one line
- * (kernel, shapes, layout, epilogue): host-side only, nothing changes on the device. */
+ * (kernel, shapes, layout, epilogue): host-side only, nothing changes on the device.
+ * Kernels are launched with the programmatic-stream-serialisation attribute: a
+ * kernel's CTAs may be scheduled onto SMs the previous kernel of the stream has
+ * already left and run their prologue there; each waits for that kernel to complete
+ * before it touches a tensor, so stream order is kept.  PIKE_PDL=0 in the
+ * environment at creation takes the attribute off (results are identical). */
 pike_status_t pike_create(pike_handle_t *handle, int device);
 pike_status_t pike_destroy(pike_handle_t handle);
 

@@ -40,6 +40,7 @@ struct pike_handle_s {
     bool attention_regs_ok;       // the attention kernels were compiled with the registers their setmaxnreg split needs
     float2 *noalloc_partials;     // device address of the built-in scratch of pike_linear_softmax_noalloc (set on its first call)
     bool log;                     // PIKE_LOG=1 in the environment at pike_create: one stderr line per kernel selection
+    bool pdl;                     // launches carry the programmatic-stream-serialisation attribute (off with PIKE_PDL=0)
     // encoded tensor maps, most recent use first (a model calls the same few GEMMs on the same buffers over and over)
     static constexpr size_t MAP_CACHE_SIZE = 48;
     struct CachedMap { TensorMapKey key; CUtensorMap map; };

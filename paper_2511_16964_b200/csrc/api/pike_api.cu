@@ -56,6 +56,7 @@ pike_status_t run_gemm(pike_handle_t h, const void *a_ptr, int64_t lda, const pi
     }
     pike::GemmArgs g;
     memset(&g, 0, sizeof(g));
+    g.pdl = h->pdl ? 1 : 0;
     g.M = (int)M; g.N = (int)N; g.K = (int)K;
     g.w_is_nk = w_is_nk ? 1 : 0;
     g.f16 = w->dtype == PIKE_F16 ? 1 : 0;
@@ -138,7 +139,7 @@ pike_status_t run_softmax_finish(pike_handle_t h, pike_tensor_t *out, const floa
     PIKE_LOGF(h, "softmax_finish_kernel M=%lld N=%lld pairs_per_row=%d", (long long)M, (long long)N, num_n);
     TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
     return pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0], partials, num_n, (int)M, (int)N,
-                                       stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+                                       stream, 0, 1, h->pdl) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 }  // namespace pike_api
@@ -182,6 +183,8 @@ pike_status_t pike_create(pike_handle_t *handle, int device)
     {
         const char *env = getenv("PIKE_LOG");
         h->log = env != nullptr && env[0] != '\0' && env[0] != '0';
+        env = getenv("PIKE_PDL");
+        h->pdl = !(env != nullptr && env[0] == '0');
     }
     void *fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -347,6 +350,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
             if (t != nullptr && t->dtype != PIKE_F32) return PIKE_ERR_DTYPE;
         pike::Fp32ChainArgs a;
         memset(&a, 0, sizeof(a));
+        a.pdl = h->pdl ? 1 : 0;
         a.x = static_cast<const float *>(x->data);
         a.w = static_cast<const float *>(w->data);
         a.bias = bias ? static_cast<const float *>(bias->data) : nullptr;
@@ -398,7 +402,7 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
                                               pike::GEMM_BN, (int)s.M, (int)s.N, gamma ? gamma->data : nullptr,
                                               gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
                                               beta && beta->dtype == PIKE_F32, epi->eps, x->dtype == PIKE_F16,
-                                              stream) != cudaSuccess)
+                                              stream, h->pdl) != cudaSuccess)
                 return PIKE_ERR_CUDA;
         } else {
             return run_softmax_finish(h, out, partials, s.M, s.N, stream);
@@ -459,7 +463,7 @@ pike_status_t pike_linear_softmax_shard_local(pike_handle_t h, const pike_tensor
     const int num_n = (int)((s.N + pike::GEMM_BN - 1) / pike::GEMM_BN);
     TimedLaunch timed(h, PIKE_KERNEL_SOFTMAX_FINISH, stream);
     return pike::launch_softmax_row_stats(partials, num_n, reinterpret_cast<float2 *>(row_stats), (int)s.M,
-                                          stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+                                          stream, h->pdl) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 pike_status_t pike_linear_softmax_shard_finish(pike_handle_t h, pike_tensor_t *out, const float *all_stats,
@@ -481,7 +485,7 @@ pike_status_t pike_linear_softmax_shard_finish(pike_handle_t h, pike_tensor_t *o
     // pair of (row m, shard r) at all_stats[(r*M + m)*2]: row stride 1 pair, "tile" stride M pairs
     return pike::launch_softmax_finish(static_cast<float *>(out->data), out->stride[0],
                                        reinterpret_cast<const float2 *>(all_stats), (int)num_shards, (int)M,
-                                       (int)out->shape[1], stream, 1, M) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+                                       (int)out->shape[1], stream, 1, M, h->pdl) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
 }
 
 pike_status_t pike_grouped_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, const pike_tensor_t *w,
@@ -600,7 +604,8 @@ pike_status_t pike_mlp_block(pike_handle_t h, const pike_tensor_t *x, const pike
         if (pike::launch_layernorm_bf16(x->data, x->stride[0], z, D, gamma ? gamma->data : nullptr,
                                         gamma && gamma->dtype == PIKE_F32, beta ? beta->data : nullptr,
                                         beta && beta->dtype == PIKE_F32, epi->eps, (int)M, (int)D,
-                                        x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream) != cudaSuccess)
+                                        x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream,
+                                        h->pdl) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // h = act(z @ w1 + b1), rounded to the chain's 16-bit type
@@ -657,6 +662,7 @@ static pike_status_t run_attention(pike_handle_t h, const pike_tensor_t *q, cons
     if (pike_status_t st = make_map_bhsd(h, &tmV, q->dtype, v->data, B, H, Sk, D, eff_stride(v, 0), eff_stride(v, 1), eff_stride(v, 2))) return st;
     pike::AttnArgs a;
     memset(&a, 0, sizeof(a));
+    a.pdl = h->pdl ? 1 : 0;
     a.BH = (int)(B * H); a.H = (int)H; a.S = (int)S; a.Sk = (int)Sk; a.D = (int)D;
     a.scale = scale;
     a.causal = causal ? 1 : 0;
@@ -784,7 +790,8 @@ pike_status_t pike_attention_block(pike_handle_t h, const pike_tensor_t *x, cons
         TimedLaunch timed(h, PIKE_KERNEL_LAYERNORM_BF16, stream);
         if (pike::launch_layernorm_bf16(x->data, E, z, E, gamma ? gamma->data : nullptr, gamma && gamma->dtype == PIKE_F32,
                                         beta ? beta->data : nullptr, beta && beta->dtype == PIKE_F32, epi->eps, (int)M,
-                                        (int)E, x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream) != cudaSuccess)
+                                        (int)E, x->dtype == PIKE_F16, h->status, h->limit_ns, h->num_sms, stream,
+                                        h->pdl) != cudaSuccess)
             return PIKE_ERR_CUDA;
     }
     // qkv = z @ w_qkv + b_qkv, laid out [B, S, 3, H, 128]

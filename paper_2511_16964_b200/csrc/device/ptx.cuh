@@ -141,6 +141,17 @@ __device__ __forceinline__ void abort_drain()
     for (int i = 0; i < 1000; ++i) __nanosleep(1000);
 }
 
+// ------------------------------------------------ programmatic dependent launch ----
+// A grid launched with the programmatic-stream-serialisation attribute may be scheduled while the previous kernel
+// of its stream still runs: its CTAs take the SMs that kernel's CTAs have left.  pdl_wait() returns once that kernel
+// has completed and its writes are visible; every kernel executes it after a prologue that touches no global tensor
+// (barrier initialisation, tensor-memory allocation, descriptor prefetch) and before its first global access.  It
+// is a no-op in a launch without the attribute.  No kernel here signals its dependents early
+// (griddepcontrol.launch_dependents): with the signal at kernel start the next kernel's CTAs sat beside the GEMM's
+// for its whole run and the logits + softmax chain got 3 % slower; leaving it to each CTA's exit keeps the gain
+// (launch latency and prologue hidden in the previous kernel's tail) without that cost.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // --------------------------------------------------------------------- TMA ----
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map)
 {

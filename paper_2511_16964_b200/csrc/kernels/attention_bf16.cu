@@ -130,6 +130,7 @@ attention_bf16_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                 // nothing above touched a global tensor
     const uint32_t tmem_base = ctrl->tmem_base;
     const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_ATTN};
 
@@ -464,8 +465,8 @@ static cudaError_t launch_attention_d(const CUtensorMap &tmQ, const CUtensorMap 
     const int num_pairs = (num_q_tiles + 1) / 2;
     const long long num_items = (long long)((num_pairs + 1) / 2) * a.BH;   // slots: two items each
     const unsigned grid = (unsigned)(num_items < num_sms ? num_items : num_sms);   // persistent: one CTA per SM
-    attention_bf16_kernel<D, F16><<<dim3(grid), THREADS, SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
-    return cudaGetLastError();
+    return launch_kernel(attention_bf16_kernel<D, F16>, dim3(grid), dim3(THREADS), SMEM_BYTES, stream, a.pdl != 0, tmQ, tmK,
+                         tmV, a);
 }
 
 // shared-memory limit of one instantiation; regs_ok is cleared if it was compiled with fewer registers than

@@ -61,6 +61,7 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
     const long long row0 = (long long)((int)blockIdx.x / cn) * BM;
     const int n0 = rank * BN;
     const int n_loc = min(max(a.N - n0, 0), BN);      // columns this CTA owns (0 for a padding rank)
+    pdl_wait();
 
     float acc[RPT][CW][4];
 #pragma unroll
@@ -284,11 +285,13 @@ cudaError_t launch_one(const Fp32ChainArgs &a, int cn, cudaStream_t stream)
     cfg.blockDim = dim3(FT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = (unsigned)cn; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cn; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see launch_kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.pdl != 0 ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, fp32_chain_kernel<RPT, CW, NK>, a, kc);
 }
 

@@ -331,12 +331,11 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
     const int clusters = most < max_clusters ? (int)most : max_clusters;
     const dim3 grid(2 * clusters), block(THREADS);
     switch (a.act) {
-    case ACT_GELU_ERF:  gemm_bf16_kernel<ACT_GELU_ERF><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
-    case ACT_GELU_TANH: gemm_bf16_kernel<ACT_GELU_TANH><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
-    case ACT_SILU:      gemm_bf16_kernel<ACT_SILU><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
-    default:            gemm_bf16_kernel<ACT_NONE><<<grid, block, SMEM_BYTES_GEMM, stream>>>(tmA, tmB, args); break;
+    case ACT_GELU_ERF:  return launch_kernel(gemm_bf16_kernel<ACT_GELU_ERF>, grid, block, SMEM_BYTES_GEMM, stream, a.pdl != 0, tmA, tmB, args);
+    case ACT_GELU_TANH: return launch_kernel(gemm_bf16_kernel<ACT_GELU_TANH>, grid, block, SMEM_BYTES_GEMM, stream, a.pdl != 0, tmA, tmB, args);
+    case ACT_SILU:      return launch_kernel(gemm_bf16_kernel<ACT_SILU>, grid, block, SMEM_BYTES_GEMM, stream, a.pdl != 0, tmA, tmB, args);
+    default:            return launch_kernel(gemm_bf16_kernel<ACT_NONE>, grid, block, SMEM_BYTES_GEMM, stream, a.pdl != 0, tmA, tmB, args);
     }
-    return cudaGetLastError();
 }
 
 }  // namespace pike

@@ -65,6 +65,7 @@ __device__ __forceinline__ uint32_t pair_setup(Ctrl *ctrl, const CUtensorMap *tm
     __syncthreads();
     cluster_sync_all();          // the peer's barriers are initialised before anything signals them
     tc_fence_after();
+    pdl_wait();                  // everything above touched no global tensor; from here on the previous kernel's output is read
     return ctrl->tmem_base;
 }
 

@@ -4,7 +4,31 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace pike {
+
+// One kernel launch on `stream`.  With `pdl` the launch carries the programmatic-stream-serialisation attribute:
+// the grid may be scheduled while the previous kernel in the stream is still running (its CTAs take the SMs that
+// kernel's CTAs have left), which hides the launch latency and the prologue between the kernels of a chain and
+// between calls.  Every kernel of this library executes griddepcontrol.wait before its first access to a global
+// tensor, so the attribute is safe behind any predecessor.
+template <typename... P, typename... A>
+inline cudaError_t launch_kernel(void (*kern)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                                 A &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<A>(args)...);
+}
 
 enum : uint32_t {
     KID_GEMM = 1,
@@ -21,6 +45,7 @@ struct Fp32ChainArgs {
     int w_is_nk;
     int act, reduce;
     float scale, eps;
+    int pdl;        // launch with programmatic stream serialisation (see launch_kernel)
 };
 cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, int num_sms, cudaStream_t stream);
 
@@ -58,6 +83,7 @@ struct GemmArgs {
     // one-pass logits + softmax kernel only
     unsigned int *stripe_counters;   // device, one per 256-row stripe, zero at launch
     int test_withhold_partials;      // test hook: block 0 never counts itself in, so every stripe wait runs out
+    int pdl;                         // launch with programmatic stream serialisation (see launch_kernel); not for the one-pass kernel
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
 // the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
@@ -80,20 +106,23 @@ cudaError_t launch_gemm_softmax_onepass(const CUtensorMap &tmA, const CUtensorMa
 // (status / limit_ns: the device status word and the bound of the kernel's waits for its row copies)
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream);
+                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream,
+                                  bool pdl = false);
 // p[m,:] = exp(v[m,:] - m_row) / l_row in place, (m_row, l_row) combined from the partials
 // Pair t of row m sits at partials[m*pair_row_stride + t*pair_tile_stride] (pair_row_stride 0 = num_n_tiles,
 // the layout the GEMM epilogue writes; {1, M} reads pairs stored [t][m], as an all-gather over GPUs lays them).
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
-                                  cudaStream_t stream, long long pair_row_stride = 0, long long pair_tile_stride = 1);
+                                  cudaStream_t stream, long long pair_row_stride = 0, long long pair_tile_stride = 1,
+                                  bool pdl = false);
 // stats[m] = the row's per-tile (max, sum exp) pairs [M, num_n_tiles] folded into one pair
-cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream);
+cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream,
+                                     bool pdl = false);
 
 // out = (v - mean)/sqrt(var + eps)*gamma + beta in place (v 16-bit or f32), statistics combined from the
 // per-(row, n-tile) (mean, sum of squared deviations) pairs; tile_n = columns per tile
 cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
                                     int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
-                                    int beta_f32, float eps, int f16, cudaStream_t stream);
+                                    int beta_f32, float eps, int f16, cudaStream_t stream, bool pdl = false);
 
 // ---- attention ---------------------------------------------------------------------
 struct AttnArgs {
@@ -106,6 +135,7 @@ struct AttnArgs {
     long long out_b, out_h, out_s;
     unsigned int *status;
     unsigned long long limit_ns;
+    int pdl;        // launch with programmatic stream serialisation (see launch_kernel)
 };
 cudaError_t launch_attention_bf16(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV,
                                   const AttnArgs &a, int num_sms, bool regs_ok, cudaStream_t stream);

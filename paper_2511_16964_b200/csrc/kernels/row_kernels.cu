@@ -41,6 +41,7 @@ layernorm_bf16_kernel(const uint16_t *__restrict__ x, long long ldx, uint16_t *_
     __shared__ float red[32];
     const int tid = threadIdx.x;
     const long long row = blockIdx.x;
+    pdl_wait();
     const uint4 *xr = reinterpret_cast<const uint4 *>(x + row * ldx);
     const int nchunks = D / 8;  // D % 8 == 0
 
@@ -106,13 +107,6 @@ constexpr int LNW_STAGE_BYTES = LNW_MAX_CHUNKS * 32 * 16;   // 8 KiB: one row of
 constexpr int LNW_PARAM_BYTES = LNW_MAX_CHUNKS * 32 * 8 * 4;   // 16 KiB: 4096 fp32 values (or 16-bit ones in half of it)
 constexpr size_t LNW_SMEM_BYTES = 128 + (size_t)LNW_WARPS * LNW_STAGES * LNW_STAGE_BYTES + 2 * LNW_PARAM_BYTES;
 
-__device__ __forceinline__ float warp_sum(float x)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-    return x;
-}
-
 // eight consecutive parameters starting at element e (e % 8 == 0) as fp32, from the CTA's copy in shared memory;
 // KIND 0 = absent, 1 = 16-bit (the type of x), 2 = f32
 template <int KIND, bool F16>
@@ -144,6 +138,7 @@ layernorm_bf16_warp_kernel(const uint16_t *__restrict__ x, long long ldx, uint16
     __shared__ uint64_t full[LNW_WARPS][LNW_STAGES];
     __shared__ uint32_t abort_word;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    pdl_wait();
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(lnw_smem) + 127) & ~uintptr_t(127));
     uint8_t *ring = base + (size_t)warp * LNW_STAGES * LNW_STAGE_BYTES;
     uint8_t *gamma_s = base + (size_t)LNW_WARPS * LNW_STAGES * LNW_STAGE_BYTES, *beta_s = gamma_s + LNW_PARAM_BYTES;
@@ -264,6 +259,7 @@ softmax_finish_kernel(float *__restrict__ v, long long ldv, const float2 *__rest
     __shared__ float red[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long row = blockIdx.x;
+    pdl_wait();
     // pair t of this row; [row][tile] for one GEMM's tiles, [shard][row] for pairs gathered from other GPUs
     const float2 *pr = partials + row * pair_row_stride;
 
@@ -313,6 +309,7 @@ softmax_row_stats_kernel(const float2 *__restrict__ partials, int num_n_tiles, f
 {
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * (STATS_THREADS / 32) + (threadIdx.x >> 5);
+    pdl_wait();
     if (row >= M) return;
     const float2 *pr = partials + row * num_n_tiles;
     float m = -INFINITY;
@@ -343,6 +340,7 @@ layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__
     const bool f16 = f16_flag != 0;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long row = blockIdx.x;
+    pdl_wait();
     const float2 *pr = partials + row * num_n_tiles;
     auto block_sum256 = [&](float x) {
 #pragma unroll
@@ -405,16 +403,12 @@ layernorm_finish_kernel(void *__restrict__ vout, long long ldv, const float2 *__
 
 cudaError_t launch_layernorm_finish(void *v, int out_f32, long long ldv, const float2 *partials, int num_n_tiles,
                                     int tile_n, int M, int N, const void *gamma, int gamma_f32, const void *beta,
-                                    int beta_f32, float eps, int f16, cudaStream_t stream)
+                                    int beta_f32, float eps, int f16, cudaStream_t stream, bool pdl)
 {
     if (M <= 0) return cudaSuccess;
-    if (out_f32)
-        layernorm_finish_kernel<true><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
-                                                                    gamma_f32, beta, beta_f32, eps, f16);
-    else
-        layernorm_finish_kernel<false><<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, tile_n, N, gamma,
-                                                                     gamma_f32, beta, beta_f32, eps, f16);
-    return cudaGetLastError();
+    auto kern = out_f32 ? layernorm_finish_kernel<true> : layernorm_finish_kernel<false>;
+    return launch_kernel(kern, dim3(M), dim3(SM_THREADS), 0, stream, pdl, v, ldv, partials, num_n_tiles, tile_n, N, gamma,
+                         gamma_f32, beta, beta_f32, eps, f16);
 }
 
 cudaError_t setup_row_kernels()
@@ -436,7 +430,8 @@ cudaError_t setup_row_kernels()
 
 cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long long ldz, const void *gamma,
                                   int gamma_f32, const void *beta, int beta_f32, float eps, int M, int D, int f16,
-                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream)
+                                  unsigned int *status, unsigned long long limit_ns, int num_sms, cudaStream_t stream,
+                                  bool pdl)
 {
     if (M <= 0) return cudaSuccess;
     if (D % 8 != 0 || D > LN_THREADS * LN_MAX_CHUNKS * 8) return cudaErrorInvalidValue;
@@ -451,36 +446,35 @@ cudaError_t launch_layernorm_bf16(const void *x, long long ldx, void *z, long lo
 #define PIKE_LN_CASE(G, B)                                                                                          \
     if (gk == G && bk == B) {                                                                                       \
         auto kern = f16 ? layernorm_bf16_warp_kernel<G, B, true> : layernorm_bf16_warp_kernel<G, B, false>;        \
-        kern<<<grid, block, LNW_SMEM_BYTES, stream>>>(xp, ldx, zp, ldz, gamma, beta, eps, M, D, status, limit_ns);  \
+        return launch_kernel(kern, grid, block, LNW_SMEM_BYTES, stream, pdl, xp, ldx, zp, ldz, gamma, beta, eps, M, D, \
+                             status, limit_ns);                                                                     \
     }
         PIKE_LN_CASE(0, 0) PIKE_LN_CASE(0, 1) PIKE_LN_CASE(0, 2) PIKE_LN_CASE(1, 0) PIKE_LN_CASE(1, 1)
         PIKE_LN_CASE(1, 2) PIKE_LN_CASE(2, 0) PIKE_LN_CASE(2, 1) PIKE_LN_CASE(2, 2)
 #undef PIKE_LN_CASE
-        return cudaGetLastError();
+        return cudaErrorInvalidValue;   // not reached: every (gk, bk) has a case
     }
-    layernorm_bf16_kernel<<<M, LN_THREADS, 0, stream>>>(static_cast<const uint16_t *>(x), ldx,
-                                                         static_cast<uint16_t *>(z), ldz, gamma, gamma_f32, beta,
-                                                         beta_f32, eps, D, f16);
-    return cudaGetLastError();
+    return launch_kernel(layernorm_bf16_kernel, dim3(M), dim3(LN_THREADS), 0, stream, pdl,
+                         static_cast<const uint16_t *>(x), ldx, static_cast<uint16_t *>(z), ldz, gamma, gamma_f32, beta,
+                         beta_f32, eps, D, f16);
 }
 
 cudaError_t launch_softmax_finish(float *v, long long ldv, const float2 *partials, int num_n_tiles, int M, int N,
-                                  cudaStream_t stream, long long pair_row_stride, long long pair_tile_stride)
+                                  cudaStream_t stream, long long pair_row_stride, long long pair_tile_stride, bool pdl)
 {
     if (M <= 0) return cudaSuccess;
     if (pair_row_stride == 0) pair_row_stride = num_n_tiles;
-    softmax_finish_kernel<<<M, SM_THREADS, 0, stream>>>(v, ldv, partials, num_n_tiles, pair_row_stride,
-                                                        pair_tile_stride, N);
-    return cudaGetLastError();
+    return launch_kernel(softmax_finish_kernel, dim3(M), dim3(SM_THREADS), 0, stream, pdl, v, ldv, partials, num_n_tiles,
+                         pair_row_stride, pair_tile_stride, N);
 }
 
-cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream)
+cudaError_t launch_softmax_row_stats(const float2 *partials, int num_n_tiles, float2 *stats, int M, cudaStream_t stream,
+                                     bool pdl)
 {
     if (M <= 0) return cudaSuccess;
     const int rows_per_block = STATS_THREADS / 32;
-    softmax_row_stats_kernel<<<(M + rows_per_block - 1) / rows_per_block, STATS_THREADS, 0, stream>>>(
-        partials, num_n_tiles, stats, M);
-    return cudaGetLastError();
+    return launch_kernel(softmax_row_stats_kernel, dim3((M + rows_per_block - 1) / rows_per_block), dim3(STATS_THREADS), 0,
+                         stream, pdl, partials, num_n_tiles, stats, M);
 }
 
 }  // namespace pike

@@ -106,3 +106,32 @@ def test_kernel_selection_log_goes_to_stderr_when_asked_for():
         assert (len(lines) == 2) == expect, res.stderr[-1000:]
         if expect:
             assert "gemm_bf16_kernel M=64 K=64 N=256" in lines[0] and "softmax_finish_kernel" in lines[1]
+
+
+def test_results_do_not_depend_on_programmatic_dependent_launch():
+    """PIKE_PDL=0 at handle creation takes the launch attribute off: the chains' results are bit-identical with it
+    on (the default) and off, over back-to-back calls that reuse one output and one workspace."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("import torch, hashlib, paper_2511_16964_b200 as P\n"
+            "g = torch.Generator(device='cuda').manual_seed(5)\n"
+            "r = lambda *s: (torch.randn(*s, device='cuda', generator=g) * 0.5).to(torch.bfloat16)\n"
+            "x, gm, bt, w1, b1, w2, b2 = r(640, 512), r(512), r(512), r(512, 1024) * 0.1, r(1024), r(1024, 512) * 0.1, r(512)\n"
+            "ws = torch.empty(P.pike_mlp_block_workspace(x, w1), dtype=torch.uint8, device='cuda'); out = torch.empty_like(x)\n"
+            "wl = r(512, 3000) * 0.1\n"
+            "h = hashlib.sha256()\n"
+            "for i in range(20):\n"
+            "    P.pike_mlp_block(x, gm, bt, w1, b1, w2, b2, out=out, workspace=ws)\n"
+            "    p = P.pike_linear_epilogue(out, wl, reduce='softmax', out_dtype=torch.float32)\n"
+            "    x = out.clone()\n"
+            "    h.update(p.cpu().numpy().tobytes()); h.update(out.view(torch.int16).cpu().numpy().tobytes())\n"
+            "print('DIGEST', h.hexdigest())\n")
+    digests = []
+    for flag in ("1", "0"):
+        res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, cwd=root,
+                             env=dict(os.environ, PIKE_PDL=flag), timeout=300)
+        assert res.returncode == 0, res.stderr[-1000:]
+        digests.append([l for l in res.stdout.splitlines() if l.startswith("DIGEST")][0])
+    assert digests[0] == digests[1]
