@@ -50,7 +50,7 @@ GEMM_ALGORITHMIC_BYTES_PER_STEP = 1.615e9
 # from the ncu captures summarised in profiles/gemm_bf16_kernel_dram_per_step.md: the value used, the spread
 # over repeated captures, and the SHA-256 (first 16 hex digits) of the kernel's sources at capture time.  The
 # line reports the traffic only while the sources still hash to that value.
-GEMM_DRAM_CAPTURE = {"bytes": 2.733e9, "min": 2.7023e9, "max": 2.7867e9, "captures": 3, "sources_sha16": "5b094d5806d56614"}
+GEMM_DRAM_CAPTURE = {"bytes": 2.690e9, "min": 2.6493e9, "max": 2.7112e9, "captures": 3, "sources_sha16": "6ad71bf36a446835"}
 GEMM_SOURCES = ("paper_2511_16964_b200/csrc/kernels/gemm_bf16.cu", "paper_2511_16964_b200/csrc/kernels/gemm_tile.cuh",
                 "paper_2511_16964_b200/csrc/device/ptx.cuh", "paper_2511_16964_b200/csrc/device/act.cuh",
                 "paper_2511_16964_b200/csrc/kernels/kernels.h")
@@ -836,6 +836,22 @@ def context_rows(torch, d, scale, names, budget_s=150.0):
                 flush)
         except Exception as exc:       # noqa: BLE001 - a context row must never break the benchmark
             rows["C5_sdpa_ms"], rows["C5_sdpa_error"] = None, repr(exc)[:200]
+    # What plain streaming kernels of the row kernels' sizes reach on this GPU, cold like them: a copy of C3's
+    # activations (as many bytes as its LayerNorm reads and writes), torch's own LayerNorm on them, and an in-place
+    # elementwise pass over an fp32 buffer of C4's logits' size (the bytes of the softmax finishing pass).
+    try:
+        if "C3" in names:
+            x = d["c3x"]
+            y = torch.empty_like(x)
+            rows["C3_layernorm_copy_same_bytes_ms"] = _timed_cold(torch, lambda: y.copy_(x), flush, iters=5)
+            rows["C3_layernorm_torch_ms"] = _timed_cold(
+                torch, lambda: F.layer_norm(x, (x.shape[1],), d["c3g"], d["c3be"], 1e-5), flush, iters=5)
+        if "C4" in names:
+            z = torch.empty((d["c4x"].shape[0], d["c4w"].shape[1]), dtype=torch.float32, device=device)
+            rows["C4_finish_inplace_same_bytes_ms"] = _timed_cold(torch, lambda: z.mul_(1.0009765625), flush, iters=5)
+            del z
+    except Exception as exc:           # noqa: BLE001
+        rows["streaming_rows_error"] = repr(exc)[:200]
     ops = eager_ops(torch, d, scale)
     for n in ("C2", "C3", "C5"):
         if n not in names:
@@ -849,7 +865,8 @@ def context_rows(torch, d, scale, names, budget_s=150.0):
         except Exception as exc:       # noqa: BLE001
             rows[f"{n}_compile_ms"], rows[f"{n}_compile_error"] = None, repr(exc)[:200]
     rows["seconds_spent"] = time.perf_counter() - t_start
-    rows["note"] = "C5_sdpa = torch scaled_dot_product_attention (is_causal); *_compile = torch.compile(default) of the eager composition"
+    rows["note"] = ("C5_sdpa = torch scaled_dot_product_attention (is_causal); *_compile = torch.compile(default) of the eager "
+                    "composition; *_same_bytes = a plain copy / in-place pass moving the bytes of that row kernel, cold")
     return rows
 
 
