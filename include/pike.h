@@ -24,6 +24,9 @@
  *    reports host-detectable errors only.  Device-detected conditions (a bounded
  *    wait inside a kernel that ran out) land in a status word that
  *    pike_get_last_device_status reads after the caller has synchronised.
+ *    A chain call only launches kernels (no allocation, no copy, no event unless
+ *    profiling is on), so a sequence of calls on a capturing stream becomes a CUDA
+ *    graph that can be replayed on new contents of the same buffers.
  *  - There is no CPU or library fallback: a device that is not compute
  *    capability 10.x yields PIKE_ERR_ARCH, an unsupported shape or combination
  *    PIKE_ERR_UNSUPPORTED.

@@ -110,3 +110,58 @@ def test_temporaries_belong_to_the_stream_the_kernels_run_on():
     check_bf16(host64(got3), O.mlp_block(c3["x"], c3["gamma"], c3["beta"], c3["w1"], c3["b1"], c3["w2"], c3["b2"],
                                          eps=c3["eps"]), what="mlp block with a temporary workspace on a side stream")
     del keep, junk
+
+
+def test_chains_replay_from_a_cuda_graph():
+    """With caller-owned outputs and workspaces a chain call allocates nothing and synchronises nothing, so a
+    sequence of calls can be captured into a CUDA graph once and replayed: every replay on new input CONTENTS (same
+    buffers) gives bit for bit what the same calls give when issued directly."""
+    import paper_2511_16964_b200 as P
+    c3 = G.config3(M=300, D=136, F=520, seed=41, affine=True)
+    c5 = G.config5(B=1, H=2, S=300, seed=42)
+    c1 = G.config1(M=40, K=64, N=72, seed=43)
+    x3, g3, be3, w1, b1, w2, b2 = (dev(c3[k], BF16) for k in ("x", "gamma", "beta", "w1", "b1", "w2", "b2"))
+    q, k, v = (dev(c5[n], BF16) for n in "qkv")
+    d1 = {n: dev(c1[n], F32) for n in ("x", "w", "b", "gamma", "beta")}
+    wl = dev(c3["w1"], BF16)                                            # logits weights for the softmax chain
+    out3, out5 = torch.empty_like(x3), torch.empty_like(q)
+    out1 = torch.empty((40, 72), device="cuda", dtype=F32)
+    out4 = torch.empty((300, 520), device="cuda", dtype=F32)
+    ws3 = torch.empty(P.pike_mlp_block_workspace(x3, w1), dtype=torch.uint8, device="cuda")
+    ws4 = torch.empty(P.pike_linear_epilogue_workspace(x3, wl, reduce="softmax", out_dtype=F32), dtype=torch.uint8,
+                      device="cuda")
+
+    def calls(stream=None):
+        P.pike_linear_epilogue(d1["x"], d1["w"], d1["b"], None, d1["gamma"], d1["beta"], act="gelu_erf",
+                               reduce="layernorm", eps=c1["eps"], out=out1, stream=stream)
+        P.pike_mlp_block(x3, g3, be3, w1, b1, w2, b2, act="gelu_tanh", eps=c3["eps"], out=out3, workspace=ws3,
+                         stream=stream)
+        P.pike_linear_epilogue(out3, wl, reduce="softmax", out_dtype=F32, out=out4, workspace=ws4, stream=stream)
+        P.pike_attention_chain(q, k, v, scale=float(c5["scale"]), causal=True, out=out5, stream=stream)
+
+    calls()                                  # warm: tensor maps encoded, the library's lazy state settled
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        calls()
+    for rep in range(3):
+        x3.copy_(dev(G.config3(M=300, D=136, F=520, seed=50 + rep, affine=True)["x"], BF16))
+        q.copy_(dev(G.config5(B=1, H=2, S=300, seed=60 + rep)["q"], BF16))
+        d1["x"].copy_(dev(G.config1(M=40, K=64, N=72, seed=70 + rep)["x"], F32))
+        for o in (out1, out3, out4, out5):
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got = [o.clone() for o in (out1, out3, out4, out5)]
+        for o in (out1, out3, out4, out5):
+            o.zero_()
+        calls()
+        torch.cuda.synchronize()
+        for a, b in zip(got, (out1, out3, out4, out5)):
+            assert torch.equal(a.view(torch.int32) if a.dtype == F32 else a.view(torch.int16),
+                               b.view(torch.int32) if b.dtype == F32 else b.view(torch.int16))
+    assert P.pike_get_last_device_status() == (0, 0)
+    # and the replayed MLP block is the right answer, not merely a reproducible one
+    c3r = G.config3(M=300, D=136, F=520, seed=52, affine=True)
+    want = O.mlp_block(c3r["x"], c3["gamma"], c3["beta"], c3["w1"], c3["b1"], c3["w2"], c3["b2"], act="gelu_tanh", eps=c3["eps"])
+    check_bf16(host64(out3), want, what="graph replay MLP block")
