@@ -162,7 +162,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // this CTA stages its half of the item's W columns; for a half tile the boxes keep their size
             // (the bytes a stage waits for stay the same) and only their first 64 columns are used
             produce_tile(tiles, ctrl, &tmA, &tmB, rp, num_kb, rt.row0 + (int)rank * BM,
-                         n_blk * BN + wk.col_off + (int)rank * (wk.ncols / 2), rt.group, p.w_is_nk != 0, rank, leader, ctx);
+                         n_blk * BN + wk.col_off + (int)rank * (wk.ncols / 2), rt.group, p.w_is_nk != 0, rank, leader, ctx,
+                         p.alternate_k != 0 && (((w - cluster_id) / num_clusters) & 1) != 0);
         }
     } else if (warp == 1) {
         // ---------- MMA issuer (leader CTA only; warp-uniform loop, one elected lane issues)
@@ -324,6 +325,12 @@ cudaError_t launch_gemm_bf16(const CUtensorMap &tmA, const CUtensorMap &tmB, con
         const bool along_n = a.group_offsets == nullptr && bytes_w + bytes_a * groups_n < bytes_a + bytes_w * groups_m;
         args.group_along_n = along_n ? 1 : 0;
         args.group_m = (int)(along_n ? gn : gm);
+        // The clusters that run side by side (74 = about 8 x 9 tiles) read about 17 slabs per round.  Where those
+        // no longer fit in half the L2, a round's slabs are gone from it when the next round - which shares the
+        // panel's slabs - begins, except their ends: each cluster then walks k in alternating directions (measured
+        // on 8192x16384x4096: 1665 -> 1505 MB read; with 2 MB slabs, which stay resident anyway, the alternation only
+        // costs sharing between clusters that are a round apart: +4 %, so it stays off there).
+        args.alternate_k = 17 * slab > (64ll << 20) ? 1 : 0;
     }
     // up to two work items per tile (see work_plan): small problems get both halves of a tile onto
     // different clusters

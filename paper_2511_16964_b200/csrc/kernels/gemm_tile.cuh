@@ -82,12 +82,16 @@ __device__ __forceinline__ void pair_teardown(Ctrl *ctrl, uint32_t tmem_base, in
 }
 
 // Producer warp, one tile: this CTA's 128 rows of A from row0 and its W columns from col0 (weight matrix `group`),
-// all k-blocks, through the ring.  Warp-uniform; `leader` is the one elected lane that issues.
+// all k-blocks, through the ring.  Warp-uniform; `leader` is the one elected lane that issues.  With `descending`
+// the k-blocks are fetched last to first (the sum does not care): a cluster alternates the direction from one of
+// its tiles to the next, so a tile that shares a slab with the previous one starts on the part of it that was read
+// last and is still in L2.
 __device__ __forceinline__ void produce_tile(uint8_t *tiles, Ctrl *ctrl, const CUtensorMap *tmA, const CUtensorMap *tmB,
                                              RingPos &rp, int num_kb, int row0, int col0, int group, bool w_is_nk,
-                                             uint32_t rank, bool leader, const WaitCtx &ctx)
+                                             uint32_t rank, bool leader, const WaitCtx &ctx, bool descending = false)
 {
-    for (int kb = 0; kb < num_kb; ++kb) {
+    for (int i = 0; i < num_kb; ++i) {
+        const int kb = descending ? num_kb - 1 - i : i;
         mbar_wait(&ctrl->empty[rp.s], rp.ph ^ 1, ctx, BAR_EMPTY);
         uint8_t *a_s = tiles + (size_t)rp.s * STAGE_BYTES;
         uint8_t *b_s = a_s + A_BYTES;

@@ -84,6 +84,7 @@ struct GemmArgs {
     unsigned int *stripe_counters;   // device, one per 256-row stripe, zero at launch
     int test_withhold_partials;      // test hook: block 0 never counts itself in, so every stripe wait runs out
     int pdl;                         // launch with programmatic stream serialisation (see launch_kernel); not for the one-pass kernel
+    int alternate_k;                 // set by the launcher: a cluster walks k downwards on every other of its tiles
 };
 // A CTA pair computes a (2*GEMM_BM) x GEMM_BN tile; each CTA stages GEMM_BM rows of A and half of
 // the tile's W columns.  Tensor-map boxes: A {GEMM_BK, GEMM_BM}; W as [N,K] {GEMM_BK, GEMM_BN/2};
