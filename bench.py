@@ -665,11 +665,13 @@ def run_ours(args):
                         "full_size_seconds_extrapolated": sum(full.values()), "full_size_seconds_per_config": full}
 
     # ---- the further workloads (outside `value`): one at a time, each with its own tensors ---------------
+    variants = None
     if world == 1 and not args.no_extras:
         del suite, d, out, chains, host_act, host_out
         torch.cuda.empty_cache()
         for x in EXTRA:
             per_config[x] = extra_workload(P, torch, device, x, not args.no_eager)
+        variants = variant_rows(P, torch, device)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -698,7 +700,7 @@ def run_ours(args):
         "frac_of_nominal_2250": value / world / NOMINAL_BF16_TFLOPS,
         "sustained": sustained, "per_config": per_config, "context": context, "kernels": kernels, "parity": parity,
         "host_call_us": host_call_us, "library_gemm_same_box": library_gemm,
-        "graph_replay_ms_per_step": graph_ms,
+        "graph_replay_ms_per_step": graph_ms, "variants": variants,
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -742,6 +744,55 @@ def extra_workload(P, torch, device, name, with_eager, iters=10):
     del s
     torch.cuda.empty_cache()
     return row
+
+
+def variant_rows(P, torch, device, runs=5):
+    """Further shapes and types the entry points accept (parity of each in tests/): timed here cold, one by one, on
+    seeded random tensors; never part of `value`.  TFLOP/s counts GEMM flops (attention: the live half under the mask)."""
+    BF16, F16, F32 = torch.bfloat16, torch.float16, torch.float32
+    g = torch.Generator(device=device).manual_seed(2511)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def rn(*shape, dt=BF16, sc=1.0):
+        return (torch.randn(*shape, device=device, generator=g) * sc).to(dt)
+
+    def attn(B, H, S, Sk, D, dt, causal):
+        q, k, v = rn(B, H, S, D, dt=dt), rn(B, H, Sk, D, dt=dt), rn(B, H, Sk, D, dt=dt)
+        o = torch.empty_like(q)
+        fl = 4.0 * B * H * D * (S * (S + 1) / 2 if causal else S * Sk)
+        return (lambda: P.pike_attention_chain(q, k, v, scale=D ** -0.5, causal=causal, out=o)), fl
+
+    def linear(M, K, N, dt, **kw):
+        x, w, b = rn(M, K, dt=dt), rn(K, N, dt=dt, sc=K ** -0.5), rn(N, dt=dt)
+        r = rn(M, N, dt=dt) if kw.pop("residual", False) else None
+        gm, be = (rn(N, dt=dt), rn(N, dt=dt)) if kw.get("reduce") == "layernorm" else (None, None)
+        o = torch.empty((M, N), dtype=kw.get("out_dtype", dt), device=device)
+        nbytes = P.pike_linear_epilogue_workspace(x, w, **{k: v for k, v in kw.items() if k in ("act", "scale", "reduce", "eps", "out_dtype")})
+        ws = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=device)
+        return (lambda: P.pike_linear_epilogue(x, w, b, r, gm, be, out=o, workspace=ws, **kw)), 2.0 * M * K * N
+
+    cases = {
+        "attention non-causal bf16 B8 H32 S2048 D128": lambda: attn(8, 32, 2048, 2048, 128, BF16, False),
+        "attention causal bf16 B8 H64 S2048 D64": lambda: attn(8, 64, 2048, 2048, 64, BF16, True),
+        "attention causal f16 B8 H32 S2048 D128": lambda: attn(8, 32, 2048, 2048, 128, F16, True),
+        "cross attention bf16 B8 H32 S1024 Sk4096 D128": lambda: attn(8, 32, 1024, 4096, 128, BF16, False),
+        "linear+GELU+LayerNorm (split-row epilogue) bf16 8192x4096x4096": lambda: linear(8192, 4096, 4096, BF16, act="gelu_tanh", reduce="layernorm"),
+        "linear+SiLU+scale+residual f16 4096^3": lambda: linear(4096, 4096, 4096, F16, act="silu", scale=0.5, residual=True),
+    }
+    rows = {}
+    for name, make in cases.items():
+        try:
+            fn, fl = make()
+            ms = _timed_cold(torch, fn, flush, iters=runs)
+            rows[name] = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
+                          "frac_of_nominal_2250": fl / (ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+            del fn
+        except Exception as exc:           # noqa: BLE001 - a context row must never break the benchmark
+            rows[name] = {"ms": None, "error": repr(exc)[:200]}
+        torch.cuda.empty_cache()
+    st, _ = P.pike_get_last_device_status()
+    rows["device_status"] = st
+    return rows
 
 
 def host_call_overhead(P, torch, suite, calls=400):
