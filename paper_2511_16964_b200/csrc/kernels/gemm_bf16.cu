@@ -140,14 +140,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();           // 0 = leader
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    // barriers, tensor memory and the wait for the previous kernel of the stream first: the group offsets below are
+    // device data that kernel may have written
+    const uint32_t tmem_base = pair_setup(ctrl, &tmA, &tmB, warp);
+    const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
     build_group_table(p, first_tile);
     const int num_m = count_row_tiles(p, first_tile), num_n = (p.N + BN - 1) / BN;
     const int num_tiles = num_m * num_n;
     const int num_kb = (p.K + BK - 1) / BK;
     const WorkPlan plan = work_plan(num_tiles, num_clusters, p.row_partials == 0);
-
-    const uint32_t tmem_base = pair_setup(ctrl, &tmA, &tmB, warp);
-    const WaitCtx ctx{p.status, &ctrl->abort, p.limit_ns, KID_GEMM};
 
     if (warp == 0) {
         // -------------------- TMA producer (warp-uniform loop, one elected lane issues)
