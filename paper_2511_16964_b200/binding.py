@@ -145,9 +145,13 @@ def _tensor(t):
     d.data = t.data_ptr()
     d.dtype = _dtype_code(t)
     d.ndim = t.dim()
-    for i in range(t.dim()):
+    # torch leaves the stride of an extent-1 dimension arbitrary (a [1, K] view of a [K, 1] array keeps stride 1);
+    # the C ABI wants every outer stride to cover the dimensions inside it, so such strides are canonicalised here
+    inner = 1
+    for i in reversed(range(t.dim())):
         d.shape[i] = t.shape[i]
-        d.stride[i] = t.stride(i)
+        d.stride[i] = t.stride(i) if t.shape[i] != 1 else max(inner, 1)
+        inner = max(inner, d.stride[i] * t.shape[i])
     return ctypes.byref(d)
 
 

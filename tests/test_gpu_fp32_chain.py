@@ -71,3 +71,19 @@ def test_empty_batch_and_rejections():
         buf = torch.zeros(4 * 16 + 1, device="cuda")
         P.pike_linear_epilogue(buf[1:].view(4, 16), w)
     assert e.value.code == 4
+
+
+@pytest.mark.parametrize("M,K,N", [(182, 148, 1), (91, 1, 840), (1, 64, 72)])
+def test_extent_one_dimensions_with_arbitrary_strides(M, K, N):
+    """torch leaves the stride of an extent-1 dimension arbitrary: a [1, K] transpose view of a [K, 1] tensor keeps
+    stride 1 for its single row.  Such views are accepted (the binding hands the C ABI canonical strides)."""
+    import paper_2511_16964_b200 as P
+    c = G.config1(M=M, K=K, N=N, seed=9)
+    w_t = dev(c["w"], F32).t()                              # [N, K] view of the [K, N] tensor
+    if N == 1 or K == 1:
+        assert w_t.is_contiguous() and w_t.stride() != (K, 1)      # the case this test is about
+    x = dev(c["x"], F32)
+    out = P.pike_linear_epilogue(x, w_t if w_t.is_contiguous() else w_t.contiguous(), dev(c["b"], F32), act="gelu_erf",
+                                 reduce="layernorm", eps=c["eps"], w_is_nk=True)
+    want = O.linear_epilogue(c["x"], c["w"], c["b"], act="gelu_erf", reduce="layernorm", eps=c["eps"])
+    check_f32(host64(out), want, 1e-4, f"{M}x{K}x{N} with an extent-1 stride")
