@@ -141,3 +141,33 @@ def test_rejections():
         P.pike_attention_chain(q, q.clone(), q.clone(), scale=0.0)
     assert e.value.code == 6
     assert P.pike_attention_chain_workspace(q, scale=1.0) == 0
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f16"])
+@pytest.mark.parametrize("pattern", ["rising", "falling", "late spike", "huge scores"])
+def test_row_maxima_that_move_between_key_tiles(pattern, dtype):
+    """The accumulator is only rescaled when a row's maximum grows by more than a threshold (lazy rescale): keys
+    whose scores rise steadily from tile to tile force a rescale at every step, falling ones none after the first,
+    a single late key with a far larger score makes everything before it vanish, and scores in the hundreds leave
+    one probability per row.  All four must come out like the plain definition."""
+    import paper_2511_16964_b200 as P
+    tdt = BF16 if dtype == "bf16" else torch.float16
+    S, D = 5 * 128 + 37, 128
+    c = G.config5(B=1, H=2, S=S, D=D, seed=77, dtype=dtype)
+    k = c["k"].astype(np.float64)
+    tile = np.arange(S) // 128
+    if pattern == "rising":
+        k *= (1.0 + 2.0 * tile)[None, None, :, None]
+    elif pattern == "falling":
+        k *= (1.0 + 2.0 * tile[::-1])[None, None, :, None]
+    elif pattern == "late spike":
+        k[:, :, 4 * 128 + 5, :] = 6.0 * np.sign(c["q"][:, :, -1:, :].astype(np.float64).mean(axis=2))
+    else:
+        k *= 16.0
+    k = G.round_to(k.astype(np.float32), dtype)
+    scale = 1.0 if pattern == "huge scores" else c["scale"]
+    for causal in (False, True):
+        got = host64(P.pike_attention_chain(dev(c["q"], tdt), dev(k, tdt), dev(c["v"], tdt), scale=scale, causal=causal))
+        assert P.pike_get_last_device_status() == (0, 0)
+        want = O.attention(c["q"], k, c["v"], scale=scale, causal=causal)
+        check_bf16(got, want, what=f"{pattern} {dtype} causal={causal}")
