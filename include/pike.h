@@ -129,7 +129,8 @@ pike_status_t pike_get_last_device_status(pike_handle_t handle, pike_status_t *s
 pike_status_t pike_set_wait_limit_ns(pike_handle_t handle, uint64_t ns);
 
 /* Test hook for the failure-detection path (no counterpart in the paper): the NEXT bf16 GEMM launched
- * through this handle issues no operand loads, so its first wait for data runs out after the wait limit,
+ * through this handle issues no operand loads (the next fp32 chain, if that comes first: none of the bulk copies
+ * its small-problem kernel stages 16-byte aligned operands with), so its first wait for data runs out after the wait limit,
  * the kernel records where, skips its remaining waits, runs to its end (the output is garbage) and
  * pike_get_last_device_status reports PIKE_ERR_TIMEOUT.  Nothing faults, traps or hangs; the context and
  * the handle stay usable.  Use with a small pike_set_wait_limit_ns. */

@@ -31,7 +31,7 @@ struct pike_handle_s {
     int num_sms;
     unsigned int *status;  // device, 4 words
     unsigned long long limit_ns;
-    bool withhold_next;    // pike_test_withhold_loads: applies to the next bf16 GEMM launch only
+    bool withhold_next;    // pike_test_withhold_loads: applies to the next bf16 GEMM or fp32 chain launch only
     bool withhold_partials_next;   // pike_test_withhold_partials: applies to the next one-pass softmax launch only
     PFN_cuTensorMapEncodeTiled_v12000 encode;
     cudaStream_t aux_stream;      // non-blocking; carries the status-word reads so that they wait for nobody's kernels
@@ -90,7 +90,8 @@ struct TimedLaunch {
     }
 };
 
-// Encode (or fetch from the handle's cache) a tiled tensor map with 128-byte swizzle over 16-bit elements.
+// Encode (or fetch from the handle's cache) a tiled tensor map: 128-byte swizzle over 16-bit elements, no swizzle
+// over fp32 elements (the fp32 chain reads its tiles with plain shared-memory loads).
 inline pike_status_t tensor_map(pike_handle_t h, CUtensorMap *out, const TensorMapKey &key)
 {
     for (size_t i = 0; i < h->map_cache.size(); ++i) {
@@ -109,7 +110,8 @@ inline pike_status_t tensor_map(pike_handle_t h, CUtensorMap *out, const TensorM
     for (int i = 0; i < 4; ++i) { dims[i] = key.dims[i]; box[i] = key.box[i]; }
     for (int i = 0; i < 3; ++i) strides[i] = key.strides[i];
     const CUresult r = h->encode(out, static_cast<CUtensorMapDataType>(key.dtype), key.rank, const_cast<void *>(key.ptr),
-                                 dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 key.dtype == CU_TENSOR_MAP_DATA_TYPE_FLOAT32 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return PIKE_ERR_CUDA;
     if (h->map_cache.size() >= pike_handle_s::MAP_CACHE_SIZE) h->map_cache.pop_back();
@@ -134,6 +136,18 @@ inline pike_status_t make_map_2d(pike_handle_t h, CUtensorMap *map, pike_dtype_t
     TensorMapKey k = make_key(ptr, dt, 2);
     k.dims[0] = cols; k.dims[1] = rows;
     k.strides[0] = pitch_elems * 2;
+    k.box[0] = box_cols; k.box[1] = box_rows;
+    return tensor_map(h, map, k);
+}
+
+// fp32 [rows, cols] row-major matrix -> unswizzled tensor map with a (box_cols x box_rows) box
+inline pike_status_t make_map_2d_f32(pike_handle_t h, CUtensorMap *map, const void *ptr, uint64_t rows, uint64_t cols,
+                                     uint64_t pitch_elems, uint32_t box_cols, uint32_t box_rows)
+{
+    TensorMapKey k = make_key(ptr, PIKE_BF16, 2);
+    k.dtype = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+    k.dims[0] = cols; k.dims[1] = rows;
+    k.strides[0] = pitch_elems * 4;
     k.box[0] = box_cols; k.box[1] = box_rows;
     return tensor_map(h, map, k);
 }

@@ -363,10 +363,24 @@ pike_status_t pike_linear_epilogue(pike_handle_t h, const pike_tensor_t *x, cons
         a.w_is_nk = s.w_is_nk;
         a.act = (int)epi->act; a.reduce = (int)epi->reduce;
         a.scale = epi->scale; a.eps = epi->eps;
+        a.status = h->status; a.limit_ns = h->limit_ns;
+        a.test_withhold_loads = h->withhold_next ? 1 : 0;
+        h->withhold_next = false;
         PIKE_LOGF(h, "fp32_chain_kernel M=%d K=%d N=%d act=%d reduce=%d w=%s", a.M, a.K, a.N, a.act, a.reduce,
                   a.w_is_nk ? "[N,K]" : "[K,N]");
+        pike::Fp32ChainPlan plan = pike::plan_fp32_chain(a, h->num_sms);
+        CUtensorMap tm_x, tm_w;
+        // a map that cannot be encoded (a pitch beyond the format's range, say) only means per-thread copies
+        if (plan.tma_x && make_map_2d_f32(h, &tm_x, a.x, (uint64_t)a.M, (uint64_t)a.K, (uint64_t)a.ldx, plan.x_box[0],
+                                          plan.x_box[1]) != PIKE_OK)
+            plan.tma_x = 0;
+        if (plan.tma_w && make_map_2d_f32(h, &tm_w, a.w, (uint64_t)a.K, (uint64_t)a.N, (uint64_t)a.ldw, plan.w_box[0],
+                                          plan.w_box[1]) != PIKE_OK)
+            plan.tma_w = 0;
+        PIKE_LOGF(h, "fp32_chain plan rows/thread=%d cols/cta=%d cluster=%d kc=%d tiled x=%d w=%d", plan.rpt, 32 * plan.cw,
+                  plan.cn, plan.kc, plan.tma_x, plan.tma_w);
         TimedLaunch timed(h, PIKE_KERNEL_FP32_CHAIN, stream);
-        return pike::launch_fp32_chain(a, h->num_sms, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
+        return pike::launch_fp32_chain(a, plan, &tm_x, &tm_w, stream) == cudaSuccess ? PIKE_OK : PIKE_ERR_CUDA;
     }
 
     for (const pike_tensor_t *t : {bias, residual, gamma, beta})

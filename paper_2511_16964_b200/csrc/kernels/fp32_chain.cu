@@ -6,8 +6,14 @@
 // (BN = 32, 64 or 128 columns each, at most 8 CTAs for N <= 1024).  Each CTA stages only its own
 // column slice of W (K x BN) and the BM rows of x in shared memory, so W crosses the L2 once per
 // row block instead of once per CTA-row as a one-CTA-per-row layout would have it, and the
-// whole problem spreads over many SMs even when M is small.  Thread (lane, warp) accumulates
-// columns lane + 32c of rows warp + 8i; k runs in ascending order per output (plain fp32 FMA).
+// whole problem spreads over many SMs even when M is small.
+// Two kernels share the staging, the epilogue and the reduction:
+//  - fp32_chain_splitk_kernel (BM = 8; small problems, whose time is a chain of latencies): the eight
+//    warps split k, every thread accumulates all 8 rows of its columns over its warp's k slice (8 FMAs per
+//    shared-memory word of W instead of one), and the warps' partial sums meet in shared memory.  Operands
+//    arrive as row-wise bulk copies on one mbarrier where the addresses allow it.
+//  - fp32_chain_kernel (BM = 16 or 32; problems that fill the chip): thread (lane, warp) accumulates
+//    columns lane + 32c of rows warp + 8i over all of k.
 // The LayerNorm / softmax reduction over N never leaves the cluster: every warp reduces its rows
 // over the CTA's columns with shuffles, the CTAs publish one pair per row - (mean, sum of squared
 // deviations) or (max, sum exp) - in their shared memory, and after one cluster barrier every CTA
@@ -16,12 +22,15 @@
 #include "../device/ptx.cuh"
 #include "kernels.h"
 
+#include <string.h>
+
 namespace pike {
 namespace {
 
-constexpr int FT = 256;                    // 8 warps: warp = row lane, lane = column lane
-constexpr int SMEM_FLOATS_MAX = 24576;     // 96 KiB of operand tiles per CTA
+constexpr int FT = 256;                    // 8 warps
+constexpr int SMEM_FLOATS_MAX = 24576;     // 96 KiB of shared memory per CTA
 constexpr int MAX_BM = 32;
+constexpr int SPLITK_BM = 8;
 
 __device__ __forceinline__ float act_by_id(int act, float y)
 {
@@ -46,134 +55,99 @@ __device__ __forceinline__ float warp_max_f(float x)
     return x;
 }
 
-// RPT rows and CW columns per thread: the CTA tile is (8 RPT) x (32 CW).  NK: w is [N,K].
-template <int RPT, int CW, bool NK>
-__global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, const int kc)
+// The per-column parameters of a thread's columns (n0 + lane + 32c); fetched before the main loop so that
+// their latency hides under it.
+template <int CW>
+struct ColParams {
+    float bias[CW], gamma[CW], beta[CW];
+};
+template <int CW>
+__device__ __forceinline__ void load_col_params(const Fp32ChainArgs &a, int n0, int lane, ColParams<CW> &p)
 {
-    constexpr int BM = 8 * RPT, BN = 32 * CW;
-    extern __shared__ __align__(16) float smem[];
-    __shared__ float2 stat[MAX_BM];        // this CTA's per-row pair, read by the whole cluster
-    float *x_s = smem;                     // [BM][kc]
-    float *w_s = x_s + BM * kc;            // [kc][BN], or [BN][kc + 1] for NK (odd pitch: no bank conflicts)
-
-    const int tid = threadIdx.x, lane = tid & 31, rg = tid >> 5;
-    const int cn = (int)cluster_nctas(), rank = (int)cluster_ctarank();
-    const long long row0 = (long long)((int)blockIdx.x / cn) * BM;
-    const int n0 = rank * BN;
-    const int n_loc = min(max(a.N - n0, 0), BN);      // columns this CTA owns (0 for a padding rank)
-    pdl_wait();
-
-    float acc[RPT][CW][4];
-#pragma unroll
-    for (int i = 0; i < RPT; ++i)
-#pragma unroll
-        for (int c = 0; c < CW; ++c)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][c][j] = 0.0f;
-    // the per-column parameters are fetched now, so their latency hides under the main loop
-    float bias_r[CW], gamma_r[CW], beta_r[CW];
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
         const int col = n0 + lane + 32 * c;
         const bool col_ok = col < a.N;
-        bias_r[c] = (a.bias != nullptr && col_ok) ? __ldg(a.bias + col) : 0.0f;
-        gamma_r[c] = (a.reduce == 1 && a.gamma != nullptr && col_ok) ? __ldg(a.gamma + col) : 1.0f;
-        beta_r[c] = (a.reduce == 1 && a.beta != nullptr && col_ok) ? __ldg(a.beta + col) : 0.0f;
+        p.bias[c] = (a.bias != nullptr && col_ok) ? __ldg(a.bias + col) : 0.0f;
+        p.gamma[c] = (a.reduce == 1 && a.gamma != nullptr && col_ok) ? __ldg(a.gamma + col) : 1.0f;
+        p.beta[c] = (a.reduce == 1 && a.beta != nullptr && col_ok) ? __ldg(a.beta + col) : 0.0f;
     }
+}
 
-    const bool x_vec = (a.ldx & 3) == 0;                         // rows of x start on 16-byte boundaries
-    const bool w_vec = (a.ldw & 3) == 0 && (n_loc & 3) == 0;
-    for (int k0 = 0; k0 < a.K; k0 += kc) {
-        const int kn = min(kc, a.K - k0);
-        const int kn4 = kn & ~3;
-        __syncthreads();                                         // the previous chunk has been consumed
-        // Everything is fetched with asynchronous copies, so all of a thread's loads are in flight together (the
-        // problem is small: its time is a few memory latencies, which must not add up).  16-byte copies where
-        // the rows are 16-byte aligned, 4-byte copies otherwise; elements outside the tensors are written as zeros.
-        // ---- x rows [row0, row0 + BM) x k [k0, k0 + kn)
-        const int kr = (kn + 3) & ~3;          // the FMA loop reads k in quads: positions kn .. kr-1 must hold zeros
-        if (x_vec) {
-            for (int idx = tid; idx < BM * (kr >> 2); idx += FT) {
-                const int r = idx / (kr >> 2), k = (idx - r * (kr >> 2)) << 2;
-                const long long row = row0 + r;
-                const float *src = a.x + (row < a.M ? row * a.ldx + k0 + k : 0);
-                if (k < kn4) {
-                    cp_async_16(x_s + r * kc + k, src, row < a.M);
-                } else {                        // the quad that holds the end of the row, element by element
+// ---- staging with per-thread asynchronous copies: any alignment, any tail.  16-byte copies where the rows
+// are 16-byte aligned, 4-byte copies otherwise; elements outside the tensors are written as zeros.  All of a
+// thread's copies are in flight together; the caller waits for them (cp_async_wait_all + __syncthreads).
+// x rows [row0, row0 + BM) x k [k0, k0 + kn) -> x_s [BM][kc]; positions kn .. kr-1 (kr = kn rounded up to four:
+// the FMA loops read k in quads) are zeroed.
+template <int BM>
+__device__ __forceinline__ void stage_x_cp_async(const Fp32ChainArgs &a, float *x_s, int kc, int k0, int kn,
+                                                 long long row0, int tid)
+{
+    const int kn4 = kn & ~3, kr = (kn + 3) & ~3;
+    if ((a.ldx & 3) == 0) {
+        const int qpr = kr >> 2;               // quads per row
+        for (int idx = tid; idx < BM * qpr; idx += FT) {
+            const int r = idx / qpr, k = (idx - r * qpr) << 2;
+            const long long row = row0 + r;
+            const float *src = a.x + (row < a.M ? row * a.ldx + k0 + k : 0);
+            if (k < kn4) {
+                cp_async_16(x_s + r * kc + k, src, row < a.M);
+            } else {                            // the quad that holds the end of the row, element by element
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const bool ok = row < a.M && k + j < kn;
-                        cp_async_4(x_s + r * kc + k + j, ok ? src + j : a.x, ok);
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    const bool ok = row < a.M && k + j < kn;
+                    cp_async_4(x_s + r * kc + k + j, ok ? src + j : a.x, ok);
                 }
+            }
+        }
+    } else {
+        for (int idx = tid; idx < BM * kr; idx += FT) {
+            const int r = idx / kr, k = idx - r * kr;
+            const long long row = row0 + r;
+            const bool ok = row < a.M && k < kn;
+            cp_async_4(x_s + r * kc + k, ok ? a.x + row * a.ldx + k0 + k : a.x, ok);
+        }
+    }
+}
+// This CTA's column slice of W: [kc][BN], or for [N,K] weights transposed as [BN][kc + 1], one element per
+// copy (the odd pitch that keeps the FMA loop free of bank conflicts leaves no 16-byte aligned rows).
+template <int BN, bool NK>
+__device__ __forceinline__ void stage_w_cp_async(const Fp32ChainArgs &a, float *w_s, int kc, int k0, int kn, int n0,
+                                                 int n_loc, int tid)
+{
+    const int kr = (kn + 3) & ~3;
+    if constexpr (!NK) {
+        if ((a.ldw & 3) == 0 && (n_loc & 3) == 0) {
+            for (int idx = tid; idx < kr * (BN >> 2); idx += FT) {
+                const int k = idx / (BN >> 2), c = (idx - k * (BN >> 2)) << 2;
+                const bool ok = c < n_loc && k < kn;
+                cp_async_16(w_s + k * BN + c, ok ? a.w + (long long)(k0 + k) * a.ldw + n0 + c : a.w, ok);
             }
         } else {
-            for (int idx = tid; idx < BM * kr; idx += FT) {
-                const int r = idx / kr, k = idx - r * kr;
-                const long long row = row0 + r;
-                const bool ok = row < a.M && k < kn;
-                cp_async_4(x_s + r * kc + k, ok ? a.x + row * a.ldx + k0 + k : a.x, ok);
+            for (int idx = tid; idx < kr * BN; idx += FT) {
+                const int k = idx / BN, c = idx - k * BN;
+                const bool ok = c < n_loc && k < kn;
+                cp_async_4(w_s + k * BN + c, ok ? a.w + (long long)(k0 + k) * a.ldw + n0 + c : a.w, ok);
             }
         }
-        // ---- this CTA's column slice of W
-        if (n_loc > 0) {
-            if constexpr (!NK) {
-                if (w_vec) {
-                    for (int idx = tid; idx < kr * (BN >> 2); idx += FT) {
-                        const int k = idx / (BN >> 2), c = (idx - k * (BN >> 2)) << 2;
-                        const bool ok = c < n_loc && k < kn;
-                        cp_async_16(w_s + k * BN + c, ok ? a.w + (long long)(k0 + k) * a.ldw + n0 + c : a.w, ok);
-                    }
-                } else {
-                    for (int idx = tid; idx < kr * BN; idx += FT) {
-                        const int k = idx / BN, c = idx - k * BN;
-                        const bool ok = c < n_loc && k < kn;
-                        cp_async_4(w_s + k * BN + c, ok ? a.w + (long long)(k0 + k) * a.ldw + n0 + c : a.w, ok);
-                    }
-                }
-            } else {
-                // [N,K] weights land transposed, one element per copy: the odd pitch that keeps the FMA loop free of
-                // bank conflicts leaves no 16-byte aligned rows
-                const int pitch = kc + 1;
-                for (int idx = tid; idx < BN * kr; idx += FT) {
-                    const int c = idx / kr, k = idx - c * kr;
-                    const bool ok = c < n_loc && k < kn;
-                    cp_async_4(w_s + c * pitch + k, ok ? a.w + (long long)(n0 + c) * a.ldw + k0 + k : a.w, ok);
-                }
-            }
-        }
-        cp_async_wait_all();
-        __syncthreads();
-        if (n_loc > 0) {
-            // four k at a time: one 16-byte broadcast load of x per row, four column loads of w, and four
-            // independent accumulators per output (k = 0, 1, 2, 3 mod 4) so that consecutive FMAs do not wait
-            // for one another; the tail of a chunk that is not a multiple of four reads the zeros staged above
-#pragma unroll 2
-            for (int k = 0; k < kn; k += 4) {
-                float4 xv[RPT];
-                float wv[CW][4];
-#pragma unroll
-                for (int i = 0; i < RPT; ++i) xv[i] = *reinterpret_cast<const float4 *>(x_s + (rg + 8 * i) * kc + k);
-#pragma unroll
-                for (int c = 0; c < CW; ++c)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        wv[c][j] = NK ? w_s[(lane + 32 * c) * (kc + 1) + k + j] : w_s[(k + j) * BN + lane + 32 * c];
-#pragma unroll
-                for (int i = 0; i < RPT; ++i)
-#pragma unroll
-                    for (int c = 0; c < CW; ++c) {
-                        acc[i][c][0] = fmaf(xv[i].x, wv[c][0], acc[i][c][0]);
-                        acc[i][c][1] = fmaf(xv[i].y, wv[c][1], acc[i][c][1]);
-                        acc[i][c][2] = fmaf(xv[i].z, wv[c][2], acc[i][c][2]);
-                        acc[i][c][3] = fmaf(xv[i].w, wv[c][3], acc[i][c][3]);
-                    }
-            }
+    } else {
+        const int pitch = kc + 1;
+        for (int idx = tid; idx < BN * kr; idx += FT) {
+            const int c = idx / kr, k = idx - c * kr;
+            const bool ok = c < n_loc && k < kn;
+            cp_async_4(w_s + c * pitch + k, ok ? a.w + (long long)(n0 + c) * a.ldw + k0 + k : a.w, ok);
         }
     }
+}
 
-    // ---- epilogue in registers: bias -> activation -> scale -> residual
-    float v[RPT][CW];
+// ---- from the dot products to the stored output: bias -> activation -> scale -> residual in registers, then
+// the row reduction.  Warp rg owns rows rg + 8i of the block, lane the columns n0 + lane + 32c.
+template <int RPT, int CW>
+__device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, float (&v)[RPT][CW],
+                                                      const ColParams<CW> &p, float2 *stat, long long row0, int n0,
+                                                      int n_loc, int lane, int rg, int cn)
+{
+    constexpr int BN = 32 * CW;
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
         const int col = n0 + lane + 32 * c;
@@ -181,8 +155,7 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
             const long long row = row0 + rg + 8 * i;
-            const float dot = (acc[i][c][0] + acc[i][c][1]) + (acc[i][c][2] + acc[i][c][3]);
-            float y = a.scale * act_by_id(a.act, dot + bias_r[c]);
+            float y = a.scale * act_by_id(a.act, v[i][c] + p.bias[c]);
             if (a.residual != nullptr && col_ok && row < a.M) y += __ldg(a.residual + row * a.ldr + col);
             v[i][c] = y;
         }
@@ -220,35 +193,27 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
             if (lane == 0) stat[rg + 8 * i] = make_float2(s0, s1);
         }
         cluster_sync_all();                            // every rank's pairs are visible cluster-wide
-        // ---- merge the ranks' pairs (lane r fetches rank r's pair; merged in rank order, so every CTA
-        //      of the cluster computes bit-identical statistics)
+        // ---- merge the ranks' pairs: lane r fetches rank r's pair, the merge is a warp reduction over the
+        //      lanes (the same tree in every CTA, so the whole cluster computes bit-identical statistics).
+        //      LayerNorm pools the ranks' moments about the pooled mean (deviations of means: no E[x^2] - E[x]^2
+        //      cancellation).
+        const float nr = lane < cn ? (float)min(max(a.N - lane * BN, 0), BN) : 0.0f;   // columns of rank `lane`
+        const float inv_n = 1.0f / (float)a.N;
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
             float2 mine = make_float2(0.0f, 0.0f);
             if (lane < cn) mine = ld_shared_cluster_f32x2(mapa_shared(smem_u32(&stat[rg + 8 * i]), (uint32_t)lane));
             if (a.reduce == 1) {
-                float n_run = 0.0f, mean = 0.0f, m2 = 0.0f;
-                for (int r = 0; r < cn; ++r) {
-                    const float mr = __shfl_sync(0xffffffffu, mine.x, r), qr = __shfl_sync(0xffffffffu, mine.y, r);
-                    const float nr = (float)min(max(a.N - r * BN, 0), BN);
-                    if (nr > 0.0f) {                   // pairwise (Chan) update: no E[x^2] - E[x]^2 cancellation
-                        const float n_new = n_run + nr, delta = mr - mean;
-                        mean += delta * (nr / n_new);
-                        m2 += qr + delta * delta * (n_run * nr / n_new);
-                        n_run = n_new;
-                    }
-                }
-                const float rstd = rsqrtf(m2 / (float)a.N + a.eps);
+                const float mean = warp_sum_f(nr * mine.x) * inv_n;
+                const float d = mine.x - mean;
+                const float m2 = warp_sum_f(mine.y + nr * d * d);
+                const float rstd = rsqrtf(m2 * inv_n + a.eps);
 #pragma unroll
-                for (int c = 0; c < CW; ++c) v[i][c] = (v[i][c] - mean) * rstd * gamma_r[c] + beta_r[c];
+                for (int c = 0; c < CW; ++c) v[i][c] = (v[i][c] - mean) * rstd * p.gamma[c] + p.beta[c];
             } else {
-                float m = -INFINITY;
-                for (int r = 0; r < cn; ++r) m = fmaxf(m, __shfl_sync(0xffffffffu, mine.x, r));
-                float l = 0.0f;
-                for (int r = 0; r < cn; ++r) {
-                    const float mr = __shfl_sync(0xffffffffu, mine.x, r), lr = __shfl_sync(0xffffffffu, mine.y, r);
-                    if (lr > 0.0f) l += lr * expf(mr - m);
-                }
+                const bool has = nr > 0.0f && mine.y > 0.0f;
+                const float m = warp_max_f(has ? mine.x : -INFINITY);
+                const float l = warp_sum_f(has ? mine.y * expf(mine.x - m) : 0.0f);
                 const float inv = 1.0f / l;
 #pragma unroll
                 for (int c = 0; c < CW; ++c) v[i][c] = expf(v[i][c] - m) * inv;
@@ -272,16 +237,200 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
     if (a.reduce != 0) cluster_wait();
 }
 
+// ---- small problems: the warps split k ------------------------------------------------------------
+// CTA tile 8 x (32 CW).  Warp w accumulates ALL 8 rows of columns lane + 32c over its eighth of every staged
+// k chunk (k ascending), so a word of W read from shared memory feeds 8 FMAs and a 16-byte broadcast of x
+// feeds 4 CW; the eight partial sums per output meet in shared memory and are added in a fixed tree.
+// Staging: where the tensors allow a tensor map (16-byte aligned base and row pitch; W as [K,N]) ONE thread
+// fetches the chunk's x rows and W slice as two tiled copies completing on one mbarrier (bounded wait); rows,
+// columns and k past the tensors arrive as zeros.  Otherwise the per-thread asynchronous copies above.
+// (Row-wise untiled bulk copies were measured too: 264 small copies per CTA queue up for about 11 cycles each.)
+// NK: w is [N,K].
+template <int CW, bool NK>
+__global__ void __launch_bounds__(FT) fp32_chain_splitk_kernel(const Fp32ChainArgs a, const int kc, const int tma_x,
+                                                               const int tma_w,
+                                                               const __grid_constant__ CUtensorMap tm_x,
+                                                               const __grid_constant__ CUtensorMap tm_w)
+{
+    constexpr int BM = SPLITK_BM, BN = 32 * CW;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ float2 stat[BM];            // this CTA's per-row pair, read by the whole cluster
+    __shared__ uint64_t full;              // the tiled copies of a chunk complete here
+    __shared__ uint32_t abort_word;
+    // tiled copies want 128-byte aligned destinations: x_s is, and w_s follows it by 32 kc bytes (kc a multiple of 4)
+    float *x_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));   // [BM][kc]
+    float *w_s = x_s + BM * kc;                            // [kc][BN], or [BN][kc + 1] for NK
+    float *red = w_s + (NK ? BN * (kc + 1) : kc * BN);     // [8 warps][BM][BN]
+
+    const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
+    const int cn = (int)cluster_nctas(), rank = (int)cluster_ctarank();
+    const long long row0 = (long long)((int)blockIdx.x / cn) * BM;
+    const int n0 = rank * BN;
+    const int n_loc = min(max(a.N - n0, 0), BN);          // columns this CTA owns (0 for a padding rank)
+    const bool x_tiled = tma_x != 0, w_tiled = !NK && tma_w != 0 && n_loc > 0;
+    const uint32_t chunk_bytes = (x_tiled ? (uint32_t)(BM * kc * 4) : 0u) + (w_tiled ? (uint32_t)(kc * BN * 4) : 0u);
+    if (tid == 0) {
+        abort_word = 0;
+        mbar_init(&full, 1);
+        fence_barrier_init();
+        if (x_tiled) tma_prefetch_desc(&tm_x);
+        if (w_tiled) tma_prefetch_desc(&tm_w);
+    }
+    __syncthreads();
+    pdl_wait();
+    const WaitCtx ctx{a.status, &abort_word, a.limit_ns, KID_FP32_CHAIN};
+
+    float acc[BM][CW];
+#pragma unroll
+    for (int r = 0; r < BM; ++r)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) acc[r][c] = 0.0f;
+    ColParams<CW> prm;
+
+    uint32_t phase = 0;
+    for (int k0 = 0; k0 < a.K; k0 += kc) {
+        const int kn = min(kc, a.K - k0);
+        const int kr = (kn + 3) & ~3;
+        if (k0 > 0) __syncthreads();       // the previous chunk has been consumed
+        if (tid == 0 && chunk_bytes != 0) {
+            mbar_arrive_expect_tx(&full, chunk_bytes);     // whole boxes: what lies outside the tensors is zero-filled
+            if (a.test_withhold_loads == 0) {
+                if (x_tiled) tma_load_2d(x_s, &tm_x, &full, k0, (int)row0);
+                if (w_tiled) tma_load_2d(w_s, &tm_w, &full, n0, k0);
+            }
+        }
+        if (!x_tiled) stage_x_cp_async<BM>(a, x_s, kc, k0, kn, row0, tid);
+        if (!w_tiled && n_loc > 0) stage_w_cp_async<BN, NK>(a, w_s, kc, k0, kn, n0, n_loc, tid);
+        if (k0 == 0) load_col_params<CW>(a, n0, lane, prm);   // in flight beside the operands
+        cp_async_wait_all();
+        if (chunk_bytes != 0) {
+            if (!mbar_wait(&full, phase, ctx, 1u)) abort_drain();   // ran out: let the copies land, finish with what is there
+            phase ^= 1u;
+        }
+        __syncthreads();
+        if (n_loc > 0) {
+            const int ks = ((kr + 31) >> 5) << 2;          // k per warp, a multiple of four
+            const int kb = wp * ks, ke = min(kb + ks, kr);
+#pragma unroll 2
+            for (int k = kb; k < ke; k += 4) {
+                float4 xv[BM];
+                float wv[CW][4];
+#pragma unroll
+                for (int r = 0; r < BM; ++r) xv[r] = *reinterpret_cast<const float4 *>(x_s + r * kc + k);
+#pragma unroll
+                for (int c = 0; c < CW; ++c)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        wv[c][j] = NK ? w_s[(lane + 32 * c) * (kc + 1) + k + j] : w_s[(k + j) * BN + lane + 32 * c];
+#pragma unroll
+                for (int r = 0; r < BM; ++r)
+#pragma unroll
+                    for (int c = 0; c < CW; ++c) {
+                        float s = acc[r][c];
+                        s = fmaf(xv[r].x, wv[c][0], s);
+                        s = fmaf(xv[r].y, wv[c][1], s);
+                        s = fmaf(xv[r].z, wv[c][2], s);
+                        s = fmaf(xv[r].w, wv[c][3], s);
+                        acc[r][c] = s;
+                    }
+            }
+        }
+    }
+
+    // ---- the eight warps' partial sums -> thread (warp = row, lane = column)
+#pragma unroll
+    for (int r = 0; r < BM; ++r)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) red[(wp * BM + r) * BN + lane + 32 * c] = acc[r][c];
+    __syncthreads();
+    float v[1][CW];
+#pragma unroll
+    for (int c = 0; c < CW; ++c) {
+        float part[8];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) part[w] = red[(w * BM + wp) * BN + lane + 32 * c];
+        v[0][c] = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+    }
+    epilogue_reduce_store<1, CW>(a, v, prm, stat, row0, n0, n_loc, lane, wp, cn);
+}
+
+// ---- problems that fill the chip: every thread walks all of k ---------------------------------------
+// RPT rows and CW columns per thread: the CTA tile is (8 RPT) x (32 CW).  NK: w is [N,K].
 template <int RPT, int CW, bool NK>
-cudaError_t launch_one(const Fp32ChainArgs &a, int cn, cudaStream_t stream)
+__global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, const int kc)
 {
     constexpr int BM = 8 * RPT, BN = 32 * CW;
-    int kc = (SMEM_FLOATS_MAX / (BM + BN + 1)) & ~3;
-    const int k4 = (a.K + 3) & ~3;
-    if (kc > k4) kc = k4;
-    const size_t smem = sizeof(float) * ((size_t)BM * kc + (NK ? (size_t)BN * (kc + 1) : (size_t)kc * BN));
+    extern __shared__ __align__(16) float smem[];
+    __shared__ float2 stat[MAX_BM];        // this CTA's per-row pair, read by the whole cluster
+    float *x_s = smem;                     // [BM][kc]
+    float *w_s = x_s + BM * kc;            // [kc][BN], or [BN][kc + 1] for NK (odd pitch: no bank conflicts)
+
+    const int tid = threadIdx.x, lane = tid & 31, rg = tid >> 5;
+    const int cn = (int)cluster_nctas(), rank = (int)cluster_ctarank();
+    const long long row0 = (long long)((int)blockIdx.x / cn) * BM;
+    const int n0 = rank * BN;
+    const int n_loc = min(max(a.N - n0, 0), BN);      // columns this CTA owns (0 for a padding rank)
+    pdl_wait();
+
+    float acc[RPT][CW][4];
+#pragma unroll
+    for (int i = 0; i < RPT; ++i)
+#pragma unroll
+        for (int c = 0; c < CW; ++c)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][c][j] = 0.0f;
+    ColParams<CW> prm;
+    load_col_params<CW>(a, n0, lane, prm);
+
+    for (int k0 = 0; k0 < a.K; k0 += kc) {
+        const int kn = min(kc, a.K - k0);
+        __syncthreads();                                         // the previous chunk has been consumed
+        stage_x_cp_async<BM>(a, x_s, kc, k0, kn, row0, tid);
+        if (n_loc > 0) stage_w_cp_async<BN, NK>(a, w_s, kc, k0, kn, n0, n_loc, tid);
+        cp_async_wait_all();
+        __syncthreads();
+        if (n_loc > 0) {
+            // four k at a time: one 16-byte broadcast load of x per row, four column loads of w, and four
+            // independent accumulators per output (k = 0, 1, 2, 3 mod 4) so that consecutive FMAs do not wait
+            // for one another; the tail of a chunk that is not a multiple of four reads the zeros staged above
+#pragma unroll 2
+            for (int k = 0; k < kn; k += 4) {
+                float4 xv[RPT];
+                float wv[CW][4];
+#pragma unroll
+                for (int i = 0; i < RPT; ++i) xv[i] = *reinterpret_cast<const float4 *>(x_s + (rg + 8 * i) * kc + k);
+#pragma unroll
+                for (int c = 0; c < CW; ++c)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        wv[c][j] = NK ? w_s[(lane + 32 * c) * (kc + 1) + k + j] : w_s[(k + j) * BN + lane + 32 * c];
+#pragma unroll
+                for (int i = 0; i < RPT; ++i)
+#pragma unroll
+                    for (int c = 0; c < CW; ++c) {
+                        acc[i][c][0] = fmaf(xv[i].x, wv[c][0], acc[i][c][0]);
+                        acc[i][c][1] = fmaf(xv[i].y, wv[c][1], acc[i][c][1]);
+                        acc[i][c][2] = fmaf(xv[i].z, wv[c][2], acc[i][c][2]);
+                        acc[i][c][3] = fmaf(xv[i].w, wv[c][3], acc[i][c][3]);
+                    }
+            }
+        }
+    }
+
+    float v[RPT][CW];
+#pragma unroll
+    for (int i = 0; i < RPT; ++i)
+#pragma unroll
+        for (int c = 0; c < CW; ++c) v[i][c] = (acc[i][c][0] + acc[i][c][1]) + (acc[i][c][2] + acc[i][c][3]);
+    epilogue_reduce_store<RPT, CW>(a, v, prm, stat, row0, n0, n_loc, lane, rg, cn);
+}
+
+template <typename Kernel, typename... Extra>
+cudaError_t launch_clusters(Kernel kern, const Fp32ChainArgs &a, int bm, int cn, size_t smem, int kc, cudaStream_t stream,
+                            Extra... extra)
+{
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(cn * ((a.M + BM - 1) / BM)));
+    cfg.gridDim = dim3((unsigned)(cn * ((a.M + bm - 1) / bm)));
     cfg.blockDim = dim3(FT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -292,29 +441,59 @@ cudaError_t launch_one(const Fp32ChainArgs &a, int cn, cudaStream_t stream)
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.pdl != 0 ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, fp32_chain_kernel<RPT, CW, NK>, a, kc);
+    return cudaLaunchKernelEx(&cfg, kern, a, kc, extra...);
 }
 
-template <int RPT, int CW>
-cudaError_t launch_nk(const Fp32ChainArgs &a, int cn, cudaStream_t stream)
+// chunk length along k: what fits the shared memory beside the other operand, a multiple of four
+int chunk_k(int K, int rpt, int cw, bool tiled)
 {
-    return a.w_is_nk ? launch_one<RPT, CW, true>(a, cn, stream) : launch_one<RPT, CW, false>(a, cn, stream);
-}
-
-template <int RPT>
-cudaError_t launch_cw(const Fp32ChainArgs &a, int cw, int cn, cudaStream_t stream)
-{
-    switch (cw) {
-    case 1:  return launch_nk<RPT, 1>(a, cn, stream);
-    case 2:  return launch_nk<RPT, 2>(a, cn, stream);
-    default: return launch_nk<RPT, 4>(a, cn, stream);
-    }
+    const int bm = 8 * rpt, bn = 32 * cw;
+    int kc = rpt == 1 ? ((SMEM_FLOATS_MAX - 8 * SPLITK_BM * bn - bn) / (bm + bn)) & ~3
+                      : (SMEM_FLOATS_MAX / (bm + bn + 1)) & ~3;
+    if (tiled && kc > 256) kc = 256;                       // a tensor-map box has at most 256 elements per dimension
+    const int k4 = (K + 3) & ~3;
+    return kc > k4 ? k4 : kc;
 }
 
 template <int RPT, int CW, bool NK>
-cudaError_t setup_one()
+cudaError_t launch_one(const Fp32ChainArgs &a, const Fp32ChainPlan &p, cudaStream_t stream)
 {
-    return cudaFuncSetAttribute(fp32_chain_kernel<RPT, CW, NK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    constexpr int BM = 8 * RPT, BN = 32 * CW;
+    const size_t smem = sizeof(float) * ((size_t)BM * p.kc + (NK ? (size_t)BN * (p.kc + 1) : (size_t)p.kc * BN));
+    return launch_clusters(fp32_chain_kernel<RPT, CW, NK>, a, BM, p.cn, smem, p.kc, stream);
+}
+
+template <int CW, bool NK>
+cudaError_t launch_splitk(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const CUtensorMap &tm_x, const CUtensorMap &tm_w,
+                          cudaStream_t stream)
+{
+    constexpr int BM = SPLITK_BM, BN = 32 * CW;
+    const size_t smem = 128 + sizeof(float) * ((size_t)BM * p.kc + (NK ? (size_t)BN * (p.kc + 1) : (size_t)p.kc * BN) +
+                                               (size_t)8 * BM * BN);
+    return launch_clusters(fp32_chain_splitk_kernel<CW, NK>, a, BM, p.cn, smem, p.kc, stream, p.tma_x, p.tma_w, tm_x, tm_w);
+}
+
+template <int RPT>
+cudaError_t launch_cw(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const CUtensorMap &tm_x, const CUtensorMap &tm_w,
+                      cudaStream_t stream)
+{
+#define PIKE_FP32_LAUNCH(C)                                                                                          \
+    if constexpr (RPT == 1)                                                                                          \
+        return a.w_is_nk ? launch_splitk<C, true>(a, p, tm_x, tm_w, stream) : launch_splitk<C, false>(a, p, tm_x, tm_w, stream); \
+    else                                                                                                             \
+        return a.w_is_nk ? launch_one<RPT, C, true>(a, p, stream) : launch_one<RPT, C, false>(a, p, stream);
+    switch (p.cw) {
+    case 1:  PIKE_FP32_LAUNCH(1)
+    case 2:  PIKE_FP32_LAUNCH(2)
+    default: PIKE_FP32_LAUNCH(4)
+    }
+#undef PIKE_FP32_LAUNCH
+}
+
+template <typename Kernel>
+cudaError_t raise_smem_limit(Kernel kern)
+{
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)(sizeof(float) * (SMEM_FLOATS_MAX + 8 * 32 * 4)));
 }
 
@@ -323,28 +502,54 @@ cudaError_t setup_one()
 cudaError_t setup_fp32_chain()
 {
     cudaError_t e = cudaSuccess;
-#define PIKE_FP32_SETUP(R, C)                                                      \
-    if (e == cudaSuccess) e = setup_one<R, C, false>();                            \
-    if (e == cudaSuccess) e = setup_one<R, C, true>();
-    PIKE_FP32_SETUP(1, 1) PIKE_FP32_SETUP(1, 2) PIKE_FP32_SETUP(1, 4)
+#define PIKE_FP32_SETUP(R, C)                                                                     \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, C, false>);                  \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, C, true>);
     PIKE_FP32_SETUP(2, 1) PIKE_FP32_SETUP(2, 2) PIKE_FP32_SETUP(2, 4)
     PIKE_FP32_SETUP(4, 1) PIKE_FP32_SETUP(4, 2) PIKE_FP32_SETUP(4, 4)
+#undef PIKE_FP32_SETUP
+#define PIKE_FP32_SETUP(C)                                                                        \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_splitk_kernel<C, false>);              \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_splitk_kernel<C, true>);
+    PIKE_FP32_SETUP(1) PIKE_FP32_SETUP(2) PIKE_FP32_SETUP(4)
 #undef PIKE_FP32_SETUP
     return e;
 }
 
-cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, int num_sms, cudaStream_t stream)
+Fp32ChainPlan plan_fp32_chain(const Fp32ChainArgs &a, int num_sms)
+{
+    Fp32ChainPlan p = {};
+    // columns per CTA: the narrowest slice that keeps the cluster within 8 CTAs (N <= 1024 checked by the caller)
+    p.cw = a.N <= 256 ? 1 : (a.N <= 512 ? 2 : 4);
+    const int need = (a.N + 32 * p.cw - 1) / (32 * p.cw);
+    p.cn = 1;
+    while (p.cn < need) p.cn *= 2;                      // power of two; ranks past N own no columns
+    // rows per CTA: small problems spread over as many SMs as they can fill, large ones amortise W over more rows
+    if ((long long)p.cn * ((a.M + 7) / 8) <= 2ll * num_sms) p.rpt = 1;
+    else if ((long long)p.cn * ((a.M + 15) / 16) <= 4ll * num_sms) p.rpt = 2;
+    else p.rpt = 4;
+    if (p.rpt == 1) {   // tensor maps want 16-byte aligned bases and row pitches
+        p.tma_x = (a.ldx & 3) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
+        p.tma_w = !a.w_is_nk && (a.ldw & 3) == 0 && (reinterpret_cast<uintptr_t>(a.w) & 15) == 0;
+    }
+    p.kc = chunk_k(a.K, p.rpt, p.cw, p.tma_x || p.tma_w);
+    p.x_box[0] = (uint32_t)p.kc;      p.x_box[1] = SPLITK_BM;
+    p.w_box[0] = (uint32_t)(32 * p.cw); p.w_box[1] = (uint32_t)p.kc;
+    return p;
+}
+
+cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const CUtensorMap *tm_x, const CUtensorMap *tm_w,
+                              cudaStream_t stream)
 {
     if (a.M <= 0) return cudaSuccess;
-    // columns per CTA: the narrowest slice that keeps the cluster within 8 CTAs (N <= 1024 checked by the caller)
-    const int cw = a.N <= 256 ? 1 : (a.N <= 512 ? 2 : 4);
-    const int need = (a.N + 32 * cw - 1) / (32 * cw);
-    int cn = 1;
-    while (cn < need) cn *= 2;                          // power of two; ranks past N own no columns
-    // rows per CTA: small problems spread over as many SMs as they can fill, large ones amortise W over more rows
-    if ((long long)cn * ((a.M + 7) / 8) <= 2ll * num_sms) return launch_cw<1>(a, cw, cn, stream);
-    if ((long long)cn * ((a.M + 15) / 16) <= 4ll * num_sms) return launch_cw<2>(a, cw, cn, stream);
-    return launch_cw<4>(a, cw, cn, stream);
+    CUtensorMap none;
+    memset(&none, 0, sizeof(none));
+    const CUtensorMap &mx = (p.tma_x && tm_x != nullptr) ? *tm_x : none, &mw = (p.tma_w && tm_w != nullptr) ? *tm_w : none;
+    switch (p.rpt) {
+    case 1:  return launch_cw<1>(a, p, mx, mw, stream);
+    case 2:  return launch_cw<2>(a, p, mx, mw, stream);
+    default: return launch_cw<4>(a, p, mx, mw, stream);
+    }
 }
 
 }  // namespace pike

@@ -34,6 +34,7 @@ enum : uint32_t {
     KID_GEMM = 1,
     KID_ATTN = 2,
     KID_LAYERNORM = 3,
+    KID_FP32_CHAIN = 4,
 };
 
 // ---- fp32 CUDA-core chain: out = reduce(scale*act(x@w+b)+res) ------------------
@@ -46,8 +47,23 @@ struct Fp32ChainArgs {
     int act, reduce;
     float scale, eps;
     int pdl;        // launch with programmatic stream serialisation (see launch_kernel)
+    unsigned int *status;            // device status word and the bound of the kernel's wait for its tiled copies
+    unsigned long long limit_ns;
+    int test_withhold_loads;         // test hook: the tiled copies are not issued, so the wait for them runs out
 };
-cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, int num_sms, cudaStream_t stream);
+// How a problem is laid over the chip: rows per thread (1 = the split-k kernel for small problems, 8 rows per
+// cluster; 2, 4 = 16 or 32 rows), 32 cw columns per CTA, cn CTAs per cluster, kc = k per staged chunk.  tma_x / tma_w:
+// the split-k kernel fetches that operand through a tensor map (fp32, no swizzle, zero fill) with the box given
+// here - x as {K, M} with box {kc, 8}, w [K,N] as {N, K} with box {32 cw, kc}; the caller encodes the maps, or
+// clears the flag to fall back to per-thread copies.
+struct Fp32ChainPlan {
+    int rpt, cw, cn, kc;
+    int tma_x, tma_w;
+    uint32_t x_box[2], w_box[2];
+};
+Fp32ChainPlan plan_fp32_chain(const Fp32ChainArgs &a, int num_sms);
+cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, const Fp32ChainPlan &plan, const CUtensorMap *tm_x,
+                              const CUtensorMap *tm_w, cudaStream_t stream);
 
 // ---- once per device (with that device current): function attributes and launch limits ------------
 // Each setup_* raises the dynamic shared-memory limit of its kernels on the current device, so that

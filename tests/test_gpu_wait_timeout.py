@@ -35,3 +35,30 @@ def test_a_wait_that_nothing_satisfies_times_out_and_is_reported():
     torch.cuda.synchronize()
     check_bf16(got, O.linear_epilogue(c["x"], c["w"]), what="GEMM after a reported timeout")
     assert P.pike_get_last_device_status() == (0, 0)
+
+
+def test_the_fp32_chain_reports_bulk_copies_that_never_land():
+    """The small-problem fp32 kernel stages aligned operands with bulk copies on one mbarrier; with the copies
+    withheld its bounded wait runs out, the cluster still meets at its barriers and exits, and the next call is right."""
+    import paper_2511_16964_b200 as P
+    F32 = torch.float32
+    c = G.config1()
+    args = [dev(c[k], F32) for k in ("x", "w", "b")] + [None, dev(c["gamma"], F32), dev(c["beta"], F32)]
+    kw = dict(act="gelu_erf", reduce="layernorm", eps=c["eps"])
+    assert P.pike_get_last_device_status() == (0, 0)
+    P.pike_set_wait_limit_ns(2_000_000)
+    try:
+        P.pike_test_withhold_loads()
+        P.pike_linear_epilogue(*args, **kw)
+        torch.cuda.synchronize()
+        status, where = P.pike_get_last_device_status()
+        assert status == 10                          # PIKE_ERR_TIMEOUT
+        assert where >> 16 == 4 and where & 0xFFFF == 1          # fp32 chain, its one barrier
+        assert P.pike_get_last_device_status() == (0, 0)
+    finally:
+        P.pike_set_wait_limit_ns(0)
+    got = host64(P.pike_linear_epilogue(*args, **kw))
+    torch.cuda.synchronize()
+    want = O.linear_epilogue(c["x"], c["w"], c["b"], None, c["gamma"], c["beta"], **kw)
+    assert np.abs(got - want).max() <= 1e-4
+    assert P.pike_get_last_device_status() == (0, 0)
