@@ -8,10 +8,11 @@
 // row block instead of once per CTA-row as a one-CTA-per-row layout would have it, and the
 // whole problem spreads over many SMs even when M is small.
 // Two kernels share the staging, the epilogue and the reduction:
-//  - fp32_chain_splitk_kernel (BM = 8; small problems, whose time is a chain of latencies): the eight
-//    warps split k, every thread accumulates all 8 rows of its columns over its warp's k slice (8 FMAs per
-//    shared-memory word of W instead of one), and the warps' partial sums meet in shared memory.  Operands
-//    arrive as row-wise bulk copies on one mbarrier where the addresses allow it.
+//  - fp32_chain_splitk_kernel (BM = 8; small problems, whose time is a chain of latencies): groups of
+//    threads split k, every thread accumulates a 4 x 4 register tile over its k slice (16 FMAs per 16-byte
+//    shared-memory load of either operand: the shared-memory pipe, not the FMA pipe, bounds a tile this small),
+//    and the slices' partial sums meet in shared memory.  Operands arrive as two tiled copies on one mbarrier
+//    where the tensors allow a tensor map.
 //  - fp32_chain_kernel (BM = 16 or 32; problems that fill the chip): thread (lane, warp) accumulates
 //    columns lane + 32c of rows warp + 8i over all of k.
 // The LayerNorm / softmax reduction over N never leaves the cluster: every warp reduces its rows
@@ -167,18 +168,25 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
         for (int i = 0; i < RPT; ++i) {
             float s0, s1;
             if (a.reduce == 1) {                       // LayerNorm: (mean, sum of squared deviations) of n_loc values
-                float s = 0.0f;
-#pragma unroll
-                for (int c = 0; c < CW; ++c) s += (lane + 32 * c < n_loc) ? v[i][c] : 0.0f;
-                const float mean = n_loc > 0 ? warp_sum_f(s) / (float)n_loc : 0.0f;
-                float d2 = 0.0f;
+                // one pass over values shifted by the CTA's first column (the shift keeps sum d^2 - (sum d)^2 / n
+                // free of the cancellation a plain sum of squares suffers when the mean dwarfs the spread); the two
+                // sums travel through the shuffles side by side
+                const float v0 = __shfl_sync(0xffffffffu, v[i][0], 0);
+                float sd = 0.0f, sq = 0.0f;
 #pragma unroll
                 for (int c = 0; c < CW; ++c) {
-                    const float d = v[i][c] - mean;
-                    d2 += (lane + 32 * c < n_loc) ? d * d : 0.0f;
+                    const float d = (lane + 32 * c < n_loc) ? v[i][c] - v0 : 0.0f;
+                    sd += d;
+                    sq = fmaf(d, d, sq);
                 }
-                s0 = mean;
-                s1 = warp_sum_f(d2);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    sd += __shfl_xor_sync(0xffffffffu, sd, o);
+                    sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                }
+                const float inv = n_loc > 0 ? 1.0f / (float)n_loc : 0.0f;
+                s0 = n_loc > 0 ? v0 + sd * inv : 0.0f;
+                s1 = fmaxf(sq - sd * sd * inv, 0.0f);
             } else {                                   // softmax: (max, sum exp(v - max))
                 float m = -INFINITY;
 #pragma unroll
@@ -193,27 +201,40 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
             if (lane == 0) stat[rg + 8 * i] = make_float2(s0, s1);
         }
         cluster_sync_all();                            // every rank's pairs are visible cluster-wide
-        // ---- merge the ranks' pairs: lane r fetches rank r's pair, the merge is a warp reduction over the
-        //      lanes (the same tree in every CTA, so the whole cluster computes bit-identical statistics).
-        //      LayerNorm pools the ranks' moments about the pooled mean (deviations of means: no E[x^2] - E[x]^2
-        //      cancellation).
-        const float nr = lane < cn ? (float)min(max(a.N - lane * BN, 0), BN) : 0.0f;   // columns of rank `lane`
+        // ---- merge the ranks' pairs: lane l fetches the pair of rank l mod 8, so every group of eight lanes holds
+        //      all ranks and three shuffle steps give every lane the merged value (the same tree in every CTA, so
+        //      the whole cluster computes bit-identical statistics).  LayerNorm pools the ranks' moments about
+        //      rank 0's mean (deviations of means: no E[x^2] - E[x]^2 cancellation), three sums side by side.
+        const int rk = lane & 7;
+        const float nr = rk < cn ? (float)min(max(a.N - rk * BN, 0), BN) : 0.0f;       // columns of rank rk
         const float inv_n = 1.0f / (float)a.N;
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
             float2 mine = make_float2(0.0f, 0.0f);
-            if (lane < cn) mine = ld_shared_cluster_f32x2(mapa_shared(smem_u32(&stat[rg + 8 * i]), (uint32_t)lane));
+            if (rk < cn) mine = ld_shared_cluster_f32x2(mapa_shared(smem_u32(&stat[rg + 8 * i]), (uint32_t)rk));
             if (a.reduce == 1) {
-                const float mean = warp_sum_f(nr * mine.x) * inv_n;
-                const float d = mine.x - mean;
-                const float m2 = warp_sum_f(mine.y + nr * d * d);
+                const float mean0 = __shfl_sync(0xffffffffu, mine.x, 0);       // every lane takes part in the shuffle
+                const float e = nr > 0.0f ? mine.x - mean0 : 0.0f;
+                float sa = nr * e, sb = nr * e * e, sc = mine.y;
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) {
+                    sa += __shfl_xor_sync(0xffffffffu, sa, o);
+                    sb += __shfl_xor_sync(0xffffffffu, sb, o);
+                    sc += __shfl_xor_sync(0xffffffffu, sc, o);
+                }
+                const float mean = mean0 + sa * inv_n;
+                const float m2 = fmaxf(sc + sb - sa * sa * inv_n, 0.0f);
                 const float rstd = rsqrtf(m2 * inv_n + a.eps);
 #pragma unroll
                 for (int c = 0; c < CW; ++c) v[i][c] = (v[i][c] - mean) * rstd * p.gamma[c] + p.beta[c];
             } else {
                 const bool has = nr > 0.0f && mine.y > 0.0f;
-                const float m = warp_max_f(has ? mine.x : -INFINITY);
-                const float l = warp_sum_f(has ? mine.y * expf(mine.x - m) : 0.0f);
+                float m = has ? mine.x : -INFINITY;
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+                float l = has ? mine.y * expf(mine.x - m) : 0.0f;
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
                 const float inv = 1.0f / l;
 #pragma unroll
                 for (int c = 0; c < CW; ++c) v[i][c] = expf(v[i][c] - m) * inv;
@@ -238,9 +259,11 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
 }
 
 // ---- small problems: the warps split k ------------------------------------------------------------
-// CTA tile 8 x (32 CW).  Warp w accumulates ALL 8 rows of columns lane + 32c over its eighth of every staged
-// k chunk (k ascending), so a word of W read from shared memory feeds 8 FMAs and a 16-byte broadcast of x
-// feeds 4 CW; the eight partial sums per output meet in shared memory and are added in a fixed tree.
+// CTA tile 8 x (32 CW).  A thread accumulates 4 rows x 4 adjacent columns over one of 16 / CW slices of every
+// staged k chunk (k ascending): per four k it issues four 16-byte loads of x and four of W for 64 FMAs (one
+// column and 8 rows per thread, measured first, spent 3,000 cycles in this loop at 128 x 256 x 256 against 2,000
+// for everything else: a 16-byte load whose lanes all read one address still costs the pipe as much as one that
+// reads 512 bytes).  The slices' partial sums meet in shared memory and are added in a fixed tree.
 // Staging: where the tensors allow a tensor map (16-byte aligned base and row pitch; W as [K,N]) ONE thread
 // fetches the chunk's x rows and W slice as two tiled copies completing on one mbarrier (bounded wait); rows,
 // columns and k past the tensors arrive as zeros.  Otherwise the per-thread asynchronous copies above.
@@ -260,7 +283,7 @@ __global__ void __launch_bounds__(FT) fp32_chain_splitk_kernel(const Fp32ChainAr
     // tiled copies want 128-byte aligned destinations: x_s is, and w_s follows it by 32 kc bytes (kc a multiple of 4)
     float *x_s = reinterpret_cast<float *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));   // [BM][kc]
     float *w_s = x_s + BM * kc;                            // [kc][BN], or [BN][kc + 1] for NK
-    float *red = w_s + (NK ? BN * (kc + 1) : kc * BN);     // [8 warps][BM][BN]
+    float *red = w_s + (((NK ? BN * (kc + 1) : kc * BN) + 3) & ~3);   // [16 / CW k slices][BM][BN], 16-byte aligned
 
     const int tid = threadIdx.x, lane = tid & 31, wp = tid >> 5;
     const int cn = (int)cluster_nctas(), rank = (int)cluster_ctarank();
@@ -280,11 +303,16 @@ __global__ void __launch_bounds__(FT) fp32_chain_splitk_kernel(const Fp32ChainAr
     pdl_wait();
     const WaitCtx ctx{a.status, &abort_word, a.limit_ns, KID_FP32_CHAIN};
 
-    float acc[BM][CW];
+    // thread tile: 4 rows x 4 adjacent columns; 8 CW column groups x 2 row groups cover the CTA tile, and
+    // NS = 16 / CW groups of such threads split k.  Lanes: column group, then the low part of the k slice; warps:
+    // row group, then the high part (so a warp's x loads touch one row group and distinct banks).
+    constexpr int CG = 8 * CW, NS = 16 / CW, S_LO = 32 / CG;
+    const int cg = lane % CG, rgp = wp & 1, slice = (wp >> 1) * S_LO + lane / CG;
+    float acc[4][4];
 #pragma unroll
-    for (int r = 0; r < BM; ++r)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int c = 0; c < CW; ++c) acc[r][c] = 0.0f;
+        for (int c = 0; c < 4; ++c) acc[i][c] = 0.0f;
     ColParams<CW> prm;
 
     uint32_t phase = 0;
@@ -309,47 +337,57 @@ __global__ void __launch_bounds__(FT) fp32_chain_splitk_kernel(const Fp32ChainAr
         }
         __syncthreads();
         if (n_loc > 0) {
-            const int ks = ((kr + 31) >> 5) << 2;          // k per warp, a multiple of four
-            const int kb = wp * ks, ke = min(kb + ks, kr);
+            const int ks = (((kr + NS - 1) / NS) + 3) & ~3;          // k per slice, a multiple of four
+            const int kb = slice * ks, ke = min(kb + ks, kr);
+            const float *xp = x_s + (rgp * 4) * kc;
 #pragma unroll 2
             for (int k = kb; k < ke; k += 4) {
-                float4 xv[BM];
-                float wv[CW][4];
+                float4 xv[4];
+                float wv[4][4];                                        // [k offset][column]
 #pragma unroll
-                for (int r = 0; r < BM; ++r) xv[r] = *reinterpret_cast<const float4 *>(x_s + r * kc + k);
+                for (int i = 0; i < 4; ++i) xv[i] = *reinterpret_cast<const float4 *>(xp + i * kc + k);
 #pragma unroll
-                for (int c = 0; c < CW; ++c)
+                for (int j = 0; j < 4; ++j) {
+                    if constexpr (NK) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        wv[c][j] = NK ? w_s[(lane + 32 * c) * (kc + 1) + k + j] : w_s[(k + j) * BN + lane + 32 * c];
+                        for (int c = 0; c < 4; ++c) wv[j][c] = w_s[(4 * cg + c) * (kc + 1) + k + j];
+                    } else {
+                        const float4 t = *reinterpret_cast<const float4 *>(w_s + (k + j) * BN + 4 * cg);
+                        wv[j][0] = t.x; wv[j][1] = t.y; wv[j][2] = t.z; wv[j][3] = t.w;
+                    }
+                }
 #pragma unroll
-                for (int r = 0; r < BM; ++r)
+                for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int c = 0; c < CW; ++c) {
-                        float s = acc[r][c];
-                        s = fmaf(xv[r].x, wv[c][0], s);
-                        s = fmaf(xv[r].y, wv[c][1], s);
-                        s = fmaf(xv[r].z, wv[c][2], s);
-                        s = fmaf(xv[r].w, wv[c][3], s);
-                        acc[r][c] = s;
+                    for (int c = 0; c < 4; ++c) {
+                        float t = acc[i][c];
+                        t = fmaf(xv[i].x, wv[0][c], t);
+                        t = fmaf(xv[i].y, wv[1][c], t);
+                        t = fmaf(xv[i].z, wv[2][c], t);
+                        t = fmaf(xv[i].w, wv[3][c], t);
+                        acc[i][c] = t;
                     }
             }
         }
     }
 
-    // ---- the eight warps' partial sums -> thread (warp = row, lane = column)
+    // ---- the slices' partial sums -> thread (warp = row, lane = column), added in a fixed tree
 #pragma unroll
-    for (int r = 0; r < BM; ++r)
-#pragma unroll
-        for (int c = 0; c < CW; ++c) red[(wp * BM + r) * BN + lane + 32 * c] = acc[r][c];
+    for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<float4 *>(red + (slice * BM + rgp * 4 + i) * BN + 4 * cg) =
+            make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
     __syncthreads();
     float v[1][CW];
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-        float part[8];
+        float part[NS];
 #pragma unroll
-        for (int w = 0; w < 8; ++w) part[w] = red[(w * BM + wp) * BN + lane + 32 * c];
-        v[0][c] = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+        for (int w = 0; w < NS; ++w) part[w] = red[(w * BM + wp) * BN + lane + 32 * c];
+#pragma unroll
+        for (int step = 1; step < NS; step *= 2)
+#pragma unroll
+            for (int w = 0; w + step < NS; w += 2 * step) part[w] += part[w + step];
+        v[0][c] = part[0];
     }
     epilogue_reduce_store<1, CW>(a, v, prm, stat, row0, n0, n_loc, lane, wp, cn);
 }
@@ -448,7 +486,7 @@ cudaError_t launch_clusters(Kernel kern, const Fp32ChainArgs &a, int bm, int cn,
 int chunk_k(int K, int rpt, int cw, bool tiled)
 {
     const int bm = 8 * rpt, bn = 32 * cw;
-    int kc = rpt == 1 ? ((SMEM_FLOATS_MAX - 8 * SPLITK_BM * bn - bn) / (bm + bn)) & ~3
+    int kc = rpt == 1 ? ((SMEM_FLOATS_MAX - 16 * SPLITK_BM * 32 - bn - 4) / (bm + bn)) & ~3
                       : (SMEM_FLOATS_MAX / (bm + bn + 1)) & ~3;
     if (tiled && kc > 256) kc = 256;                       // a tensor-map box has at most 256 elements per dimension
     const int k4 = (K + 3) & ~3;
@@ -468,8 +506,8 @@ cudaError_t launch_splitk(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const 
                           cudaStream_t stream)
 {
     constexpr int BM = SPLITK_BM, BN = 32 * CW;
-    const size_t smem = 128 + sizeof(float) * ((size_t)BM * p.kc + (NK ? (size_t)BN * (p.kc + 1) : (size_t)p.kc * BN) +
-                                               (size_t)8 * BM * BN);
+    const size_t smem = 128 + sizeof(float) * ((size_t)BM * p.kc + (NK ? (size_t)BN * (p.kc + 1) + 3 : (size_t)p.kc * BN) +
+                                               (size_t)16 * BM * 32);
     return launch_clusters(fp32_chain_splitk_kernel<CW, NK>, a, BM, p.cn, smem, p.kc, stream, p.tma_x, p.tma_w, tm_x, tm_w);
 }
 
