@@ -814,11 +814,11 @@ def host_call_overhead(P, torch, suite, calls=400):
     for name, args_, e, o, n in (("pike_linear_epilogue_fp32_128x256x256", a1, e1, o1, calls),
                                  ("pike_linear_epilogue_bf16_4096^3", a2, e2, o2, 60)):
         for _ in range(3):
-            lib.pike_linear_epilogue(h, *args_, ctypes.byref(e), o, None, 0, stream)
+            lib.pike_linear_epilogue(h, *args_, e, o, None, 0, stream)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         for _ in range(n):
-            lib.pike_linear_epilogue(h, *args_, ctypes.byref(e), o, None, 0, stream)
+            lib.pike_linear_epilogue(h, *args_, e, o, None, 0, stream)
         t1 = time.perf_counter()
         torch.cuda.synchronize()
         res[name] = (t1 - t0) / n * 1e6

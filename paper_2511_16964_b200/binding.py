@@ -67,6 +67,8 @@ def library_path() -> str:
 def load_library() -> ctypes.CDLL:
     """dlopen libpike.so and declare the prototypes.  Raises if it was not built."""
     global _lib
+    if _lib is not None:
+        return _lib
     with _lock:
         if _lib is None:
             if not os.path.exists(_LIB_PATH):
@@ -112,8 +114,7 @@ def pike_status_string(code: int) -> str:
 
 def _handle(device: torch.device) -> ctypes.c_void_p:
     idx = device.index if device.index is not None else torch.cuda.current_device()
-    with _lock:
-        h = _handles.get(idx)
+    h = _handles.get(idx)
     if h is None:
         lib = load_library()
         h = ctypes.c_void_p()
@@ -125,46 +126,62 @@ def _handle(device: torch.device) -> ctypes.c_void_p:
     return h
 
 
+_DTYPE_CODE = {torch.float32: PIKE_F32, torch.bfloat16: PIKE_BF16, torch.float16: PIKE_F16}
+_I64x4 = ctypes.c_int64 * 4
+# Descriptors already built, keyed by everything they hold: a model calls the same chains on the same buffers over
+# and over, and building a ctypes structure costs more host time than the small chains' kernels take.
+_desc_cache: dict = {}
+_epi_cache: dict = {}
+_ws_bytes_cache: dict = {}
+_CACHE_LIMIT = 4096
+
+
 def _dtype_code(t: torch.Tensor) -> int:
-    if t.dtype == torch.float32:
-        return PIKE_F32
-    if t.dtype == torch.bfloat16:
-        return PIKE_BF16
-    if t.dtype == torch.float16:
-        return PIKE_F16
-    raise TypeError(f"unsupported dtype {t.dtype}")
+    try:
+        return _DTYPE_CODE[t.dtype]
+    except KeyError:
+        raise TypeError(f"unsupported dtype {t.dtype}") from None
 
 
 def _tensor(t):
     """torch CUDA tensor -> pike_tensor_t (by reference); None -> NULL."""
     if t is None:
         return None
+    shape, stride = t.shape, t.stride()
+    key = (t.data_ptr(), shape, stride, t.dtype)
+    ref = _desc_cache.get(key)
+    if ref is not None:
+        return ref
     if not t.is_cuda:
         raise ValueError("tensors must live in CUDA device memory")
-    d = pike_tensor_t()
-    d.data = t.data_ptr()
-    d.dtype = _dtype_code(t)
-    d.ndim = t.dim()
-    # torch leaves the stride of an extent-1 dimension arbitrary (a [1, K] view of a [K, 1] array keeps stride 1);
-    # the C ABI wants every outer stride to cover the dimensions inside it, so such strides are canonicalised here
-    inner = 1
-    for i in reversed(range(t.dim())):
-        d.shape[i] = t.shape[i]
-        d.stride[i] = t.stride(i) if t.shape[i] != 1 else max(inner, 1)
-        inner = max(inner, d.stride[i] * t.shape[i])
-    return ctypes.byref(d)
+    if len(shape) > 4:
+        raise ValueError("at most four dimensions")
+    if 1 in shape:
+        # torch leaves the stride of an extent-1 dimension arbitrary (a [1, K] view of a [K, 1] array keeps stride
+        # 1); the C ABI wants every outer stride to cover the dimensions inside it, so such strides are canonicalised
+        stride, inner = list(stride), 1
+        for i in reversed(range(len(shape))):
+            if shape[i] == 1:
+                stride[i] = max(inner, 1)
+            inner = max(inner, stride[i] * shape[i])
+    ref = ctypes.byref(pike_tensor_t(key[0], _dtype_code(t), len(shape), _I64x4(*shape), _I64x4(*stride)))
+    if len(_desc_cache) >= _CACHE_LIMIT:
+        _desc_cache.clear()
+    _desc_cache[key] = ref
+    return ref
 
 
-def _epilogue(act, scale, reduce, eps, out_dtype, flags) -> pike_epilogue_t:
-    e = pike_epilogue_t()
-    e.struct_size = ctypes.sizeof(pike_epilogue_t)
-    e.act = ACT[act]
-    e.scale = float(scale)
-    e.reduce = REDUCE[reduce]
-    e.eps = float(eps)
-    e.out_dtype = {torch.float32: PIKE_F32, torch.bfloat16: PIKE_BF16, torch.float16: PIKE_F16}[out_dtype]
-    e.flags = flags
-    return e
+def _epilogue(act, scale, reduce, eps, out_dtype, flags):
+    """The epilogue descriptor, by reference."""
+    key = (act, scale, reduce, eps, out_dtype, flags)
+    ref = _epi_cache.get(key)
+    if ref is None:
+        e = pike_epilogue_t(ctypes.sizeof(pike_epilogue_t), ACT[act], float(scale), REDUCE[reduce], float(eps),
+                            _DTYPE_CODE[out_dtype], flags)
+        if len(_epi_cache) >= _CACHE_LIMIT:
+            _epi_cache.clear()
+        ref = _epi_cache[key] = ctypes.byref(e)
+    return ref
 
 
 def _stream(stream) -> ctypes.c_void_p:
@@ -179,12 +196,23 @@ def _on(stream):
     return contextlib.nullcontext() if stream is None else torch.cuda.stream(stream)
 
 
-def _workspace(query, device, workspace, stream):
+def _workspace(query, device, workspace, stream, key=None):
     """(keep-alive, pointer, bytes) of the workspace: the caller's, or a temporary of the size `query()`
-    returns, allocated on `stream`.  A caller-supplied workspace is sized by the C side's own check."""
+    returns, allocated on `stream` (nothing when the chain needs none).  The size depends on the shapes, types and
+    flags in `key` only, so it is asked for once per key.  A caller-supplied workspace is sized by the C side's
+    own check."""
     if workspace is None:
+        need = _ws_bytes_cache.get(key) if key is not None else None
+        if need is None:
+            need = int(query())
+            if key is not None:
+                if len(_ws_bytes_cache) >= _CACHE_LIMIT:
+                    _ws_bytes_cache.clear()
+                _ws_bytes_cache[key] = need
+        if need == 0:
+            return None, None, 0
         with _on(stream):
-            workspace = torch.empty(max(int(query()), 256), dtype=torch.uint8, device=device)
+            workspace = torch.empty(need, dtype=torch.uint8, device=device)
     return workspace, ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
 
 
@@ -239,7 +267,7 @@ def pike_linear_epilogue_workspace(x, w, *, act="none", scale=1.0, reduce="none"
     e = _epilogue(act, scale, reduce, eps, out_dtype, (FLAG_W_IS_NK if w_is_nk else 0) | (FLAG_ONE_PASS if one_pass else 0))
     n = ctypes.c_size_t(0)
     _check(load_library().pike_linear_epilogue_workspace(_handle(x.device), _tensor(x), _tensor(w),
-                                                         ctypes.byref(e), ctypes.byref(n)),
+                                                         e, ctypes.byref(n)),
            "pike_linear_epilogue_workspace")
     return n.value
 
@@ -256,9 +284,10 @@ def pike_linear_epilogue(x, w, bias=None, residual=None, gamma=None, beta=None, 
     e = _epilogue(act, scale, reduce, eps, out_dtype, (FLAG_W_IS_NK if w_is_nk else 0) | (FLAG_ONE_PASS if one_pass else 0))
     ws, ws_ptr, ws_bytes = _workspace(
         lambda: pike_linear_epilogue_workspace(x, w, act=act, scale=scale, reduce=reduce, eps=eps, out_dtype=out_dtype,
-                                               w_is_nk=w_is_nk, one_pass=one_pass), x.device, workspace, stream)
+                                               w_is_nk=w_is_nk, one_pass=one_pass), x.device, workspace, stream,
+        ("linear", x.device, x.shape, w.shape, x.dtype, out_dtype, reduce, w_is_nk, one_pass))
     _check(load_library().pike_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
-                                               _tensor(residual), _tensor(gamma), _tensor(beta), ctypes.byref(e),
+                                               _tensor(residual), _tensor(gamma), _tensor(beta), e,
                                                _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
            "pike_linear_epilogue")
     return out
@@ -268,7 +297,7 @@ def pike_linear_softmax_shard_workspace(x, w, *, act="none", scale=1.0, w_is_nk=
     e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
     n = ctypes.c_size_t(0)
     _check(load_library().pike_linear_softmax_shard_workspace(_handle(x.device), _tensor(x), _tensor(w),
-                                                              ctypes.byref(e), ctypes.byref(n)),
+                                                              e, ctypes.byref(n)),
            "pike_linear_softmax_shard_workspace")
     return n.value
 
@@ -289,9 +318,9 @@ def pike_linear_softmax_shard_local(x, w, bias=None, *, act="none", scale=1.0, w
     e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
     ws, ws_ptr, ws_bytes = _workspace(
         lambda: pike_linear_softmax_shard_workspace(x, w, act=act, scale=scale, w_is_nk=w_is_nk), x.device, workspace,
-        stream)
+        stream, ("shard", x.device, x.shape, w.shape, x.dtype, w_is_nk))
     _check(load_library().pike_linear_softmax_shard_local(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
-                                                          ctypes.byref(e), _tensor(out),
+                                                          e, _tensor(out),
                                                           ctypes.c_void_p(row_stats.data_ptr()), ws_ptr, ws_bytes,
                                                           _stream(stream)),
            "pike_linear_softmax_shard_local")
@@ -323,7 +352,7 @@ def pike_linear_softmax_noalloc(x, w, bias=None, *, out, act="none", scale=1.0, 
     streams must not overlap (they share one scratch array).  See include/pike.h."""
     e = _epilogue(act, scale, "softmax", 0.0, torch.float32, FLAG_W_IS_NK if w_is_nk else 0)
     _check(load_library().pike_linear_softmax_noalloc(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
-                                                      ctypes.byref(e), _tensor(out), _stream(stream)),
+                                                      e, _tensor(out), _stream(stream)),
            "pike_linear_softmax_noalloc")
     return out
 
@@ -331,7 +360,7 @@ def pike_linear_softmax_noalloc(x, w, bias=None, *, out, act="none", scale=1.0, 
 def pike_mlp_block_workspace(x, w1, *, act="gelu_tanh", eps=1e-5, w_is_nk=False) -> int:
     e = _epilogue(act, 1.0, "none", eps, x.dtype, FLAG_W_IS_NK if w_is_nk else 0)
     n = ctypes.c_size_t(0)
-    _check(load_library().pike_mlp_block_workspace(_handle(x.device), _tensor(x), _tensor(w1), ctypes.byref(e),
+    _check(load_library().pike_mlp_block_workspace(_handle(x.device), _tensor(x), _tensor(w1), e,
                                                    ctypes.byref(n)), "pike_mlp_block_workspace")
     return n.value
 
@@ -344,9 +373,9 @@ def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5,
             out = torch.empty_like(x)
     e = _epilogue(act, 1.0, "none", eps, x.dtype, FLAG_W_IS_NK if w_is_nk else 0)
     ws, ws_ptr, ws_bytes = _workspace(lambda: pike_mlp_block_workspace(x, w1, act=act, eps=eps, w_is_nk=w_is_nk),
-                                      x.device, workspace, stream)
+                                      x.device, workspace, stream, ("mlp", x.device, x.shape, w1.shape, x.dtype, w_is_nk))
     _check(load_library().pike_mlp_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta), _tensor(w1),
-                                         _tensor(b1), _tensor(w2), _tensor(b2), ctypes.byref(e), _tensor(out),
+                                         _tensor(b1), _tensor(w2), _tensor(b2), e, _tensor(out),
                                          ws_ptr, ws_bytes, _stream(stream)), "pike_mlp_block")
     return out
 
@@ -354,7 +383,7 @@ def pike_mlp_block(x, gamma, beta, w1, b1, w2, b2, *, act="gelu_tanh", eps=1e-5,
 def pike_attention_chain_workspace(q, *, scale, causal=True) -> int:
     e = _epilogue("none", scale, "none", 0.0, q.dtype, FLAG_CAUSAL if causal else 0)
     n = ctypes.c_size_t(0)
-    _check(load_library().pike_attention_chain_workspace(_handle(q.device), _tensor(q), ctypes.byref(e),
+    _check(load_library().pike_attention_chain_workspace(_handle(q.device), _tensor(q), e,
                                                          ctypes.byref(n)), "pike_attention_chain_workspace")
     return n.value
 
@@ -366,7 +395,7 @@ def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
             out = torch.empty_like(q)
     e = _epilogue("none", scale, "none", 0.0, q.dtype, FLAG_CAUSAL if causal else 0)
     _check(load_library().pike_attention_chain(_handle(q.device), _tensor(q), _tensor(k), _tensor(v),
-                                               ctypes.byref(e), _tensor(out), None, 0, _stream(stream)),
+                                               e, _tensor(out), None, 0, _stream(stream)),
            "pike_attention_chain")
     return out
 
@@ -374,7 +403,7 @@ def pike_attention_chain(q, k, v, *, scale, causal=True, out=None, stream=None):
 def pike_attention_block_workspace(x, *, scale, causal=True, eps=1e-5, w_is_nk=False) -> int:
     e = _epilogue("none", scale, "none", eps, x.dtype, (FLAG_CAUSAL if causal else 0) | (FLAG_W_IS_NK if w_is_nk else 0))
     n = ctypes.c_size_t(0)
-    _check(load_library().pike_attention_block_workspace(_handle(x.device), _tensor(x), ctypes.byref(e), ctypes.byref(n)),
+    _check(load_library().pike_attention_block_workspace(_handle(x.device), _tensor(x), e, ctypes.byref(n)),
            "pike_attention_block_workspace")
     return n.value
 
@@ -391,7 +420,7 @@ def pike_attention_block(x, gamma, beta, w_qkv, b_qkv, w_o, b_o, *, scale, causa
         workspace, stream)
     _check(load_library().pike_attention_block(_handle(x.device), _tensor(x), _tensor(gamma), _tensor(beta),
                                                _tensor(w_qkv), _tensor(b_qkv), _tensor(w_o), _tensor(b_o),
-                                               ctypes.byref(e), _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
+                                               e, _tensor(out), ws_ptr, ws_bytes, _stream(stream)),
            "pike_attention_block")
     return out
 
@@ -410,6 +439,6 @@ def pike_grouped_linear_epilogue(x, w, bias, residual, group_offsets, *, act="no
     e = _epilogue(act, scale, "none", 0.0, out_dtype, FLAG_W_IS_NK if w_is_nk else 0)
     _check(load_library().pike_grouped_linear_epilogue(_handle(x.device), _tensor(x), _tensor(w), _tensor(bias),
                                                        _tensor(residual), ctypes.c_void_p(group_offsets.data_ptr()),
-                                                       ctypes.byref(e), _tensor(out), _stream(stream)),
+                                                       e, _tensor(out), _stream(stream)),
            "pike_grouped_linear_epilogue")
     return out

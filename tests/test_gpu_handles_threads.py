@@ -42,10 +42,10 @@ def test_two_handles_on_two_threads():
                 e1 = B._epilogue("gelu_erf", 1.0, "layernorm", 1e-5, F32, 0)
                 e5 = B._epilogue("none", float(c5["scale"]), "none", 0.0, BF16, B.FLAG_CAUSAL)
                 rc = lib.pike_linear_epilogue(h, B._tensor(x2), B._tensor(w2), B._tensor(b2), B._tensor(r2), None, None,
-                                              ctypes.byref(e2), B._tensor(o2), None, 0, sp)
+                                              e2, B._tensor(o2), None, 0, sp)
                 rc |= lib.pike_linear_epilogue(h, B._tensor(x1), B._tensor(w1), B._tensor(b1), None, None, None,
-                                               ctypes.byref(e1), B._tensor(o1), None, 0, sp)
-                rc |= lib.pike_attention_chain(h, B._tensor(q), B._tensor(k), B._tensor(v), ctypes.byref(e5),
+                                               e1, B._tensor(o1), None, 0, sp)
+                rc |= lib.pike_attention_chain(h, B._tensor(q), B._tensor(k), B._tensor(v), e5,
                                                B._tensor(o5), None, 0, sp)
                 assert rc == 0
                 outs.append((o2, o1, o5))
