@@ -13,6 +13,11 @@ def pytest_configure(config):
 
 
 def pytest_collection_modifyitems(config, items):
+    # no test here needs minutes: one that stops making progress fails after five instead of holding a GPU
+    if config.pluginmanager.hasplugin("timeout"):
+        for item in items:
+            if item.get_closest_marker("timeout") is None:
+                item.add_marker(pytest.mark.timeout(300))
     try:
         import torch
         has_gpu = torch.cuda.is_available()
