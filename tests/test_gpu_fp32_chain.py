@@ -87,3 +87,53 @@ def test_extent_one_dimensions_with_arbitrary_strides(M, K, N):
                                  reduce="layernorm", eps=c["eps"], w_is_nk=True)
     want = O.linear_epilogue(c["x"], c["w"], c["b"], act="gelu_erf", reduce="layernorm", eps=c["eps"])
     check_f32(host64(out), want, 1e-4, f"{M}x{K}x{N} with an extent-1 stride")
+
+
+@pytest.mark.parametrize("M,K,N", [(64, 256, 256), (40, 700, 512), (24, 300, 1000), (9, 520, 96), (128, 64, 1024)])
+@pytest.mark.parametrize("nk", [False, True])
+def test_small_problem_kernel_is_exact_on_integers(M, K, N, nk):
+    """Small integers make every product and partial sum exact in fp32 whatever the summation order, so the k slices,
+    the 4x4 register tiles, the chunks of k (one, or several of 256) and every ragged edge of the small-problem
+    kernel must reproduce the oracle bit for bit, with tiled copies ([K,N] weights, aligned pitches) and without."""
+    import paper_2511_16964_b200 as P
+    rng = np.random.default_rng(M * 7 + K + N + nk)
+    x = rng.integers(-4, 5, (M, K)).astype(np.float32)
+    w = rng.integers(-3, 4, (K, N)).astype(np.float32)
+    b = rng.integers(-8, 9, N).astype(np.float32)
+    r = rng.integers(-8, 9, (M, N)).astype(np.float32)
+    want = O.linear_epilogue(x, w, b, r, act="none", scale=2.0)
+    wd = dev(w.T.copy() if nk else w, F32)
+    got = P.pike_linear_epilogue(dev(x, F32), wd, dev(b, F32), dev(r, F32), act="none", scale=2.0, w_is_nk=nk)
+    assert np.array_equal(host64(got), want)
+    # the same through row pitches that are not multiples of 16 bytes: per-thread copies instead of tiled ones
+    xp = torch.zeros((M, K + 1), device="cuda", dtype=F32)
+    xp[:, :K] = dev(x, F32)
+    wrows, wcols = wd.shape
+    wp = torch.zeros((wrows, wcols + 3), device="cuda", dtype=F32)
+    wp[:, :wcols] = wd
+    got = P.pike_linear_epilogue(xp[:, :K], wp[:, :wcols], dev(b, F32), dev(r, F32), act="none", scale=2.0, w_is_nk=nk)
+    assert np.array_equal(host64(got), want)
+
+
+@pytest.mark.parametrize("reduce", ["layernorm", "softmax"])
+@pytest.mark.parametrize("M,K,N", [(40, 700, 512), (24, 300, 1000), (16, 256, 40)])
+def test_small_problem_kernel_reductions_over_wide_and_ragged_rows(M, K, N, reduce):
+    c = G.config1(M=M, K=K, N=N, seed=11)
+    rng = np.random.default_rng(N)
+    gamma = rng.uniform(0.5, 1.5, N).astype(np.float32)
+    beta = rng.uniform(-0.1, 0.1, N).astype(np.float32)
+    got, want = _run(c, act="silu", reduce=reduce, gamma=gamma, beta=beta)
+    check_f32(got, want, 1e-4, f"{M}x{K}x{N} {reduce}")
+    if reduce == "softmax":
+        assert np.abs(got.sum(axis=1) - 1.0).max() < 1e-5
+
+
+def test_layernorm_statistics_survive_a_mean_that_dwarfs_the_spread():
+    """The one-pass shifted statistics and the pooled merge across the cluster must not lose the variance when
+    every value sits near 100 and the row's spread is about 0.4 (a residual of 100 added to each output).  Bar 2e-4:
+    an fp32 value near 100 carries a rounding error of up to 3.8e-6, which the division by the spread multiplies by 2.5
+    before anything else is counted."""
+    c = G.config1(M=32, K=256, N=512, seed=5)
+    res = np.full((32, 512), 100.0, np.float32)
+    got, want = _run(c, act="gelu_erf", reduce="layernorm", residual=res)
+    check_f32(got, want, 2e-4, "mean 100")
