@@ -13,8 +13,8 @@
 //    shared-memory load of either operand: the shared-memory pipe, not the FMA pipe, bounds a tile this small),
 //    and the slices' partial sums meet in shared memory.  Operands arrive as two tiled copies on one mbarrier
 //    where the tensors allow a tensor map.
-//  - fp32_chain_kernel (BM = 16 or 32; problems that fill the chip): thread (lane, warp) accumulates
-//    columns lane + 32c of rows warp + 8i over all of k.
+//  - fp32_chain_kernel (BM = 16, 32 or 64, 128 columns per CTA; problems that fill the chip): warp = rows
+//    warp + 8i, lane = four adjacent columns, over all of k.
 // The LayerNorm / softmax reduction over N never leaves the cluster: every warp reduces its rows
 // over the CTA's columns with shuffles, the CTAs publish one pair per row - (mean, sum of squared
 // deviations) or (max, sum exp) - in their shared memory, and after one cluster barrier every CTA
@@ -30,7 +30,7 @@ namespace {
 
 constexpr int FT = 256;                    // 8 warps
 constexpr int SMEM_FLOATS_MAX = 24576;     // 96 KiB of shared memory per CTA
-constexpr int MAX_BM = 32;
+constexpr int MAX_BM = 64;
 constexpr int SPLITK_BM = 8;
 
 __device__ __forceinline__ float act_by_id(int act, float y)
@@ -56,18 +56,23 @@ __device__ __forceinline__ float warp_max_f(float x)
     return x;
 }
 
-// The per-column parameters of a thread's columns (n0 + lane + 32c); fetched before the main loop so that
-// their latency hides under it.
+// A thread's c-th column inside the CTA's slice: strided over the warp (lane + 32c), or, ADJ, CW adjacent
+// columns per lane (one 16-byte shared-memory load of W feeds four of them).
+template <int CW, bool ADJ>
+__device__ __forceinline__ int col_in_cta(int lane, int c) { return ADJ ? CW * lane + c : lane + 32 * c; }
+
+// The per-column parameters of a thread's columns; fetched before the main loop so that their latency hides
+// under it.
 template <int CW>
 struct ColParams {
     float bias[CW], gamma[CW], beta[CW];
 };
-template <int CW>
+template <int CW, bool ADJ = false>
 __device__ __forceinline__ void load_col_params(const Fp32ChainArgs &a, int n0, int lane, ColParams<CW> &p)
 {
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-        const int col = n0 + lane + 32 * c;
+        const int col = n0 + col_in_cta<CW, ADJ>(lane, c);
         const bool col_ok = col < a.N;
         p.bias[c] = (a.bias != nullptr && col_ok) ? __ldg(a.bias + col) : 0.0f;
         p.gamma[c] = (a.reduce == 1 && a.gamma != nullptr && col_ok) ? __ldg(a.gamma + col) : 1.0f;
@@ -142,8 +147,8 @@ __device__ __forceinline__ void stage_w_cp_async(const Fp32ChainArgs &a, float *
 }
 
 // ---- from the dot products to the stored output: bias -> activation -> scale -> residual in registers, then
-// the row reduction.  Warp rg owns rows rg + 8i of the block, lane the columns n0 + lane + 32c.
-template <int RPT, int CW>
+// the row reduction.  Warp rg owns rows rg + 8i of the block, lane the columns n0 + col_in_cta(lane, c).
+template <int RPT, int CW, bool ADJ = false>
 __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, float (&v)[RPT][CW],
                                                       const ColParams<CW> &p, float2 *stat, long long row0, int n0,
                                                       int n_loc, int lane, int rg, int cn)
@@ -151,7 +156,7 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
     constexpr int BN = 32 * CW;
 #pragma unroll
     for (int c = 0; c < CW; ++c) {
-        const int col = n0 + lane + 32 * c;
+        const int col = n0 + col_in_cta<CW, ADJ>(lane, c);
         const bool col_ok = col < a.N;
 #pragma unroll
         for (int i = 0; i < RPT; ++i) {
@@ -175,7 +180,7 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
                 float sd = 0.0f, sq = 0.0f;
 #pragma unroll
                 for (int c = 0; c < CW; ++c) {
-                    const float d = (lane + 32 * c < n_loc) ? v[i][c] - v0 : 0.0f;
+                    const float d = (col_in_cta<CW, ADJ>(lane, c) < n_loc) ? v[i][c] - v0 : 0.0f;
                     sd += d;
                     sq = fmaf(d, d, sq);
                 }
@@ -190,11 +195,11 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
             } else {                                   // softmax: (max, sum exp(v - max))
                 float m = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < CW; ++c) m = fmaxf(m, (lane + 32 * c < n_loc) ? v[i][c] : -INFINITY);
+                for (int c = 0; c < CW; ++c) m = fmaxf(m, (col_in_cta<CW, ADJ>(lane, c) < n_loc) ? v[i][c] : -INFINITY);
                 m = warp_max_f(m);
                 float s = 0.0f;
 #pragma unroll
-                for (int c = 0; c < CW; ++c) s += (lane + 32 * c < n_loc) ? expf(v[i][c] - m) : 0.0f;
+                for (int c = 0; c < CW; ++c) s += (col_in_cta<CW, ADJ>(lane, c) < n_loc) ? expf(v[i][c] - m) : 0.0f;
                 s0 = m;
                 s1 = warp_sum_f(s);
             }
@@ -251,7 +256,7 @@ __device__ __forceinline__ void epilogue_reduce_store(const Fp32ChainArgs &a, fl
         const long long row = row0 + rg + 8 * i;
 #pragma unroll
         for (int c = 0; c < CW; ++c) {
-            const int col = n0 + lane + 32 * c;
+            const int col = n0 + col_in_cta<CW, ADJ>(lane, c);
             if (row < a.M && col < a.N) a.out[row * a.ldo + col] = v[i][c];
         }
     }
@@ -393,11 +398,15 @@ __global__ void __launch_bounds__(FT) fp32_chain_splitk_kernel(const Fp32ChainAr
 }
 
 // ---- problems that fill the chip: every thread walks all of k ---------------------------------------
-// RPT rows and CW columns per thread: the CTA tile is (8 RPT) x (32 CW).  NK: w is [N,K].
-template <int RPT, int CW, bool NK>
-__global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, const int kc)
+// CTA tile (8 RPT) x 128: warp rg owns rows rg + 8i, a lane FOUR ADJACENT columns ([K,N] weights: one 16-byte
+// load of W per k feeds 4 RPT FMAs and a 16-byte broadcast of x per row feeds 16, so the FMA pipe rather than
+// the shared-memory pipe sets the pace at RPT = 8) or, for [N,K] weights (staged transposed with an odd pitch),
+// columns lane + 32c.  k ascending per output.  Two CTAs fit an SM and cover each other's staging.
+template <int RPT, bool NK>
+__global__ void __launch_bounds__(FT, 2) fp32_chain_kernel(const Fp32ChainArgs a, const int kc)
 {
-    constexpr int BM = 8 * RPT, BN = 32 * CW;
+    constexpr int CW = 4, BM = 8 * RPT, BN = 32 * CW;
+    constexpr bool ADJ = !NK;
     extern __shared__ __align__(16) float smem[];
     __shared__ float2 stat[MAX_BM];        // this CTA's per-row pair, read by the whole cluster
     float *x_s = smem;                     // [BM][kc]
@@ -410,15 +419,13 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
     const int n_loc = min(max(a.N - n0, 0), BN);      // columns this CTA owns (0 for a padding rank)
     pdl_wait();
 
-    float acc[RPT][CW][4];
+    float acc[RPT][CW];
 #pragma unroll
     for (int i = 0; i < RPT; ++i)
 #pragma unroll
-        for (int c = 0; c < CW; ++c)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[i][c][j] = 0.0f;
+        for (int c = 0; c < CW; ++c) acc[i][c] = 0.0f;
     ColParams<CW> prm;
-    load_col_params<CW>(a, n0, lane, prm);
+    load_col_params<CW, ADJ>(a, n0, lane, prm);
 
     for (int k0 = 0; k0 < a.K; k0 += kc) {
         const int kn = min(kc, a.K - k0);
@@ -428,39 +435,38 @@ __global__ void __launch_bounds__(FT) fp32_chain_kernel(const Fp32ChainArgs a, c
         cp_async_wait_all();
         __syncthreads();
         if (n_loc > 0) {
-            // four k at a time: one 16-byte broadcast load of x per row, four column loads of w, and four
-            // independent accumulators per output (k = 0, 1, 2, 3 mod 4) so that consecutive FMAs do not wait
-            // for one another; the tail of a chunk that is not a multiple of four reads the zeros staged above
+            // four k at a time (the tail of a chunk that is not a multiple of four reads the zeros staged above)
 #pragma unroll 2
             for (int k = 0; k < kn; k += 4) {
                 float4 xv[RPT];
-                float wv[CW][4];
+                float wv[4][CW];                                 // [k offset][column]
 #pragma unroll
                 for (int i = 0; i < RPT; ++i) xv[i] = *reinterpret_cast<const float4 *>(x_s + (rg + 8 * i) * kc + k);
 #pragma unroll
-                for (int c = 0; c < CW; ++c)
+                for (int j = 0; j < 4; ++j) {
+                    if constexpr (NK) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        wv[c][j] = NK ? w_s[(lane + 32 * c) * (kc + 1) + k + j] : w_s[(k + j) * BN + lane + 32 * c];
+                        for (int c = 0; c < CW; ++c) wv[j][c] = w_s[(lane + 32 * c) * (kc + 1) + k + j];
+                    } else {
+                        const float4 t = *reinterpret_cast<const float4 *>(w_s + (k + j) * BN + 4 * lane);
+                        wv[j][0] = t.x; wv[j][1] = t.y; wv[j][2] = t.z; wv[j][3] = t.w;
+                    }
+                }
 #pragma unroll
                 for (int i = 0; i < RPT; ++i)
 #pragma unroll
                     for (int c = 0; c < CW; ++c) {
-                        acc[i][c][0] = fmaf(xv[i].x, wv[c][0], acc[i][c][0]);
-                        acc[i][c][1] = fmaf(xv[i].y, wv[c][1], acc[i][c][1]);
-                        acc[i][c][2] = fmaf(xv[i].z, wv[c][2], acc[i][c][2]);
-                        acc[i][c][3] = fmaf(xv[i].w, wv[c][3], acc[i][c][3]);
+                        float t = acc[i][c];
+                        t = fmaf(xv[i].x, wv[0][c], t);
+                        t = fmaf(xv[i].y, wv[1][c], t);
+                        t = fmaf(xv[i].z, wv[2][c], t);
+                        t = fmaf(xv[i].w, wv[3][c], t);
+                        acc[i][c] = t;
                     }
             }
         }
     }
-
-    float v[RPT][CW];
-#pragma unroll
-    for (int i = 0; i < RPT; ++i)
-#pragma unroll
-        for (int c = 0; c < CW; ++c) v[i][c] = (acc[i][c][0] + acc[i][c][1]) + (acc[i][c][2] + acc[i][c][3]);
-    epilogue_reduce_store<RPT, CW>(a, v, prm, stat, row0, n0, n_loc, lane, rg, cn);
+    epilogue_reduce_store<RPT, CW, ADJ>(a, acc, prm, stat, row0, n0, n_loc, lane, rg, cn);
 }
 
 template <typename Kernel, typename... Extra>
@@ -485,7 +491,7 @@ cudaError_t launch_clusters(Kernel kern, const Fp32ChainArgs &a, int bm, int cn,
 // chunk length along k: what fits the shared memory beside the other operand, a multiple of four
 int chunk_k(int K, int rpt, int cw, bool tiled)
 {
-    const int bm = 8 * rpt, bn = 32 * cw;
+    const int bm = 8 * rpt, bn = 32 * cw;                   // (cw = 4 whenever rpt > 1)
     int kc = rpt == 1 ? ((SMEM_FLOATS_MAX - 16 * SPLITK_BM * 32 - bn - 4) / (bm + bn)) & ~3
                       : (SMEM_FLOATS_MAX / (bm + bn + 1)) & ~3;
     if (tiled && kc > 256) kc = 256;                       // a tensor-map box has at most 256 elements per dimension
@@ -493,12 +499,12 @@ int chunk_k(int K, int rpt, int cw, bool tiled)
     return kc > k4 ? k4 : kc;
 }
 
-template <int RPT, int CW, bool NK>
+template <int RPT, bool NK>
 cudaError_t launch_one(const Fp32ChainArgs &a, const Fp32ChainPlan &p, cudaStream_t stream)
 {
-    constexpr int BM = 8 * RPT, BN = 32 * CW;
+    constexpr int BM = 8 * RPT, BN = 128;
     const size_t smem = sizeof(float) * ((size_t)BM * p.kc + (NK ? (size_t)BN * (p.kc + 1) : (size_t)p.kc * BN));
-    return launch_clusters(fp32_chain_kernel<RPT, CW, NK>, a, BM, p.cn, smem, p.kc, stream);
+    return launch_clusters(fp32_chain_kernel<RPT, NK>, a, BM, p.cn, smem, p.kc, stream);
 }
 
 template <int CW, bool NK>
@@ -511,21 +517,23 @@ cudaError_t launch_splitk(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const 
     return launch_clusters(fp32_chain_splitk_kernel<CW, NK>, a, BM, p.cn, smem, p.kc, stream, p.tma_x, p.tma_w, tm_x, tm_w);
 }
 
-template <int RPT>
-cudaError_t launch_cw(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const CUtensorMap &tm_x, const CUtensorMap &tm_w,
-                      cudaStream_t stream)
+cudaError_t launch_splitk_cw(const Fp32ChainArgs &a, const Fp32ChainPlan &p, const CUtensorMap &tm_x, const CUtensorMap &tm_w,
+                             cudaStream_t stream)
 {
-#define PIKE_FP32_LAUNCH(C)                                                                                          \
-    if constexpr (RPT == 1)                                                                                          \
-        return a.w_is_nk ? launch_splitk<C, true>(a, p, tm_x, tm_w, stream) : launch_splitk<C, false>(a, p, tm_x, tm_w, stream); \
-    else                                                                                                             \
-        return a.w_is_nk ? launch_one<RPT, C, true>(a, p, stream) : launch_one<RPT, C, false>(a, p, stream);
-    switch (p.cw) {
-    case 1:  PIKE_FP32_LAUNCH(1)
-    case 2:  PIKE_FP32_LAUNCH(2)
-    default: PIKE_FP32_LAUNCH(4)
+    switch (p.cw * 2 + (a.w_is_nk ? 1 : 0)) {
+    case 2:  return launch_splitk<1, false>(a, p, tm_x, tm_w, stream);
+    case 3:  return launch_splitk<1, true>(a, p, tm_x, tm_w, stream);
+    case 4:  return launch_splitk<2, false>(a, p, tm_x, tm_w, stream);
+    case 5:  return launch_splitk<2, true>(a, p, tm_x, tm_w, stream);
+    case 8:  return launch_splitk<4, false>(a, p, tm_x, tm_w, stream);
+    default: return launch_splitk<4, true>(a, p, tm_x, tm_w, stream);
     }
-#undef PIKE_FP32_LAUNCH
+}
+
+template <int RPT>
+cudaError_t launch_rows(const Fp32ChainArgs &a, const Fp32ChainPlan &p, cudaStream_t stream)
+{
+    return a.w_is_nk ? launch_one<RPT, true>(a, p, stream) : launch_one<RPT, false>(a, p, stream);
 }
 
 template <typename Kernel>
@@ -540,11 +548,10 @@ cudaError_t raise_smem_limit(Kernel kern)
 cudaError_t setup_fp32_chain()
 {
     cudaError_t e = cudaSuccess;
-#define PIKE_FP32_SETUP(R, C)                                                                     \
-    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, C, false>);                  \
-    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, C, true>);
-    PIKE_FP32_SETUP(2, 1) PIKE_FP32_SETUP(2, 2) PIKE_FP32_SETUP(2, 4)
-    PIKE_FP32_SETUP(4, 1) PIKE_FP32_SETUP(4, 2) PIKE_FP32_SETUP(4, 4)
+#define PIKE_FP32_SETUP(R)                                                                        \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, false>);                     \
+    if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_kernel<R, true>);
+    PIKE_FP32_SETUP(2) PIKE_FP32_SETUP(4) PIKE_FP32_SETUP(8)
 #undef PIKE_FP32_SETUP
 #define PIKE_FP32_SETUP(C)                                                                        \
     if (e == cudaSuccess) e = raise_smem_limit(fp32_chain_splitk_kernel<C, false>);              \
@@ -562,10 +569,20 @@ Fp32ChainPlan plan_fp32_chain(const Fp32ChainArgs &a, int num_sms)
     const int need = (a.N + 32 * p.cw - 1) / (32 * p.cw);
     p.cn = 1;
     while (p.cn < need) p.cn *= 2;                      // power of two; ranks past N own no columns
-    // rows per CTA: small problems spread over as many SMs as they can fill, large ones amortise W over more rows
-    if ((long long)p.cn * ((a.M + 7) / 8) <= 2ll * num_sms) p.rpt = 1;
-    else if ((long long)p.cn * ((a.M + 15) / 16) <= 4ll * num_sms) p.rpt = 2;
-    else p.rpt = 4;
+    // small problems (at most two CTAs of 8 rows per SM) spread over as many SMs as they can with narrow column
+    // slices and split k inside the CTA; everything else takes 128 columns per CTA and as many rows per CTA (64,
+    // 32, 16) as still leave every SM two CTAs
+    if ((long long)p.cn * ((a.M + 7) / 8) <= 2ll * num_sms) {
+        p.rpt = 1;
+    } else {
+        p.cw = 4;
+        const int need128 = (a.N + 127) / 128;
+        p.cn = 1;
+        while (p.cn < need128) p.cn *= 2;
+        if ((long long)p.cn * ((a.M + 63) / 64) >= 2ll * num_sms) p.rpt = 8;
+        else if ((long long)p.cn * ((a.M + 31) / 32) >= 2ll * num_sms) p.rpt = 4;
+        else p.rpt = 2;
+    }
     if (p.rpt == 1) {   // tensor maps want 16-byte aligned bases and row pitches
         p.tma_x = (a.ldx & 3) == 0 && (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
         p.tma_w = !a.w_is_nk && (a.ldw & 3) == 0 && (reinterpret_cast<uintptr_t>(a.w) & 15) == 0;
@@ -584,9 +601,10 @@ cudaError_t launch_fp32_chain(const Fp32ChainArgs &a, const Fp32ChainPlan &p, co
     memset(&none, 0, sizeof(none));
     const CUtensorMap &mx = (p.tma_x && tm_x != nullptr) ? *tm_x : none, &mw = (p.tma_w && tm_w != nullptr) ? *tm_w : none;
     switch (p.rpt) {
-    case 1:  return launch_cw<1>(a, p, mx, mw, stream);
-    case 2:  return launch_cw<2>(a, p, mx, mw, stream);
-    default: return launch_cw<4>(a, p, mx, mw, stream);
+    case 1:  return launch_splitk_cw(a, p, mx, mw, stream);
+    case 2:  return launch_rows<2>(a, p, stream);
+    case 4:  return launch_rows<4>(a, p, stream);
+    default: return launch_rows<8>(a, p, stream);
     }
 }
 
