@@ -807,6 +807,8 @@ def variant_rows(P, torch, device, runs=5):
         "cross attention bf16 B8 H32 S1024 Sk4096 D128": lambda: attn(8, 32, 1024, 4096, 128, BF16, False),
         "linear+GELU+LayerNorm (split-row epilogue) bf16 8192x4096x4096": lambda: linear(8192, 4096, 4096, BF16, act="gelu_tanh", reduce="layernorm"),
         "linear+SiLU+scale+residual f16 4096^3": lambda: linear(4096, 4096, 4096, F16, act="silu", scale=0.5, residual=True),
+        # the fp32 CUDA-core chain on a problem that fills the chip (the path is built for small, latency-bound chains)
+        "linear+GELU(erf)+LayerNorm fp32 8192x1024x1024": lambda: linear(8192, 1024, 1024, F32, act="gelu_erf", reduce="layernorm"),
     }
     rows = {}
     for name, make in cases.items():
@@ -815,6 +817,17 @@ def variant_rows(P, torch, device, runs=5):
             ms = _timed_cold(torch, fn, flush, iters=runs)
             rows[name] = {"ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
                           "frac_of_nominal_2250": fl / (ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS}
+            if " fp32 " in name:     # nominal bf16 tensor peak says nothing about fp32 FMAs: give the unfused eager time instead
+                del rows[name]["frac_of_nominal_2250"]
+                x, w, b = rn(8192, 1024, dt=F32), rn(1024, 1024, dt=F32, sc=1 / 32), rn(1024, dt=F32)
+                gm, be = rn(1024, dt=F32), rn(1024, dt=F32)
+                tf32 = torch.backends.cuda.matmul.allow_tf32
+                torch.backends.cuda.matmul.allow_tf32 = False
+                rows[name]["eager_fp32_ms"] = _timed_cold(
+                    torch, lambda: torch.nn.functional.layer_norm(torch.nn.functional.gelu(x @ w + b), (1024,), gm, be),
+                    flush, iters=runs)
+                torch.backends.cuda.matmul.allow_tf32 = tf32
+                del x, w, b, gm, be
             del fn
         except Exception as exc:           # noqa: BLE001 - a context row must never break the benchmark
             rows[name] = {"ms": None, "error": repr(exc)[:200]}
